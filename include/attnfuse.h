@@ -1,0 +1,123 @@
+/*
+ * attnfuse: the fused attention kernel of a composed variant
+ *     softmax(mask(alibi(rope(Q, K)))) @ V          (paper: Introduction, Sections 3.1 and 4.1)
+ * and its backward pass (Section 4.4), hand-written for sm_100a.
+ *
+ * Conventions for every entry point
+ *  - C linkage, plain pointers and sizes.  Unless a parameter says HOST, data pointers are DEVICE
+ *    pointers owned by the caller; the library allocates no device memory.
+ *  - Tensors are [B, H, S, D] with D contiguous, bf16 (2 bytes per element).  Query-side tensors
+ *    have Hq heads, key/value-side tensors Hkv heads; query head h reads kv head h / gqa_group.
+ *  - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *    and the call returns without synchronising.  Outputs are valid once the stream is.
+ *  - Argument errors are detected before anything is launched, leave outputs untouched and are
+ *    reported by return code; nothing throws or aborts.
+ *  - Device-side waits are bounded.  A wait that runs out makes the kernel return early and
+ *    records a code that attnfuse_device_status() reports; outputs of that launch are undefined.
+ *  - Forward and backward are run-to-run deterministic (no atomics in the data path).
+ */
+#ifndef ATTNFUSE_H_
+#define ATTNFUSE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    AF_OK = 0,
+    AF_ERR_NULL = 1,            /* a required pointer is NULL */
+    AF_ERR_SHAPE = 2,           /* unsupported or inconsistent sizes (D not 64/128, Hq != Hkv*group, ...) */
+    AF_ERR_DTYPE = 3,           /* unsupported element type */
+    AF_ERR_ALIGN = 4,           /* pointer not 16-byte aligned or stride not a multiple of 8 elements */
+    AF_ERR_SPEC = 5,            /* bad RoPE / mask specification */
+    AF_ERR_WORKSPACE = 6,       /* workspace missing or too small */
+    AF_ERR_ARCH = 7,            /* current device is not compute capability 10.x */
+    AF_ERR_CUDA = 8,            /* a CUDA runtime / driver call failed */
+    AF_ERR_DEVICE_TIMEOUT = 9   /* a bounded device-side wait ran out in an earlier launch */
+} af_status;
+
+typedef enum { AF_BF16 = 0, AF_F32 = 1 } af_dtype;
+
+/* Problem geometry.  S is both the query and the key length. */
+typedef struct { int B, Hq, Hkv, S, D; } af_shape;
+
+/* Element strides of an input tensor; the D stride is 1.  NULL where accepted = contiguous. */
+typedef struct { int64_t b, h, s; } af_strides;
+
+/* RoPE (Section 4.1): NeoX half-swap pairing (i, i + rotary_dim/2), frequency theta^(-2i/rotary_dim),
+ * row s of Q and of K sits at position pos_offset + s.  rotary_dim = 0 disables the rotation;
+ * otherwise it must be a multiple of 16 and <= D.  Dims >= rotary_dim pass through. */
+typedef struct { float theta; int rotary_dim; int pos_offset; } af_rope;
+
+/* Post-matmul score modifiers (Section 3.1: causal, sliding_window, alibi).
+ * causal != 0: keep j <= i.  window >= 0: keep |i - j| <= window (with causal: 0 <= i-j <= window);
+ * window < 0: none.  alibi_slopes: DEVICE pointer to Hq floats or NULL; adds slope[h]*(j - i) to
+ * the scaled score. */
+typedef struct { int causal; int window; const float* alibi_slopes; } af_mask;
+
+int         attnfuse_version(void);
+const char* attnfuse_strerror(af_status st);
+
+/* Reads (and clears) the device status word of the current device; synchronises the device.
+ * Returns AF_OK or AF_ERR_DEVICE_TIMEOUT; *detail (HOST, nullable) receives the raw word. */
+af_status attnfuse_device_status(unsigned int* detail);
+
+/* ---- cos/sin table (set-up step of Section 4.1; cached by the caller) --------------------------
+ * table: S * rotary_dim/2 pairs of fp32 {cos, sin}(p * theta^(-2i/rotary_dim)), p = pos_offset + s,
+ * row-major [S][rotary_dim/2]; angles are formed in fp64 before rounding.
+ * attnfuse_rope_table_bytes returns the size the caller must provide (0 when rotary_dim = 0). */
+size_t    attnfuse_rope_table_bytes(int S, int rotary_dim);
+af_status attnfuse_rope_table(const af_rope* rope, int S, void* table, void* cuda_stream);
+
+/* ---- separate RoPE pass (the pre-rotation arm of Section 5.3) -----------------------------------
+ * Rotates every row of x_in [B, n_heads, S, D] (contiguous) into x_out (may alias x_in).
+ * inverse != 0 applies the transpose rotation.  shape->Hq/Hkv are ignored; n_heads is used. */
+af_status attnfuse_rope(const af_shape* shape, int n_heads, const void* x_in, void* x_out,
+                        const af_rope* rope, const void* rope_table, int inverse, void* cuda_stream);
+
+/* ---- fused forward (Sections 2, 4.1) ---------------------------------------------------------------
+ * One kernel: rotate Q and K tiles on chip, S = Q'K'^T, scale, ALiBi, mask, online softmax, O = P V.
+ * q [B,Hq,S,D], k, v [B,Hkv,S,D] bf16 with strides sq / skv (NULL = contiguous).
+ * rope_table: from attnfuse_rope_table for the same (rope, S); may be NULL iff rotary_dim = 0.
+ * o: [B,Hq,S,D] contiguous, o_dtype AF_BF16 or AF_F32.
+ * lse: [B,Hq,S] fp32, L = m + ln(l) (Section 4.4), natural log; nullable. */
+af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, const void* v,
+                       const af_strides* sq, const af_strides* skv,
+                       const af_rope* rope, const void* rope_table, const af_mask* mask,
+                       int gqa_group, float softmax_scale,
+                       void* o, af_dtype o_dtype, float* lse, void* cuda_stream);
+
+/* Same computation with HOST buffers: q, k, v, o (bf16) and lse (nullable) are host pointers
+ * (pinned memory recommended).  `staging` is a DEVICE buffer of at least attnfuse_fwd_host_staging_bytes()
+ * bytes; the call enqueues host-to-device copies, the kernel and device-to-host copies on the stream.
+ * alibi slopes inside `mask` remain a DEVICE pointer. */
+size_t    attnfuse_fwd_host_staging_bytes(const af_shape* shape);
+af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const void* k_host, const void* v_host,
+                            const af_rope* rope, const void* rope_table, const af_mask* mask,
+                            int gqa_group, float softmax_scale,
+                            void* o_host, float* lse_host, void* staging, size_t staging_bytes,
+                            void* cuda_stream);
+
+/* ---- fused backward (Section 4.4) -------------------------------------------------------------------
+ * Three kernels: row-reduced gradients delta = rowsum(dO * O); dK/dV accumulation per key tile;
+ * dQ accumulation per query tile.  Probabilities are recomputed from lse; the rotation is recomputed
+ * on chip and gradients w.r.t. rotated rows are rotated back in the epilogues.
+ * o, d_o: [B,Hq,S,D] bf16 contiguous; lse from the forward.
+ * dq [B,Hq,S,D] (dq_dtype), dk, dv [B,Hkv,S,D] (dkv_dtype), contiguous; dk/dv sum over the group.
+ * workspace: at least attnfuse_bwd_workspace_bytes(shape) bytes (holds delta). */
+size_t    attnfuse_bwd_workspace_bytes(const af_shape* shape);
+af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, const void* v,
+                       const void* o, const float* lse, const void* d_o,
+                       const af_strides* sq, const af_strides* skv,
+                       const af_rope* rope, const void* rope_table, const af_mask* mask,
+                       int gqa_group, float softmax_scale,
+                       void* dq, af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATTNFUSE_H_ */

@@ -1,0 +1,233 @@
+"""ctypes binding with the same names as the C entry points (see include/attnfuse.h)."""
+from __future__ import annotations
+
+import ctypes
+import dataclasses
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libattnfuse.so")
+
+AF_BF16, AF_F32 = 0, 1
+
+
+class AttnFuseError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__("attnfuse error %d: %s" % (code, msg))
+        self.code = code
+
+
+class _Shape(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int), ("Hq", ctypes.c_int), ("Hkv", ctypes.c_int), ("S", ctypes.c_int),
+                ("D", ctypes.c_int)]
+
+
+class _Strides(ctypes.Structure):
+    _fields_ = [("b", ctypes.c_int64), ("h", ctypes.c_int64), ("s", ctypes.c_int64)]
+
+
+class _Rope(ctypes.Structure):
+    _fields_ = [("theta", ctypes.c_float), ("rotary_dim", ctypes.c_int), ("pos_offset", ctypes.c_int)]
+
+
+class _Mask(ctypes.Structure):
+    _fields_ = [("causal", ctypes.c_int), ("window", ctypes.c_int), ("alibi_slopes", ctypes.c_void_p)]
+
+
+@dataclasses.dataclass(frozen=True)
+class RopeSpec:
+    theta: float = 10000.0
+    rotary_dim: int = 0
+    pos_offset: int = 0
+
+
+@dataclasses.dataclass
+class MaskSpec:
+    causal: bool = True
+    window: int = -1
+    alibi_slopes: Optional[torch.Tensor] = None  # fp32 [Hq] on the device
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise AttnFuseError(-1, "libattnfuse.so is not built; run `python -m paper_2609_13612_b200.build`")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        P = ctypes.POINTER
+        L.attnfuse_version.restype = i
+        L.attnfuse_strerror.restype = ctypes.c_char_p
+        L.attnfuse_strerror.argtypes = [i]
+        L.attnfuse_device_status.restype = i
+        L.attnfuse_device_status.argtypes = [P(ctypes.c_uint)]
+        L.attnfuse_rope_table_bytes.restype = sz
+        L.attnfuse_rope_table_bytes.argtypes = [i, i]
+        L.attnfuse_rope_table.restype = i
+        L.attnfuse_rope_table.argtypes = [P(_Rope), i, vp, vp]
+        L.attnfuse_rope.restype = i
+        L.attnfuse_rope.argtypes = [P(_Shape), i, vp, vp, P(_Rope), vp, i, vp]
+        L.attnfuse_fwd.restype = i
+        L.attnfuse_fwd.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp, P(_Mask), i, f,
+                                   vp, i, vp, vp]
+        L.attnfuse_fwd_host_staging_bytes.restype = sz
+        L.attnfuse_fwd_host_staging_bytes.argtypes = [P(_Shape)]
+        L.attnfuse_fwd_host.restype = i
+        L.attnfuse_fwd_host.argtypes = [P(_Shape), vp, vp, vp, P(_Rope), vp, P(_Mask), i, f, vp, vp, vp, sz, vp]
+        L.attnfuse_bwd_workspace_bytes.restype = sz
+        L.attnfuse_bwd_workspace_bytes.argtypes = [P(_Shape)]
+        L.attnfuse_bwd.restype = i
+        L.attnfuse_bwd.argtypes = [P(_Shape), vp, vp, vp, vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp,
+                                   P(_Mask), i, f, vp, i, vp, vp, i, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def _check(code: int):
+    if code != 0:
+        raise AttnFuseError(code, lib().attnfuse_strerror(code).decode())
+
+
+def version() -> int:
+    return lib().attnfuse_version()
+
+
+def device_status() -> Tuple[int, int]:
+    d = ctypes.c_uint(0)
+    code = lib().attnfuse_device_status(ctypes.byref(d))
+    return code, d.value
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _need_cuda(*ts):
+    for t in ts:
+        if t is not None and not t.is_cuda:
+            raise AttnFuseError(-2, "tensor is not on a CUDA device (there is no CPU path)")
+
+
+def _strides(t: torch.Tensor) -> _Strides:
+    assert t.dim() == 4 and t.stride(3) == 1
+    return _Strides(t.stride(0), t.stride(1), t.stride(2))
+
+
+def _mask_struct(mask: MaskSpec) -> _Mask:
+    sl = mask.alibi_slopes
+    if sl is not None:
+        _need_cuda(sl)
+        assert sl.dtype == torch.float32 and sl.is_contiguous()
+    return _Mask(int(bool(mask.causal)), int(mask.window), sl.data_ptr() if sl is not None else None)
+
+
+def rope_table(rope_spec: RopeSpec, S: int, device=None) -> Optional[torch.Tensor]:
+    """cos/sin table [S, rotary_dim/2, 2] fp32 built on the device (None when rotary_dim == 0)."""
+    if rope_spec.rotary_dim == 0:
+        return None
+    n = lib().attnfuse_rope_table_bytes(S, rope_spec.rotary_dim)
+    device = device or torch.device("cuda", torch.cuda.current_device())
+    table = torch.empty(n // 4, dtype=torch.float32, device=device)
+    r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
+    _check(lib().attnfuse_rope_table(ctypes.byref(r), S, table.data_ptr(), _stream()))
+    return table.view(S, rope_spec.rotary_dim // 2, 2)
+
+
+def rope(x: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor], inverse: bool = False,
+         out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Separate RoPE pass over x [B,H,S,D] bf16 (contiguous)."""
+    _need_cuda(x, table, out)
+    assert x.dtype == torch.bfloat16 and x.is_contiguous()
+    B, H, S, D = x.shape
+    out = torch.empty_like(x) if out is None else out
+    assert out.dtype == torch.bfloat16 and out.is_contiguous() and out.shape == x.shape
+    sh = _Shape(B, H, H, S, D)
+    r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
+    _check(lib().attnfuse_rope(ctypes.byref(sh), H, x.data_ptr(), out.data_ptr(), ctypes.byref(r),
+                               table.data_ptr() if table is not None else None, int(bool(inverse)), _stream()))
+    return out
+
+
+def fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor],
+        mask: MaskSpec, softmax_scale: float, out: Optional[torch.Tensor] = None,
+        lse: Optional[torch.Tensor] = None, out_dtype: torch.dtype = torch.bfloat16, want_lse: bool = True):
+    """Fused forward.  q [B,Hq,S,D], k/v [B,Hkv,S,D] bf16 (last dim contiguous).  Returns (o, lse)."""
+    _need_cuda(q, k, v, table, out, lse)
+    assert q.dtype == k.dtype == v.dtype == torch.bfloat16
+    B, Hq, S, D = q.shape
+    Hkv = k.shape[1]
+    assert k.shape == v.shape == (B, Hkv, S, D) and k.stride() == v.stride()
+    if out is None:
+        out = torch.empty((B, Hq, S, D), dtype=out_dtype, device=q.device)
+    if lse is None and want_lse:
+        lse = torch.empty((B, Hq, S), dtype=torch.float32, device=q.device)
+    assert out.is_contiguous() and out.dtype in (torch.bfloat16, torch.float32)
+    sh = _Shape(B, Hq, Hkv, S, D)
+    sq, skv = _strides(q), _strides(k)
+    r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
+    m = _mask_struct(mask)
+    _check(lib().attnfuse_fwd(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), ctypes.byref(sq),
+                              ctypes.byref(skv), ctypes.byref(r), table.data_ptr() if table is not None else None,
+                              ctypes.byref(m), Hq // Hkv, float(softmax_scale), out.data_ptr(),
+                              AF_F32 if out.dtype == torch.float32 else AF_BF16,
+                              lse.data_ptr() if lse is not None else None, _stream()))
+    return out, lse
+
+
+def fwd_host(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor],
+             mask: MaskSpec, softmax_scale: float, out: torch.Tensor, lse: Optional[torch.Tensor],
+             staging: torch.Tensor):
+    """Forward with HOST (pinned) q, k, v, out, lse; `staging` is a device byte buffer."""
+    for t in (q, k, v, out):
+        assert not t.is_cuda and t.is_contiguous() and t.dtype == torch.bfloat16
+    _need_cuda(staging, table)
+    B, Hq, S, D = q.shape
+    Hkv = k.shape[1]
+    sh = _Shape(B, Hq, Hkv, S, D)
+    r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
+    m = _mask_struct(mask)
+    _check(lib().attnfuse_fwd_host(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), ctypes.byref(r),
+                                   table.data_ptr() if table is not None else None, ctypes.byref(m), Hq // Hkv,
+                                   float(softmax_scale), out.data_ptr(),
+                                   lse.data_ptr() if lse is not None else None, staging.data_ptr(),
+                                   staging.numel() * staging.element_size(), _stream()))
+    return out, lse
+
+
+def fwd_host_staging_bytes(B: int, Hq: int, Hkv: int, S: int, D: int) -> int:
+    sh = _Shape(B, Hq, Hkv, S, D)
+    return lib().attnfuse_fwd_host_staging_bytes(ctypes.byref(sh))
+
+
+def bwd(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softmax_scale: float,
+        dq_dtype: torch.dtype = torch.bfloat16, dkv_dtype: torch.dtype = torch.float32, workspace=None):
+    """Fused backward.  Returns (dq, dk, dv)."""
+    _need_cuda(q, k, v, o, lse, d_o, table, workspace)
+    B, Hq, S, D = q.shape
+    Hkv = k.shape[1]
+    assert o.is_contiguous() and d_o.is_contiguous() and lse.is_contiguous()
+    assert o.dtype == d_o.dtype == torch.bfloat16 and lse.dtype == torch.float32
+    sh = _Shape(B, Hq, Hkv, S, D)
+    n_ws = lib().attnfuse_bwd_workspace_bytes(ctypes.byref(sh))
+    if workspace is None:
+        workspace = torch.empty(n_ws, dtype=torch.uint8, device=q.device)
+    dq = torch.empty((B, Hq, S, D), dtype=dq_dtype, device=q.device)
+    dk = torch.empty((B, Hkv, S, D), dtype=dkv_dtype, device=q.device)
+    dv = torch.empty((B, Hkv, S, D), dtype=dkv_dtype, device=q.device)
+    sq, skv = _strides(q), _strides(k)
+    r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
+    m = _mask_struct(mask)
+    code = lambda dt: AF_F32 if dt == torch.float32 else AF_BF16
+    _check(lib().attnfuse_bwd(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                              lse.data_ptr(), d_o.data_ptr(), ctypes.byref(sq), ctypes.byref(skv), ctypes.byref(r),
+                              table.data_ptr() if table is not None else None, ctypes.byref(m), Hq // Hkv,
+                              float(softmax_scale), dq.data_ptr(), code(dq_dtype), dk.data_ptr(), dv.data_ptr(),
+                              code(dkv_dtype), workspace.data_ptr(), workspace.numel(), _stream()))
+    return dq, dk, dv

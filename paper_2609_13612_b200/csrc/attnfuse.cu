@@ -1,0 +1,301 @@
+// Host side of the C-ABI declared in include/attnfuse.h: argument validation, tensor-map
+// encoding, variant selection and launches.  All arithmetic of the path runs in the kernels.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "../../include/attnfuse.h"
+#include "bwd_kernel.cuh"
+#include "fwd_kernel.cuh"
+#include "rope_kernels.cuh"
+
+namespace {
+
+using namespace af;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// Tensor map over a bf16 tensor [B, H, S, D] (D contiguous) with a box of [rows x 64 columns],
+// 128-byte swizzle, zero fill outside the tensor.
+af_status make_tmap(CUtensorMap* tm, const void* ptr, int B, int H, int S, int D, const af_strides& st, int rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return AF_ERR_CUDA;
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(S), static_cast<cuuint64_t>(H),
+                          static_cast<cuuint64_t>(B)};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(st.s) * 2, static_cast<cuuint64_t>(st.h) * 2,
+                             static_cast<cuuint64_t>(st.b) * 2};
+    cuuint32_t box[4] = {static_cast<cuuint32_t>(BOX_COLS), static_cast<cuuint32_t>(rows), 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? AF_OK : AF_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+af_status check_arch() {
+    static int cached = -1;
+    if (cached < 0) {
+        int dev = 0, major = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return AF_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return AF_ERR_CUDA;
+        cached = major;
+    }
+    return cached == 10 ? AF_OK : AF_ERR_ARCH;
+}
+
+af_status check_common(const af_shape* sh, const af_rope* rope, const void* table, const af_mask* mask, int group) {
+    if (!sh || !rope || !mask) return AF_ERR_NULL;
+    if (sh->B < 1 || sh->Hq < 1 || sh->Hkv < 1 || sh->S < 1) return AF_ERR_SHAPE;
+    if (sh->D != 64 && sh->D != 128) return AF_ERR_SHAPE;
+    if (group < 1 || sh->Hkv * group != sh->Hq) return AF_ERR_SHAPE;
+    if (rope->rotary_dim < 0 || rope->rotary_dim > sh->D || (rope->rotary_dim % 16) != 0) return AF_ERR_SPEC;
+    if (rope->rotary_dim > 0 && !(rope->theta > 0.f)) return AF_ERR_SPEC;
+    if (rope->rotary_dim > 0 && !table) return AF_ERR_NULL;
+    if (table && !aligned16(table)) return AF_ERR_ALIGN;
+    return AF_OK;
+}
+
+af_status resolve_strides(const af_strides* in, int H, int S, int D, af_strides* out) {
+    if (in) {
+        *out = *in;
+    } else {
+        out->s = D;
+        out->h = static_cast<int64_t>(S) * D;
+        out->b = static_cast<int64_t>(H) * S * D;
+    }
+    if (out->s < D || out->h < 1 || out->b < 1) return AF_ERR_SHAPE;
+    if ((out->s % 8) || (out->h % 8) || (out->b % 8)) return AF_ERR_ALIGN;
+    return AF_OK;
+}
+
+int env_int(const char* name, int dflt) {
+    const char* v = getenv(name);
+    return v ? atoi(v) : dflt;
+}
+
+template <int D, int NQ, bool ROPE, int KS, int VS>
+af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, FwdParams p,
+                             cudaStream_t stream) {
+    using L = FwdSmem<D, NQ, KS, VS>;
+    auto kern = attn_fwd_kernel<D, NQ, ROPE, KS, VS>;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
+            return AF_ERR_CUDA;
+        configured = true;
+    }
+    p.n_row_blocks = (p.S + BM * NQ - 1) / (BM * NQ);
+    dim3 grid(p.B * p.Hq, p.n_row_blocks, 1);
+    kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, p);
+    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+template <int D>
+af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
+                     cudaStream_t stream) {
+    const int nq = env_int("AF_FWD_NQ", 2);
+    if (nq == 1) {
+        return p.R > 0 ? launch_fwd_variant<D, 1, true, 2, 2>(tq, tk, tv, p, stream)
+                       : launch_fwd_variant<D, 1, false, 2, 2>(tq, tk, tv, p, stream);
+    }
+    return p.R > 0 ? launch_fwd_variant<D, 2, true, 2, 2>(tq, tk, tv, p, stream)
+                   : launch_fwd_variant<D, 2, false, 2, 2>(tq, tk, tv, p, stream);
+}
+
+}  // namespace
+
+extern "C" {
+
+int attnfuse_version(void) { return 100; }
+
+const char* attnfuse_strerror(af_status st) {
+    switch (st) {
+        case AF_OK: return "ok";
+        case AF_ERR_NULL: return "required pointer is NULL";
+        case AF_ERR_SHAPE: return "unsupported or inconsistent shape";
+        case AF_ERR_DTYPE: return "unsupported dtype";
+        case AF_ERR_ALIGN: return "pointer or stride misaligned";
+        case AF_ERR_SPEC: return "bad RoPE or mask specification";
+        case AF_ERR_WORKSPACE: return "workspace missing or too small";
+        case AF_ERR_ARCH: return "device is not compute capability 10.x";
+        case AF_ERR_CUDA: return "CUDA call failed";
+        case AF_ERR_DEVICE_TIMEOUT: return "bounded device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+af_status attnfuse_device_status(unsigned int* detail) {
+    unsigned int w = 0, zero = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return AF_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&w, af::g_device_status, sizeof(w)) != cudaSuccess) return AF_ERR_CUDA;
+    if (w && cudaMemcpyToSymbol(af::g_device_status, &zero, sizeof(zero)) != cudaSuccess) return AF_ERR_CUDA;
+    if (detail) *detail = w;
+    return w ? AF_ERR_DEVICE_TIMEOUT : AF_OK;
+}
+
+size_t attnfuse_rope_table_bytes(int S, int rotary_dim) {
+    if (S < 1 || rotary_dim < 1) return 0;
+    return static_cast<size_t>(S) * (rotary_dim / 2) * sizeof(float2);
+}
+
+af_status attnfuse_rope_table(const af_rope* rope, int S, void* table, void* cuda_stream) {
+    if (!rope) return AF_ERR_NULL;
+    if (S < 1) return AF_ERR_SHAPE;
+    if (rope->rotary_dim < 0 || (rope->rotary_dim % 16) != 0 || rope->rotary_dim > 128) return AF_ERR_SPEC;
+    if (rope->rotary_dim == 0) return AF_OK;
+    if (!(rope->theta > 0.f)) return AF_ERR_SPEC;
+    if (!table) return AF_ERR_NULL;
+    if (!aligned16(table)) return AF_ERR_ALIGN;
+    const long long n = static_cast<long long>(S) * (rope->rotary_dim / 2);
+    const int threads = 256;
+    const unsigned blocks = static_cast<unsigned>((n + threads - 1) / threads);
+    rope_table_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        static_cast<float2*>(table), S, rope->rotary_dim, static_cast<double>(rope->theta), rope->pos_offset);
+    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+af_status attnfuse_rope(const af_shape* shape, int n_heads, const void* x_in, void* x_out, const af_rope* rope,
+                        const void* rope_table, int inverse, void* cuda_stream) {
+    if (!shape || !rope || !x_in || !x_out) return AF_ERR_NULL;
+    if (shape->B < 1 || n_heads < 1 || shape->S < 1 || shape->D < 16 || (shape->D % 8) != 0) return AF_ERR_SHAPE;
+    const int R = rope->rotary_dim, D = shape->D;
+    if (R < 0 || R > D || (R % 16) != 0) return AF_ERR_SPEC;
+    if (R > 0 && !rope_table) return AF_ERR_NULL;
+    if (!aligned16(x_in) || !aligned16(x_out) || (rope_table && !aligned16(rope_table))) return AF_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const long long NH = static_cast<long long>(shape->B) * n_heads;
+    if (R == 0) {
+        if (x_in != x_out &&
+            cudaMemcpyAsync(x_out, x_in, static_cast<size_t>(NH) * shape->S * D * 2, cudaMemcpyDeviceToDevice, stream) !=
+                cudaSuccess)
+            return AF_ERR_CUDA;
+        return AF_OK;
+    }
+    constexpr int HPT = 4;
+    const int per_row = (R >> 4) + ((D - R) >> 3);
+    const long long items = static_cast<long long>(shape->S) * per_row;
+    dim3 grid(static_cast<unsigned>((items + 255) / 256), static_cast<unsigned>((NH + HPT - 1) / HPT), 1);
+    if (grid.y > 65535) return AF_ERR_SHAPE;
+    rope_apply_kernel<HPT><<<grid, 256, 0, stream>>>(static_cast<const uint4*>(x_in), static_cast<uint4*>(x_out),
+                                                     static_cast<const float2*>(rope_table), static_cast<int>(NH),
+                                                     shape->S, D, R, inverse ? -1.f : 1.f);
+    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
+                       const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
+                       int gqa_group, float softmax_scale, void* o, af_dtype o_dtype, float* lse, void* cuda_stream) {
+    af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
+    if (st != AF_OK) return st;
+    if (!q || !k || !v || !o) return AF_ERR_NULL;
+    if (o_dtype != AF_BF16 && o_dtype != AF_F32) return AF_ERR_DTYPE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return AF_ERR_ALIGN;
+    if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return AF_ERR_SPEC;
+    af_strides stq, stkv;
+    if ((st = resolve_strides(sq, shape->Hq, shape->S, shape->D, &stq)) != AF_OK) return st;
+    if ((st = resolve_strides(skv, shape->Hkv, shape->S, shape->D, &stkv)) != AF_OK) return st;
+    if ((st = check_arch()) != AF_OK) return st;
+
+    CUtensorMap tq, tk, tv;
+    if ((st = make_tmap(&tq, q, shape->B, shape->Hq, shape->S, shape->D, stq, BM)) != AF_OK) return st;
+    if ((st = make_tmap(&tk, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, BN)) != AF_OK) return st;
+    if ((st = make_tmap(&tv, v, shape->B, shape->Hkv, shape->S, shape->D, stkv, BN)) != AF_OK) return st;
+
+    FwdParams p;
+    p.B = shape->B; p.Hq = shape->Hq; p.Hkv = shape->Hkv; p.S = shape->S; p.group = gqa_group;
+    p.R = rope->rotary_dim;
+    p.causal = mask->causal ? 1 : 0;
+    p.window = mask->window < 0 ? -1 : (mask->window > shape->S ? shape->S : mask->window);
+    p.scale_log2 = softmax_scale * 1.4426950408889634f;
+    p.slopes = mask->alibi_slopes;
+    p.table = static_cast<const float2*>(rope_table);
+    p.o = o; p.o_f32 = (o_dtype == AF_F32); p.lse = lse;
+    p.n_row_blocks = 0;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    return shape->D == 128 ? launch_fwd<128>(tq, tk, tv, p, stream) : launch_fwd<64>(tq, tk, tv, p, stream);
+}
+
+size_t attnfuse_fwd_host_staging_bytes(const af_shape* shape) {
+    if (!shape) return 0;
+    const size_t qn = static_cast<size_t>(shape->B) * shape->Hq * shape->S * shape->D * 2;
+    const size_t kn = static_cast<size_t>(shape->B) * shape->Hkv * shape->S * shape->D * 2;
+    const size_t ln = static_cast<size_t>(shape->B) * shape->Hq * shape->S * 4;
+    return 2 * qn + 2 * kn + ln + 1024;
+}
+
+af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const void* k_host, const void* v_host,
+                            const af_rope* rope, const void* rope_table, const af_mask* mask, int gqa_group,
+                            float softmax_scale, void* o_host, float* lse_host, void* staging, size_t staging_bytes,
+                            void* cuda_stream) {
+    if (!shape || !q_host || !k_host || !v_host || !o_host || !staging) return AF_ERR_NULL;
+    af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
+    if (st != AF_OK) return st;
+    if (staging_bytes < attnfuse_fwd_host_staging_bytes(shape)) return AF_ERR_WORKSPACE;
+    if (!aligned16(staging)) return AF_ERR_ALIGN;
+    const size_t qn = static_cast<size_t>(shape->B) * shape->Hq * shape->S * shape->D * 2;
+    const size_t kn = static_cast<size_t>(shape->B) * shape->Hkv * shape->S * shape->D * 2;
+    const size_t ln = static_cast<size_t>(shape->B) * shape->Hq * shape->S * 4;
+    uint8_t* base = static_cast<uint8_t*>(staging);
+    uint8_t *dq = base, *dk = dq + qn, *dv = dk + kn, *dob = dv + kn, *dl = dob + qn;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(dq, q_host, qn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return AF_ERR_CUDA;
+    if (cudaMemcpyAsync(dk, k_host, kn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return AF_ERR_CUDA;
+    if (cudaMemcpyAsync(dv, v_host, kn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return AF_ERR_CUDA;
+    st = attnfuse_fwd(shape, dq, dk, dv, nullptr, nullptr, rope, rope_table, mask, gqa_group, softmax_scale, dob,
+                      AF_BF16, lse_host ? reinterpret_cast<float*>(dl) : nullptr, cuda_stream);
+    if (st != AF_OK) return st;
+    if (cudaMemcpyAsync(o_host, dob, qn, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return AF_ERR_CUDA;
+    if (lse_host && cudaMemcpyAsync(lse_host, dl, ln, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return AF_ERR_CUDA;
+    return AF_OK;
+}
+
+size_t attnfuse_bwd_workspace_bytes(const af_shape* shape) {
+    if (!shape) return 0;
+    return static_cast<size_t>(shape->B) * shape->Hq * shape->S * sizeof(float) + 256;
+}
+
+af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,
+                       const float* lse, const void* d_o, const af_strides* sq, const af_strides* skv,
+                       const af_rope* rope, const void* rope_table, const af_mask* mask, int gqa_group,
+                       float softmax_scale, void* dq, af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
+    if (st != AF_OK) return st;
+    if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv) return AF_ERR_NULL;
+    if ((dq_dtype != AF_BF16 && dq_dtype != AF_F32) || (dkv_dtype != AF_BF16 && dkv_dtype != AF_F32))
+        return AF_ERR_DTYPE;
+    if (!workspace || workspace_bytes < attnfuse_bwd_workspace_bytes(shape)) return AF_ERR_WORKSPACE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv) || !aligned16(workspace) || !aligned16(lse))
+        return AF_ERR_ALIGN;
+    if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return AF_ERR_SPEC;
+    af_strides stq, stkv, stc;
+    if ((st = resolve_strides(sq, shape->Hq, shape->S, shape->D, &stq)) != AF_OK) return st;
+    if ((st = resolve_strides(skv, shape->Hkv, shape->S, shape->D, &stkv)) != AF_OK) return st;
+    resolve_strides(nullptr, shape->Hq, shape->S, shape->D, &stc);
+    if ((st = check_arch()) != AF_OK) return st;
+    (void)stc;
+    return AF_ERR_SPEC;  // backward kernels not wired yet
+}
+
+}  // extern "C"

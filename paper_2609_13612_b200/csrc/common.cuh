@@ -1,0 +1,103 @@
+// Shared device-side pieces of the attention kernels: tile geometry, mask classification,
+// and the in-shared-memory RoPE rotation of a TMA-loaded (128-byte swizzled) tile.
+#pragma once
+#include "ptx.cuh"
+
+namespace af {
+
+constexpr int BM = 128;          // query rows per tile (= TMEM lanes, one row per thread)
+constexpr int BN = 128;          // key rows per tile
+constexpr int BOX_COLS = 64;     // bf16 columns per TMA box (128 bytes: one swizzle row)
+constexpr int BOX_BYTES = 128 * 128;  // 128 rows x 128 bytes
+
+struct MaskSpec {
+    int S;
+    int causal;
+    int window;  // < 0: none; host clamps to S
+};
+
+// Key-tile range [jlo, jhi] that a query tile starting at row i0 can see (Section 5: fully masked
+// tiles are skipped).
+__device__ __forceinline__ void tile_range(const MaskSpec& m, int i0, int& jlo, int& jhi) {
+    int ilast = min(i0 + BM - 1, m.S - 1);
+    int hi_row = m.causal ? ilast : (m.window >= 0 ? min(ilast + m.window, m.S - 1) : m.S - 1);
+    int lo_row = m.window >= 0 ? max(0, i0 - m.window) : 0;
+    jlo = lo_row / BN;
+    jhi = hi_row / BN;
+}
+
+// Query-tile range [ilo, ihi] (in tiles of BM rows) that can see the key tile starting at row j0.
+__device__ __forceinline__ void qtile_range(const MaskSpec& m, int j0, int& ilo, int& ihi) {
+    int jlast = min(j0 + BN - 1, m.S - 1);
+    int lo_row = m.causal ? j0 : (m.window >= 0 ? max(0, j0 - m.window) : 0);
+    int hi_row = m.window >= 0 ? min(jlast + m.window, m.S - 1) : m.S - 1;
+    ilo = lo_row / BM;
+    ihi = hi_row / BM;
+}
+
+// True if some (i, j) of the tile pair is masked out, so per-element mask logic is needed.
+__device__ __forceinline__ bool tile_needs_mask(const MaskSpec& m, int i0, int j0) {
+    if (j0 + BN > m.S) return true;
+    if (m.causal && j0 + BN - 1 > i0) return true;
+    if (m.window >= 0) {
+        if (i0 + BM - 1 - j0 > m.window) return true;
+        if (!m.causal && j0 + BN - 1 - i0 > m.window) return true;
+    }
+    return false;
+}
+
+__device__ __forceinline__ bool pair_kept(const MaskSpec& m, int i, int j) {
+    if (j >= m.S) return false;
+    int d = i - j;
+    if (m.causal && d < 0) return false;
+    if (m.window >= 0) {
+        if (d < 0) d = -d;
+        if (d > m.window) return false;
+    }
+    return true;
+}
+
+// Byte offset of the 16-byte chunk `chunk` (8 bf16 columns) of row `r` inside a tile made of
+// D/64 TMA boxes, each [128 rows][64 cols] with the 128-byte swizzle.
+__device__ __forceinline__ uint32_t swz_chunk_offset(int r, int chunk) {
+    return static_cast<uint32_t>((chunk >> 3) * BOX_BYTES + r * 128 + (((chunk & 7) ^ (r & 7)) << 4));
+}
+
+// Rotate one word pair: (a, b) are the bf16x2 words at column pair (d, d + R/2); cs holds
+// {cos0, sin0, cos1, sin1} for the two columns of the word.  sgn = +1 forward, -1 transpose.
+__device__ __forceinline__ void rotate_word(uint32_t& a, uint32_t& b, float c0, float s0, float c1, float s1) {
+    float a0 = bf16lo_to_f32(a), a1 = bf16hi_to_f32(a);
+    float b0 = bf16lo_to_f32(b), b1 = bf16hi_to_f32(b);
+    float na0 = fmaf(a0, c0, -b0 * s0), nb0 = fmaf(b0, c0, a0 * s0);
+    float na1 = fmaf(a1, c1, -b1 * s1), nb1 = fmaf(b1, c1, a1 * s1);
+    a = pack_bf16x2(na0, na1);
+    b = pack_bf16x2(nb0, nb1);
+}
+
+// Section 4.1: rotate, in place, the first R columns of a [128 x D] bf16 tile that TMA left in
+// shared memory; row r of the tile sits at table row min(row0 + r, S-1).  Called by `nthreads`
+// threads with ids tid = 0..nthreads-1.  Column d pairs with d + R/2 (NeoX half-swap); both
+// partners of 8 consecutive columns are one 16-byte chunk each, read and written by the same
+// thread, so no shuffle and no second global load is needed.
+__device__ __forceinline__ void rotate_tile_smem(uint8_t* tile, int row0, int S, int R, const float2* table,
+                                                 int tid, int nthreads) {
+    const int CP = R >> 4;  // chunk pairs per row
+    const int half = R >> 1;
+    for (int idx = tid; idx < 128 * CP; idx += nthreads) {
+        int r = idx / CP, cp = idx - r * CP;
+        int prow = min(row0 + r, S - 1);
+        const float4* tb = reinterpret_cast<const float4*>(table + static_cast<size_t>(prow) * half + cp * 8);
+        float4 t0 = __ldg(tb), t1 = __ldg(tb + 1), t2 = __ldg(tb + 2), t3 = __ldg(tb + 3);
+        uint4* pl = reinterpret_cast<uint4*>(tile + swz_chunk_offset(r, cp));
+        uint4* ph = reinterpret_cast<uint4*>(tile + swz_chunk_offset(r, cp + CP));
+        uint4 lo = *pl, hi = *ph;
+        rotate_word(lo.x, hi.x, t0.x, t0.y, t0.z, t0.w);
+        rotate_word(lo.y, hi.y, t1.x, t1.y, t1.z, t1.w);
+        rotate_word(lo.z, hi.z, t2.x, t2.y, t2.z, t2.w);
+        rotate_word(lo.w, hi.w, t3.x, t3.y, t3.z, t3.w);
+        *pl = lo;
+        *ph = hi;
+    }
+}
+
+}  // namespace af

@@ -1,0 +1,366 @@
+// Fused forward kernel (Sections 2 and 4.1): per CTA, NQ query tiles of 128 rows of one head.
+//   TMA -> shared memory (128-byte swizzle) -> RoPE rotation in place -> tcgen05.mma S = Q'K'^T into
+//   TMEM -> scale / ALiBi / mask / online softmax in registers (one query row per thread) ->
+//   P (bf16) back into TMEM over S -> tcgen05.mma O += P V -> normalise, store O and L.
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer (one elected thread each), warps 4-7 rotate
+// Q once and every K tile, warps 8.. are one softmax warpgroup per query tile.
+#pragma once
+#include <cuda.h>
+#include "common.cuh"
+
+namespace af {
+
+struct FwdParams {
+    int B, Hq, Hkv, S, group;
+    int R;              // rotary dim (0: none)
+    int causal, window;
+    float scale_log2;   // softmax scale * log2(e)
+    const float* slopes;  // Hq ALiBi slopes or nullptr
+    const float2* table;  // [S][R/2] {cos, sin}
+    void* o;
+    int o_f32;
+    float* lse;         // nullable
+    int n_row_blocks;   // ceil(S / (128 * NQ))
+};
+
+template <int D, int NQ, int KS, int VS>
+struct FwdSmem {
+    static constexpr int TILE = 128 * D * 2;
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = OFF_Q + NQ * TILE;
+    static constexpr int OFF_V = OFF_K + KS * TILE;
+    static constexpr int OFF_BAR = OFF_V + VS * TILE;
+    // barrier slots
+    static constexpr int B_QFULL = 0, B_QROT = B_QFULL + NQ, B_KFULL = B_QROT + NQ, B_KROT = B_KFULL + KS,
+                         B_KEMPTY = B_KROT + KS, B_VFULL = B_KEMPTY + KS, B_VEMPTY = B_VFULL + VS,
+                         B_SFULL = B_VEMPTY + VS, B_PREADY = B_SFULL + NQ, B_ODONE = B_PREADY + NQ,
+                         N_BARS = B_ODONE + NQ;
+    static constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;
+    static constexpr int BYTES = OFF_MISC + 16 + 1024;  // + alignment slack
+};
+
+constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the row max grows by more
+
+template <int D, int NQ, bool ROPE, int KS, int VS>
+__global__ void __launch_bounds__(128 * (2 + NQ), 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const FwdParams p) {
+    using L = FwdSmem<D, NQ, KS, VS>;
+    constexpr int TILE = L::TILE;
+    constexpr int NBOX = D / BOX_COLS;
+    constexpr uint32_t TMEM_COLS = (NQ * (BN + D) <= 256) ? 256u : 512u;
+    constexpr uint32_t IDESC_S = idesc_bf16_f32(BM, BN, 0, 0);
+    constexpr uint32_t IDESC_O = idesc_bf16_f32(BM, D, 0, 1);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sQ = smem + L::OFF_Q;
+    uint8_t* sK = smem + L::OFF_K;
+    uint8_t* sV = smem + L::OFF_V;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_MISC + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bh = blockIdx.x, b = bh / p.Hq, h = bh - b * p.Hq, hk = h / p.group;
+    const int rb = p.n_row_blocks - 1 - static_cast<int>(blockIdx.y);  // heaviest (last) row blocks first
+    const MaskSpec ms{p.S, p.causal, p.window};
+
+    int i0[NQ], jlo[NQ], jhi[NQ];
+    int jlo_c = 0x7fffffff, jhi_c = -1;
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        i0[q] = (rb * NQ + q) * BM;
+        if (i0[q] < p.S) {
+            tile_range(ms, i0[q], jlo[q], jhi[q]);
+            jlo_c = min(jlo_c, jlo[q]);
+            jhi_c = max(jhi_c, jhi[q]);
+        } else {
+            jlo[q] = 1;
+            jhi[q] = 0;  // empty
+        }
+    }
+    const int n_it = jhi_c - jlo_c + 1;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < L::N_BARS; ++i) {
+            uint32_t cnt = 1;
+            if ((i >= L::B_QROT && i < L::B_QROT + NQ) || (i >= L::B_KROT && i < L::B_KROT + KS) ||
+                (i >= L::B_PREADY && i < L::B_PREADY + NQ))
+                cnt = 128;
+            mbar_init(&bars[i], cnt);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            prefetch_tmap(&tm_q);
+            prefetch_tmap(&tm_k);
+            prefetch_tmap(&tm_v);
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                if (jhi[q] < jlo[q]) continue;
+                mbar_arrive_expect_tx(&bars[L::B_QFULL + q], TILE);
+#pragma unroll
+                for (int bx = 0; bx < NBOX; ++bx)
+                    tma_load_4d(sQ + q * TILE + bx * BOX_BYTES, &tm_q, &bars[L::B_QFULL + q], bx * BOX_COLS, i0[q], h, b);
+            }
+            for (int it = 0; it < n_it; ++it) {
+                const int j0 = (jlo_c + it) * BN;
+                const int ks = it % KS, vs = it % VS;
+                if (!mbar_wait(&bars[L::B_KEMPTY + ks], ((it / KS) & 1) ^ 1, abort_flag, 1)) break;
+                mbar_arrive_expect_tx(&bars[L::B_KFULL + ks], TILE);
+#pragma unroll
+                for (int bx = 0; bx < NBOX; ++bx)
+                    tma_load_4d(sK + ks * TILE + bx * BOX_BYTES, &tm_k, &bars[L::B_KFULL + ks], bx * BOX_COLS, j0, hk, b);
+                if (!mbar_wait(&bars[L::B_VEMPTY + vs], ((it / VS) & 1) ^ 1, abort_flag, 2)) break;
+                mbar_arrive_expect_tx(&bars[L::B_VFULL + vs], TILE);
+#pragma unroll
+                for (int bx = 0; bx < NBOX; ++bx)
+                    tma_load_4d(sV + vs * TILE + bx * BOX_BYTES, &tm_v, &bars[L::B_VFULL + vs], bx * BOX_COLS, j0, hk, b);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr int B_KREADY = ROPE ? L::B_KROT : L::B_KFULL;
+            constexpr int B_QREADY = ROPE ? L::B_QROT : L::B_QFULL;
+            int cnt[NQ];
+            bool ok = true;
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) cnt[q] = 0;
+
+            auto issue_S = [&](int q, int ks) {
+                const uint32_t qa = smem_u32(sQ + q * TILE), ka = smem_u32(sK + ks * TILE);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
+                    mma_ss(tmem_base + q * BN, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024),
+                           IDESC_S, kk > 0);
+                }
+                mma_commit(&bars[L::B_SFULL + q]);
+            };
+            auto issue_O = [&](int q, int vs, bool acc) {
+                const uint32_t va = smem_u32(sV + vs * TILE);
+#pragma unroll
+                for (int kk = 0; kk < BN / 16; ++kk) {
+                    // V is [BN key rows][D]: MN-major B operand; 16 key rows per step = 2 KB
+                    mma_ts(tmem_base + NQ * BN + q * D, tmem_base + q * BN + kk * 8,
+                           smem_desc_sw128(va + kk * 2048, BOX_BYTES, 1024), IDESC_O, (acc || kk > 0) ? 1u : 0u);
+                }
+            };
+
+            // prologue: S of the first key tile
+#pragma unroll
+            for (int q = 0; q < NQ; ++q)
+                if (ok && jhi[q] >= jlo[q]) ok = mbar_wait(&bars[B_QREADY + q], 0, abort_flag, 3);
+            if (ok) ok = mbar_wait(&bars[B_KREADY + 0], 0, abort_flag, 4);
+            if (ok) {
+                tc_fence_after_sync();
+#pragma unroll
+                for (int q = 0; q < NQ; ++q)
+                    if (jlo_c >= jlo[q] && jlo_c <= jhi[q]) issue_S(q, 0);
+                mma_commit(&bars[L::B_KEMPTY + 0]);
+            }
+            for (int it = 0; ok && it < n_it; ++it) {
+                const int j = jlo_c + it, vs = it % VS, ks1 = (it + 1) % KS;
+                const bool next = it + 1 < n_it;
+                bool kwaited = false;
+                ok = mbar_wait(&bars[L::B_VFULL + vs], (it / VS) & 1, abort_flag, 5);
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    if (ok && j >= jlo[q] && j <= jhi[q]) {
+                        ok = mbar_wait(&bars[L::B_PREADY + q], cnt[q] & 1, abort_flag, 6);
+                        if (ok) {
+                            tc_fence_after_sync();
+                            issue_O(q, vs, cnt[q] > 0);
+                            ++cnt[q];
+                            if (j == jhi[q]) mma_commit(&bars[L::B_ODONE + q]);
+                        }
+                    }
+                    if (ok && next && j + 1 >= jlo[q] && j + 1 <= jhi[q]) {
+                        if (!kwaited) {
+                            ok = mbar_wait(&bars[B_KREADY + ks1], ((it + 1) / KS) & 1, abort_flag, 7);
+                            tc_fence_after_sync();
+                            kwaited = true;
+                        }
+                        if (ok) issue_S(q, ks1);
+                    }
+                }
+                if (ok) {
+                    mma_commit(&bars[L::B_VEMPTY + vs]);
+                    if (next) mma_commit(&bars[L::B_KEMPTY + ks1]);
+                }
+            }
+        }
+    } else if (warp >= 4 && warp < 8) {
+        // ------------------------------------------------------------ rotation warpgroup (Section 4.1)
+        if (ROPE) {
+            const int t = threadIdx.x - 128;
+            bool ok = true;
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                if (!ok || jhi[q] < jlo[q]) continue;
+                ok = mbar_wait(&bars[L::B_QFULL + q], 0, abort_flag, 8);
+                if (!ok) break;
+                rotate_tile_smem(sQ + q * TILE, i0[q], p.S, p.R, p.table, t, 128);
+                fence_proxy_async_smem();
+                mbar_arrive(&bars[L::B_QROT + q]);
+            }
+            for (int it = 0; ok && it < n_it; ++it) {
+                const int ks = it % KS;
+                ok = mbar_wait(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
+                if (!ok) break;
+                rotate_tile_smem(sK + ks * TILE, (jlo_c + it) * BN, p.S, p.R, p.table, t, 128);
+                fence_proxy_async_smem();
+                mbar_arrive(&bars[L::B_KROT + ks]);
+            }
+        }
+    } else if (warp >= 8) {
+        // ------------------------------------------------------------ softmax warpgroups (one query row per thread)
+        const int q = (warp - 8) >> 2;
+        const int row = threadIdx.x - 256 - q * 128;            // == TMEM lane
+        const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + lane_addr + q * BN;      // S (fp32) and, over it, P (bf16x2)
+        const uint32_t tO = tmem_base + lane_addr + NQ * BN + q * D;
+        const int i = i0[q] + row;
+        const float slope2 = p.slopes ? p.slopes[h] * 1.4426950408889634f : 0.f;
+        const bool alibi = p.slopes != nullptr;
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        int n = 0;
+        for (int j = jlo[q]; ok && j <= jhi[q]; ++j, ++n) {
+            const int j0 = j * BN;
+            ok = mbar_wait(&bars[L::B_SFULL + q], n & 1, abort_flag, 10);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const bool need_mask = tile_needs_mask(ms, i0[q], j0);
+            const float bias0 = slope2 * static_cast<float>(j0 - i);
+
+            // pass 1: row max of the modified scores (log2 domain)
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tS + c * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    float t = __uint_as_float(v[e]) * p.scale_log2;
+                    if (alibi) t = fmaf(slope2, static_cast<float>(c * 32 + e), t + bias0);
+                    if (need_mask && !pair_kept(ms, i, j0 + c * 32 + e)) t = -INFINITY;
+                    mx = fmaxf(mx, t);
+                }
+            }
+            // lazy rescale: keep the old reference max unless it grew by more than the threshold
+            const bool upd = mx > m_run + kRescaleThreshold;
+            float alpha = 1.f;
+            if (upd) {
+                alpha = ex2(m_run - mx);  // m_run = -inf -> 0
+                m_run = mx;
+            }
+            if (n > 0 && __any_sync(0xffffffffu, upd)) {
+#pragma unroll 1
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tO + c * 32, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                    tmem_st32(tO + c * 32, v);
+                }
+                tmem_wait_st();
+            }
+            l_run *= alpha;
+            const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+            const float nbias = bias0 - m_use;
+
+            // pass 2: p = 2^(t - m), row sum in fp32, P rounded to bf16 into TMEM (over S)
+            float psum = 0.f;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32], pk[16];
+                tmem_ld32(tS + c * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    float t0, t1;
+                    if (alibi) {
+                        t0 = fmaf(__uint_as_float(v[e]), p.scale_log2, fmaf(slope2, static_cast<float>(c * 32 + e), nbias));
+                        t1 = fmaf(__uint_as_float(v[e + 1]), p.scale_log2,
+                                  fmaf(slope2, static_cast<float>(c * 32 + e + 1), nbias));
+                    } else {
+                        t0 = fmaf(__uint_as_float(v[e]), p.scale_log2, -m_use);
+                        t1 = fmaf(__uint_as_float(v[e + 1]), p.scale_log2, -m_use);
+                    }
+                    if (need_mask) {
+                        if (!pair_kept(ms, i, j0 + c * 32 + e)) t0 = -INFINITY;
+                        if (!pair_kept(ms, i, j0 + c * 32 + e + 1)) t1 = -INFINITY;
+                    }
+                    const float p0 = ex2(t0), p1 = ex2(t1);
+                    psum += p0 + p1;
+                    pk[e >> 1] = pack_bf16x2(p0, p1);
+                }
+                tmem_st16(tS + c * 16, pk);
+            }
+            l_run += psum;
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(&bars[L::B_PREADY + q]);
+        }
+        // epilogue (Section 4.4: save L = m + ln l)
+        if (ok && jhi[q] >= jlo[q]) ok = mbar_wait(&bars[L::B_ODONE + q], 0, abort_flag, 11);
+        if (ok && jhi[q] >= jlo[q]) {
+            tc_fence_after_sync();
+            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            const size_t orow = (static_cast<size_t>(bh) * p.S + i) * D;
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tO + c * 32, v);
+                tmem_wait_ld();
+                if (i < p.S) {
+                    if (p.o_f32) {
+                        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + orow + c * 32);
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            dst[e >> 2] = make_float4(__uint_as_float(v[e]) * inv, __uint_as_float(v[e + 1]) * inv,
+                                                      __uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
+                    } else {
+                        uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.o) + orow + c * 32);
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8)
+                            dst[e >> 3] = make_uint4(
+                                pack_bf16x2(__uint_as_float(v[e]) * inv, __uint_as_float(v[e + 1]) * inv),
+                                pack_bf16x2(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv),
+                                pack_bf16x2(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv),
+                                pack_bf16x2(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv));
+                    }
+                }
+            }
+            if (p.lse && i < p.S)
+                p.lse[static_cast<size_t>(bh) * p.S + i] =
+                    l_run > 0.f ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace af

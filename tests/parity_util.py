@@ -1,0 +1,67 @@
+"""Helpers for the GPU parity tests: move seeded inputs to the device, run the CUDA path through
+the C-ABI binding, run the oracle on the same numbers, compare."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+import paper_2609_13612_b200 as af
+from paper_2609_13612_b200 import synth
+
+# Tolerance of the bf16-in / fp32-accumulate path against the fp64 oracle.
+MAX_ABS_TOL = 2e-2
+MEAN_ABS_TOL = 2e-3
+LSE_TOL = 1e-2
+
+
+def to_dev(x: np.ndarray) -> torch.Tensor:
+    """fp32 numpy array of bf16-representable values -> bf16 CUDA tensor (bit exact)."""
+    bits = synth.bf16_bits(x)
+    return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def to_np(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def specs(w: synth.Workload):
+    rope = af.RopeSpec(theta=w.theta, rotary_dim=w.R, pos_offset=w.pos_offset)
+    sl = w.alibi_slopes()
+    mask = af.MaskSpec(causal=w.causal, window=w.window,
+                       alibi_slopes=torch.from_numpy(sl).cuda() if sl is not None else None)
+    return rope, mask
+
+
+def gpu_fwd(w: synth.Workload, dev: dict, out_dtype=torch.bfloat16):
+    rope, mask = specs(w)
+    table = af.rope_table(rope, w.S)
+    o, lse = af.fwd(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale, out_dtype=out_dtype)
+    torch.cuda.synchronize()
+    code, detail = af.device_status()
+    assert code == 0, "device-side wait ran out: 0x%x" % detail
+    return o, lse
+
+
+def gpu_bwd(w: synth.Workload, dev: dict, o, lse, dq_dtype=torch.bfloat16, dkv_dtype=torch.float32):
+    rope, mask = specs(w)
+    table = af.rope_table(rope, w.S)
+    out = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale,
+                 dq_dtype=dq_dtype, dkv_dtype=dkv_dtype)
+    torch.cuda.synchronize()
+    code, detail = af.device_status()
+    assert code == 0, "device-side wait ran out: 0x%x" % detail
+    return out
+
+
+def err(got: np.ndarray, want: np.ndarray):
+    d = np.abs(got - want)
+    return float(d.max()), float(d.mean())
+
+
+def assert_close(name, got, want, max_tol=MAX_ABS_TOL, mean_tol=MEAN_ABS_TOL):
+    assert np.isfinite(got).all(), "%s has non-finite values" % name
+    mx, mean = err(got, want)
+    assert mx <= max_tol and mean <= mean_tol, "%s: max abs %.4g (tol %g), mean abs %.4g (tol %g)" % (
+        name, mx, max_tol, mean, mean_tol)
+    return mx, mean

@@ -1,0 +1,155 @@
+"""GPU parity of the fused forward and of the separate RoPE pass against the fp64 oracle,
+element by element on the same seeded inputs, through the C-ABI binding."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_13612_b200 as af
+from paper_2609_13612_b200 import synth
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+W = synth.Workload
+
+SMALL = [
+    W("norope_dense_1tile", 1, 1, 1, 128, 128, rotary_dim=0, causal=False, seed_id=101),
+    W("norope_causal_gqa", 2, 4, 2, 512, 128, rotary_dim=0, seed_id=102),
+    W("rope_causal_1tile", 1, 1, 1, 128, 128, theta=1e4, seed_id=103),
+    W("rope_causal_gqa4", 1, 8, 2, 640, 128, theta=5e5, seed_id=104),
+    W("rope_causal_d64", 2, 4, 4, 384, 64, theta=1e4, seed_id=105),
+    W("rope_dense_d64", 1, 2, 1, 300, 64, theta=1e4, causal=False, seed_id=106),
+    W("ragged_tail", 1, 4, 1, 333, 128, theta=1e4, seed_id=107),
+    W("shorter_than_tile", 1, 2, 2, 37, 128, theta=1e4, seed_id=108),
+    W("single_row", 1, 2, 1, 1, 64, theta=1e4, seed_id=109),
+    W("window_alibi", 1, 4, 2, 700, 128, theta=1e4, window=200, alibi=True, seed_id=110),
+    W("window_small", 1, 2, 2, 520, 128, theta=1e4, window=5, seed_id=111),
+    W("window_zero", 1, 2, 2, 260, 64, theta=1e4, window=0, seed_id=112),
+    W("window_noncausal", 1, 2, 1, 515, 128, theta=1e4, causal=False, window=130, seed_id=113),
+    W("alibi_noncausal", 1, 4, 4, 260, 128, theta=1e4, causal=False, alibi=True, seed_id=114),
+    W("partial_rotary", 1, 2, 2, 256, 128, theta=1e4, rotary_dim=64, seed_id=115),
+    W("partial_rotary_48_of_64", 1, 2, 2, 200, 64, theta=1e4, rotary_dim=48, seed_id=116),
+    W("pos_offset", 1, 2, 1, 384, 128, theta=5e5, pos_offset=1000, seed_id=117),
+    W("pos_offset_large", 1, 2, 1, 256, 128, theta=5e5, pos_offset=32768 - 256, sigma=0.5, seed_id=118),
+]
+
+
+def run_case(w, out_dtype=torch.bfloat16, nq=None, monkeypatch=None):
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    # poison outputs: a kernel that skips rows leaves NaNs behind
+    o = torch.full((w.B, w.Hq, w.S, w.D), float("nan"), dtype=out_dtype, device="cuda")
+    lse = torch.full((w.B, w.Hq, w.S), float("nan"), dtype=torch.float32, device="cuda")
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S)
+    af.fwd(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale, out=o, lse=lse)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    want_o, want_l = oracle.run_workload(w, t)
+    pu.assert_close(w.name + " O", pu.to_np(o), want_o)
+    got_l = pu.to_np(lse)
+    assert np.isfinite(got_l).all()
+    assert np.abs(got_l - want_l).max() <= pu.LSE_TOL
+
+
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: w.name)
+def test_forward_small(w):
+    run_case(w)
+
+
+@pytest.mark.parametrize("w", SMALL[3:8], ids=lambda w: w.name)
+def test_forward_small_one_query_tile_per_cta(w, monkeypatch):
+    monkeypatch.setenv("AF_FWD_NQ", "1")
+    run_case(w)
+
+
+def test_forward_fp32_output():
+    run_case(W("fp32_out", 1, 4, 2, 300, 128, theta=1e4, seed_id=120), out_dtype=torch.float32)
+
+
+def test_forward_strided_inputs():
+    """q, k, v given as [B,S,H,D] storage viewed as [B,H,S,D] (the layout projection GEMMs produce)."""
+    w = W("strided", 2, 4, 2, 260, 128, theta=1e4, seed_id=121)
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    perm = {k: v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3) for k, v in dev.items()}
+    assert not perm["q"].is_contiguous()
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S)
+    o, lse = af.fwd(perm["q"], perm["k"], perm["v"], rope, table, mask, w.scale)
+    o2, lse2 = af.fwd(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o2) and torch.equal(lse, lse2)
+
+
+def test_forward_is_deterministic_and_guard_bands_stay_intact():
+    w = W("guard", 1, 4, 2, 333, 128, theta=1e4, seed_id=122)
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S)
+    n = w.B * w.Hq * w.S * w.D
+    pad = 4096
+    buf = torch.full((n + 2 * pad,), 7.0, dtype=torch.bfloat16, device="cuda")
+    o = buf[pad:pad + n].view(w.B, w.Hq, w.S, w.D)
+    af.fwd(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale, out=o)
+    first = o.clone()
+    af.fwd(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale, out=o)
+    torch.cuda.synchronize()
+    assert torch.equal(first, o)
+    assert (buf[:pad] == 7.0).all() and (buf[pad + n:] == 7.0).all()
+
+
+def test_fused_equals_separate_rope_then_plain_attention():
+    """The pre-rotation arm: rotate Q and K with the separate kernel, then run the same
+    attention kernel with the rotation switched off."""
+    w = W("separate", 1, 8, 2, 640, 128, theta=5e5, seed_id=123)
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S)
+    qr = af.rope(dev["q"], rope, table)
+    kr = af.rope(dev["k"], rope, table)
+    o_sep, lse_sep = af.fwd(qr, kr, dev["v"], af.RopeSpec(), None, mask, w.scale)
+    o_fus, lse_fus = af.fwd(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale)
+    torch.cuda.synchronize()
+    # identical rounding points (rotated rows rounded to bf16 before the MMA) => identical bits
+    assert torch.equal(o_sep, o_fus) and torch.equal(lse_sep, lse_fus)
+    want_o, _ = oracle.run_workload(w, t)
+    pu.assert_close("separate O", pu.to_np(o_sep), want_o)
+
+
+@pytest.mark.parametrize("R,inverse,D", [(128, False, 128), (64, False, 128), (128, True, 128), (64, False, 64),
+                                         (48, True, 64)])
+def test_rope_kernel_matches_oracle(R, inverse, D):
+    w = W("rope", 2, 5, 5, 301, D, theta=5e5, seed_id=130 + R)
+    x = synth.draw(w, "q")
+    rs = af.RopeSpec(theta=w.theta, rotary_dim=R, pos_offset=77)
+    table = af.rope_table(rs, w.S)
+    y = af.rope(pu.to_dev(x), rs, table, inverse=inverse)
+    torch.cuda.synchronize()
+    want = oracle.rope(x, w.theta, R, 77, inverse=inverse)
+    got = pu.to_np(y)
+    # output is bf16: half an ulp of the largest magnitude (< 8) is 2^-6
+    assert np.abs(got - want).max() <= 2.0 ** -6 + 1e-6
+    assert np.abs(got - want).mean() <= 2e-3
+    # in place gives the same bits
+    xd = pu.to_dev(x)
+    af.rope(xd, rs, table, inverse=inverse, out=xd)
+    torch.cuda.synchronize()
+    assert torch.equal(xd, y)
+
+
+def test_rope_table_against_fp64_formula():
+    rs = af.RopeSpec(theta=500000.0, rotary_dim=128, pos_offset=32768 - 512)
+    table = af.rope_table(rs, 512)
+    torch.cuda.synchronize()
+    pos = rs.pos_offset + np.arange(512)[:, None]
+    freq = 500000.0 ** (-2.0 * np.arange(64) / 128)
+    assert np.abs(pu.to_np(table[..., 0]) - np.cos(pos * freq)).max() < 1e-7
+    assert np.abs(pu.to_np(table[..., 1]) - np.sin(pos * freq)).max() < 1e-7
+
+
+def test_config1_tiny_and_config2_full():
+    for w in synth.CONFIGS[:2]:
+        run_case(w)
