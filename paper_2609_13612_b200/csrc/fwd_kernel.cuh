@@ -41,6 +41,77 @@ struct FwdSmem {
 
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the row max grows by more
 
+// One key tile of the online softmax for one query row (this thread's TMEM lane):
+// reads the 128 raw scores, applies scale / ALiBi / mask in the log2 domain, updates the running
+// max and sum, writes P (bf16) over S and, when the reference max moved, rescales O.
+// MASKED / ALIBI select straight-line code: interior tiles carry no mask logic at all.
+template <int D, bool MASKED, bool ALIBI>
+__device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, float scale_log2, float slope2,
+                                             float bias0, int i, int j0, const MaskSpec& ms, float& m_run,
+                                             float& l_run) {
+    uint32_t v[BN];
+    tmem_ld32(tS, v);
+    tmem_ld32(tS + 32, v + 32);
+    tmem_ld32(tS + 64, v + 64);
+    tmem_ld32(tS + 96, v + 96);
+    tmem_wait_ld();
+    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    if (!MASKED && !ALIBI) {
+#pragma unroll
+        for (int e = 0; e < BN; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(v[e]));
+    } else {
+#pragma unroll
+        for (int e = 0; e < BN; ++e) {
+            float t = __uint_as_float(v[e]) * scale_log2;
+            if (ALIBI) t = fmaf(slope2, static_cast<float>(e), t + bias0);
+            if (MASKED) t = pair_kept(ms, i, j0 + e) ? t : -INFINITY;
+            v[e] = __float_as_uint(t);
+            mx4[e & 3] = fmaxf(mx4[e & 3], t);
+        }
+    }
+    float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+    if (!MASKED && !ALIBI) mx *= scale_log2;  // scale > 0: max commutes with it
+    // lazy rescale: keep the old reference max unless it grew by more than the threshold
+    const bool upd = mx > m_run + kRescaleThreshold;
+    float alpha = 1.f;
+    if (upd) {
+        alpha = ex2(m_run - mx);  // m_run = -inf -> 0
+        m_run = mx;
+    }
+    const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+    float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+    uint32_t pk[BN / 2];
+#pragma unroll
+    for (int e = 0; e < BN; e += 2) {
+        float t0, t1;
+        if (!MASKED && !ALIBI) {
+            t0 = fmaf(__uint_as_float(v[e]), scale_log2, -m_use);
+            t1 = fmaf(__uint_as_float(v[e + 1]), scale_log2, -m_use);
+        } else {
+            t0 = __uint_as_float(v[e]) - m_use;
+            t1 = __uint_as_float(v[e + 1]) - m_use;
+        }
+        const float p0 = ex2(t0), p1 = ex2(t1);
+        ps4[(e >> 1) & 3] += p0 + p1;
+        pk[e >> 1] = pack_bf16x2(p0, p1);
+    }
+    tmem_st32(tS, pk);
+    tmem_st32(tS + 32, pk + 32);
+    l_run = l_run * alpha + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
+    if (n > 0 && __any_sync(0xffffffffu, upd)) {
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tO + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(tO + c * 32, o);
+        }
+    }
+    tmem_wait_st();
+}
+
 template <int D, int NQ, bool ROPE, int KS, int VS>
 __global__ void __launch_bounds__(128 * (2 + NQ), 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -102,6 +173,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
+    // Register budget: the softmax warpgroups hold a full row of 128 scores; the others need little.
+    constexpr int kSoftmaxRegs = NQ == 2 ? 184 : 232;
+
+    if (warp < 4) setmaxnreg_dec<56>();
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -206,6 +281,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------ rotation warpgroup (Section 4.1)
+        setmaxnreg_dec<88>();
         if (ROPE) {
             const int t = threadIdx.x - 128;
             bool ok = true;
@@ -229,6 +305,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp >= 8) {
         // ------------------------------------------------------------ softmax warpgroups (one query row per thread)
+        setmaxnreg_inc<kSoftmaxRegs>();
         const int q = (warp - 8) >> 2;
         const int row = threadIdx.x - 256 - q * 128;            // == TMEM lane
         const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -247,75 +324,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tc_fence_after_sync();
             const bool need_mask = tile_needs_mask(ms, i0[q], j0);
             const float bias0 = slope2 * static_cast<float>(j0 - i);
-
-            // pass 1: row max of the modified scores (log2 domain)
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tS + c * 32, v);
-                tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    float t = __uint_as_float(v[e]) * p.scale_log2;
-                    if (alibi) t = fmaf(slope2, static_cast<float>(c * 32 + e), t + bias0);
-                    if (need_mask && !pair_kept(ms, i, j0 + c * 32 + e)) t = -INFINITY;
-                    mx = fmaxf(mx, t);
-                }
+            if (alibi) {
+                if (need_mask) softmax_tile<D, true, true>(tS, tO, n, p.scale_log2, slope2, bias0, i, j0, ms, m_run, l_run);
+                else softmax_tile<D, false, true>(tS, tO, n, p.scale_log2, slope2, bias0, i, j0, ms, m_run, l_run);
+            } else {
+                if (need_mask) softmax_tile<D, true, false>(tS, tO, n, p.scale_log2, slope2, bias0, i, j0, ms, m_run, l_run);
+                else softmax_tile<D, false, false>(tS, tO, n, p.scale_log2, slope2, bias0, i, j0, ms, m_run, l_run);
             }
-            // lazy rescale: keep the old reference max unless it grew by more than the threshold
-            const bool upd = mx > m_run + kRescaleThreshold;
-            float alpha = 1.f;
-            if (upd) {
-                alpha = ex2(m_run - mx);  // m_run = -inf -> 0
-                m_run = mx;
-            }
-            if (n > 0 && __any_sync(0xffffffffu, upd)) {
-#pragma unroll 1
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tO + c * 32, v);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
-                    tmem_st32(tO + c * 32, v);
-                }
-                tmem_wait_st();
-            }
-            l_run *= alpha;
-            const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
-            const float nbias = bias0 - m_use;
-
-            // pass 2: p = 2^(t - m), row sum in fp32, P rounded to bf16 into TMEM (over S)
-            float psum = 0.f;
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32], pk[16];
-                tmem_ld32(tS + c * 32, v);
-                tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float t0, t1;
-                    if (alibi) {
-                        t0 = fmaf(__uint_as_float(v[e]), p.scale_log2, fmaf(slope2, static_cast<float>(c * 32 + e), nbias));
-                        t1 = fmaf(__uint_as_float(v[e + 1]), p.scale_log2,
-                                  fmaf(slope2, static_cast<float>(c * 32 + e + 1), nbias));
-                    } else {
-                        t0 = fmaf(__uint_as_float(v[e]), p.scale_log2, -m_use);
-                        t1 = fmaf(__uint_as_float(v[e + 1]), p.scale_log2, -m_use);
-                    }
-                    if (need_mask) {
-                        if (!pair_kept(ms, i, j0 + c * 32 + e)) t0 = -INFINITY;
-                        if (!pair_kept(ms, i, j0 + c * 32 + e + 1)) t1 = -INFINITY;
-                    }
-                    const float p0 = ex2(t0), p1 = ex2(t1);
-                    psum += p0 + p1;
-                    pk[e >> 1] = pack_bf16x2(p0, p1);
-                }
-                tmem_st16(tS + c * 16, pk);
-            }
-            l_run += psum;
-            tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(&bars[L::B_PREADY + q]);
         }
