@@ -129,7 +129,8 @@ def _mask_struct(mask: MaskSpec) -> _Mask:
 
 
 def rope_table(rope_spec: RopeSpec, S: int, device=None) -> Optional[torch.Tensor]:
-    """cos/sin table [S, rotary_dim/2, 2] fp32 built on the device (None when rotary_dim == 0)."""
+    """cos/sin table [S + 1, rotary_dim/2, 2] fp32 built on the device (None when rotary_dim == 0);
+    the last row is the trailer of step constants."""
     if rope_spec.rotary_dim == 0:
         return None
     n = lib().attnfuse_rope_table_bytes(S, rope_spec.rotary_dim)
@@ -137,7 +138,7 @@ def rope_table(rope_spec: RopeSpec, S: int, device=None) -> Optional[torch.Tenso
     table = torch.empty(n // 4, dtype=torch.float32, device=device)
     r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
     _check(lib().attnfuse_rope_table(ctypes.byref(r), S, table.data_ptr(), _stream()))
-    return table.view(S, rope_spec.rotary_dim // 2, 2)
+    return table.view(S + 1, rope_spec.rotary_dim // 2, 2)
 
 
 def rope(x: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor], inverse: bool = False,

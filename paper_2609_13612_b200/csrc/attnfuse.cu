@@ -154,7 +154,7 @@ af_status attnfuse_device_status(unsigned int* detail) {
 
 size_t attnfuse_rope_table_bytes(int S, int rotary_dim) {
     if (S < 1 || rotary_dim < 1) return 0;
-    return static_cast<size_t>(S) * (rotary_dim / 2) * sizeof(float2);
+    return static_cast<size_t>(S + 1) * (rotary_dim / 2) * sizeof(float2);  // + one trailer row
 }
 
 af_status attnfuse_rope_table(const af_rope* rope, int S, void* table, void* cuda_stream) {
@@ -165,7 +165,7 @@ af_status attnfuse_rope_table(const af_rope* rope, int S, void* table, void* cud
     if (!(rope->theta > 0.f)) return AF_ERR_SPEC;
     if (!table) return AF_ERR_NULL;
     if (!aligned16(table)) return AF_ERR_ALIGN;
-    const long long n = static_cast<long long>(S) * (rope->rotary_dim / 2);
+    const long long n = static_cast<long long>(S + 1) * (rope->rotary_dim / 2);
     const int threads = 256;
     const unsigned blocks = static_cast<unsigned>((n + threads - 1) / threads);
     rope_table_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(

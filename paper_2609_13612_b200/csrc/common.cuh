@@ -100,4 +100,81 @@ __device__ __forceinline__ void rotate_tile_smem(uint8_t* tile, int row0, int S,
     }
 }
 
+// Same rotation for the common case R in {16, 32, 64, 128} (CP = R/16 chunk pairs per row), with
+// far fewer table reads: thread (rg, cp) owns chunk pair cp of rows rg, rg + RP, rg + 2 RP, ...
+// (RP = 128 / CP).  It reads the table once, for its first row, and walks to the next rows with the
+// angle-addition recurrence (cos, sin)(a + d) from (cos, sin)(a) and the constant (cos, sin)(d),
+// d = RP * theta_i, which the table carries as a trailer row.  The first-row read is split off
+// (rotate_prefetch) so that it can be issued before waiting for the tile to land.
+template <int CP>
+struct RotState {
+    float4 t[4];     // {cos, sin} x 8 frequencies at the current row
+};
+
+template <int CP>
+__device__ __forceinline__ void rotate_load_step(const float2* table, int S, int R, int tid, float4 (&step)[4]) {
+    const int cp = tid % CP;
+    const float4* tb = reinterpret_cast<const float4*>(table + static_cast<size_t>(S) * (R >> 1) + cp * 8);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) step[u] = __ldg(tb + u);
+}
+
+template <int CP>
+__device__ __forceinline__ void rotate_prefetch(RotState<CP>& st, const float2* table, int row0, int S, int R,
+                                                int tid) {
+    const int rg = tid / CP, cp = tid % CP;
+    const int prow = min(row0 + rg, S - 1);
+    const float4* tb = reinterpret_cast<const float4*>(table + static_cast<size_t>(prow) * (R >> 1) + cp * 8);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) st.t[u] = __ldg(tb + u);
+}
+
+__device__ __forceinline__ void advance_cs(float& c, float& s, float C, float Sn) {
+    const float nc = fmaf(c, C, -s * Sn), ns = fmaf(s, C, c * Sn);
+    c = nc;
+    s = ns;
+}
+
+template <int CP>
+__device__ __forceinline__ void rotate_tile_fast(uint8_t* tile, RotState<CP>& st, const float4 (&step)[4], int tid) {
+    constexpr int RP = 128 / CP;
+    constexpr int NB = CP < 4 ? CP : 4;  // rows in flight per thread: all loads of a batch are issued first
+    const int rg = tid / CP, cp = tid % CP;
+#pragma unroll
+    for (int k0 = 0; k0 < CP; k0 += NB) {
+        uint4 lo[NB], hi[NB];
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+            const int r = rg + RP * (k0 + u);
+            lo[u] = *reinterpret_cast<const uint4*>(tile + swz_chunk_offset(r, cp));
+            hi[u] = *reinterpret_cast<const uint4*>(tile + swz_chunk_offset(r, cp + CP));
+        }
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+            rotate_word(lo[u].x, hi[u].x, st.t[0].x, st.t[0].y, st.t[0].z, st.t[0].w);
+            rotate_word(lo[u].y, hi[u].y, st.t[1].x, st.t[1].y, st.t[1].z, st.t[1].w);
+            rotate_word(lo[u].z, hi[u].z, st.t[2].x, st.t[2].y, st.t[2].z, st.t[2].w);
+            rotate_word(lo[u].w, hi[u].w, st.t[3].x, st.t[3].y, st.t[3].z, st.t[3].w);
+            if (k0 + u + 1 < CP) {
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    advance_cs(st.t[w].x, st.t[w].y, step[w].x, step[w].y);
+                    advance_cs(st.t[w].z, st.t[w].w, step[w].z, step[w].w);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+            const int r = rg + RP * (k0 + u);
+            *reinterpret_cast<uint4*>(tile + swz_chunk_offset(r, cp)) = lo[u];
+            *reinterpret_cast<uint4*>(tile + swz_chunk_offset(r, cp + CP)) = hi[u];
+        }
+    }
+}
+
+// Rows of the trailer: the recurrence stride for a given rotary dim (0: no fast path).
+__host__ __device__ constexpr int rope_fast_stride(int R) {
+    return (R == 16 || R == 32 || R == 64 || R == 128) ? 128 / (R / 16) : 0;
+}
+
 }  // namespace af

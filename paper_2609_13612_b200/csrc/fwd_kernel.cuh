@@ -6,6 +6,7 @@
 // Q once and every K tile, warps 8.. are one softmax warpgroup per query tile.
 #pragma once
 #include <cuda.h>
+#include <type_traits>
 #include "common.cuh"
 
 namespace af {
@@ -174,7 +175,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t tmem_base = *tmem_slot;
 
     // Register budget: the softmax warpgroups hold a full row of 128 scores; the others need little.
-    constexpr int kSoftmaxRegs = NQ == 2 ? 184 : 232;
+    constexpr int kSoftmaxRegs = NQ == 2 ? 176 : 232;
 
     if (warp < 4) setmaxnreg_dec<56>();
     if (warp == 0) {
@@ -281,27 +282,42 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------ rotation warpgroup (Section 4.1)
-        setmaxnreg_dec<88>();
+        setmaxnreg_dec<104>();
         if (ROPE) {
             const int t = threadIdx.x - 128;
-            bool ok = true;
+            auto run = [&](auto cp_tag) {
+                constexpr int CP = decltype(cp_tag)::value;  // 0: generic path (table read per row)
+                bool ok = true;
+                float4 step[4];
+                RotState<(CP > 0 ? CP : 1)> st;
+                if (CP > 0) rotate_load_step<(CP > 0 ? CP : 1)>(p.table, p.S, p.R, t, step);
 #pragma unroll
-            for (int q = 0; q < NQ; ++q) {
-                if (!ok || jhi[q] < jlo[q]) continue;
-                ok = mbar_wait(&bars[L::B_QFULL + q], 0, abort_flag, 8);
-                if (!ok) break;
-                rotate_tile_smem(sQ + q * TILE, i0[q], p.S, p.R, p.table, t, 128);
-                fence_proxy_async_smem();
-                mbar_arrive(&bars[L::B_QROT + q]);
-            }
-            for (int it = 0; ok && it < n_it; ++it) {
-                const int ks = it % KS;
-                ok = mbar_wait(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
-                if (!ok) break;
-                rotate_tile_smem(sK + ks * TILE, (jlo_c + it) * BN, p.S, p.R, p.table, t, 128);
-                fence_proxy_async_smem();
-                mbar_arrive(&bars[L::B_KROT + ks]);
-            }
+                for (int q = 0; q < NQ; ++q) {
+                    if (!ok || jhi[q] < jlo[q]) continue;
+                    if (CP > 0) rotate_prefetch(st, p.table, i0[q], p.S, p.R, t);
+                    ok = mbar_wait(&bars[L::B_QFULL + q], 0, abort_flag, 8);
+                    if (!ok) break;
+                    if (CP > 0) rotate_tile_fast(sQ + q * TILE, st, step, t);
+                    else rotate_tile_smem(sQ + q * TILE, i0[q], p.S, p.R, p.table, t, 128);
+                    fence_proxy_async_smem();
+                    mbar_arrive(&bars[L::B_QROT + q]);
+                }
+                for (int it = 0; ok && it < n_it; ++it) {
+                    const int ks = it % KS;
+                    if (CP > 0) rotate_prefetch(st, p.table, (jlo_c + it) * BN, p.S, p.R, t);
+                    ok = mbar_wait(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
+                    if (!ok) break;
+                    if (CP > 0) rotate_tile_fast(sK + ks * TILE, st, step, t);
+                    else rotate_tile_smem(sK + ks * TILE, (jlo_c + it) * BN, p.S, p.R, p.table, t, 128);
+                    fence_proxy_async_smem();
+                    mbar_arrive(&bars[L::B_KROT + ks]);
+                }
+            };
+            if (p.R == 128) run(std::integral_constant<int, 8>{});
+            else if (p.R == 64) run(std::integral_constant<int, 4>{});
+            else if (p.R == 32) run(std::integral_constant<int, 2>{});
+            else if (p.R == 16) run(std::integral_constant<int, 1>{});
+            else run(std::integral_constant<int, 0>{});
         }
     } else if (warp >= 8) {
         // ------------------------------------------------------------ softmax warpgroups (one query row per thread)

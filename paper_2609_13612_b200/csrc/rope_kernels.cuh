@@ -6,15 +6,17 @@
 namespace af {
 
 // table[s][i] = {cos, sin}((p0 + s) * theta^(-2i/R)); the angle is formed in fp64 so that large
-// positions do not lose the fraction of a turn, then rounded to fp32.
+// positions do not lose the fraction of a turn, then rounded to fp32.  One trailer row [S][i] holds
+// {cos, sin}(stride * theta^(-2i/R)), the constant the fused kernels use to walk from row to row.
 __global__ void rope_table_kernel(float2* __restrict__ table, int S, int R, double theta, int p0) {
     const int half = R >> 1;
     const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-    if (idx >= static_cast<long long>(S) * half) return;
+    if (idx >= static_cast<long long>(S + 1) * half) return;
     const int s = static_cast<int>(idx / half), i = static_cast<int>(idx - static_cast<long long>(s) * half);
     const double freq = pow(theta, -2.0 * static_cast<double>(i) / static_cast<double>(R));
+    const double pos = s < S ? static_cast<double>(p0 + s) : static_cast<double>(rope_fast_stride(R));
     double sn, cs;
-    sincos(static_cast<double>(p0 + s) * freq, &sn, &cs);
+    sincos(pos * freq, &sn, &cs);
     table[idx] = make_float2(static_cast<float>(cs), static_cast<float>(sn));
 }
 

@@ -39,7 +39,7 @@ def test_host_only_calls(libpath):
     L = af.lib()
     assert L.attnfuse_strerror(0) == b"ok"
     assert L.attnfuse_strerror(2) != L.attnfuse_strerror(3)
-    assert L.attnfuse_rope_table_bytes(4096, 128) == 4096 * 64 * 8
+    assert L.attnfuse_rope_table_bytes(4096, 128) == 4097 * 64 * 8
     assert L.attnfuse_rope_table_bytes(4096, 0) == 0
 
 

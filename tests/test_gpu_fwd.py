@@ -113,10 +113,13 @@ def test_fused_equals_separate_rope_then_plain_attention():
     o_sep, lse_sep = af.fwd(qr, kr, dev["v"], af.RopeSpec(), None, mask, w.scale)
     o_fus, lse_fus = af.fwd(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale)
     torch.cuda.synchronize()
-    # identical rounding points (rotated rows rounded to bf16 before the MMA) => identical bits
-    assert torch.equal(o_sep, o_fus) and torch.equal(lse_sep, lse_fus)
+    # same rounding points (rotated rows rounded to bf16 before the MMA); the fused kernel walks its
+    # cos/sin from row to row, so a few bf16 roundings of rotated elements may flip by one ulp
+    assert (o_sep.float() - o_fus.float()).abs().max().item() <= 8e-3
+    assert (lse_sep - lse_fus).abs().max().item() <= 2e-3
     want_o, _ = oracle.run_workload(w, t)
     pu.assert_close("separate O", pu.to_np(o_sep), want_o)
+    pu.assert_close("fused O", pu.to_np(o_fus), want_o)
 
 
 @pytest.mark.parametrize("R,inverse,D", [(128, False, 128), (64, False, 128), (128, True, 128), (64, False, 64),
@@ -146,8 +149,9 @@ def test_rope_table_against_fp64_formula():
     torch.cuda.synchronize()
     pos = rs.pos_offset + np.arange(512)[:, None]
     freq = 500000.0 ** (-2.0 * np.arange(64) / 128)
-    assert np.abs(pu.to_np(table[..., 0]) - np.cos(pos * freq)).max() < 1e-7
-    assert np.abs(pu.to_np(table[..., 1]) - np.sin(pos * freq)).max() < 1e-7
+    assert np.abs(pu.to_np(table[:512, :, 0]) - np.cos(pos * freq)).max() < 1e-7
+    assert np.abs(pu.to_np(table[:512, :, 1]) - np.sin(pos * freq)).max() < 1e-7
+    assert np.abs(pu.to_np(table[512, :, 0]) - np.cos(16 * freq)).max() < 1e-7  # trailer: stride 16 rows for R = 128
 
 
 def test_config1_tiny_and_config2_full():
