@@ -121,6 +121,44 @@ af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
                    : launch_fwd_variant<D, 2, false, 2, 2>(tq, tk, tv, p, stream);
 }
 
+template <int D, bool DKV, bool ROPE>
+af_status launch_bwd_variant(const CUtensorMap& tx, const CUtensorMap& ty, const CUtensorMap& ta, const CUtensorMap& tb,
+                             const BwdParams& p, dim3 grid, cudaStream_t stream) {
+    using L = BwdSmem<D>;
+    auto kern = attn_bwd_kernel<D, DKV, ROPE>;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
+            return AF_ERR_CUDA;
+        configured = true;
+    }
+    kern<<<grid, 384, L::BYTES, stream>>>(tx, ty, ta, tb, p);
+    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+template <int D>
+af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                     const CUtensorMap& tdo, const void* o, const void* d_o, BwdParams p, void* dq, int dq_f32,
+                     void* dk, void* dv, int dkv_f32, float* delta, cudaStream_t stream) {
+    const long long rows = static_cast<long long>(sh->B) * sh->Hq * sh->S;
+    const long long threads = rows * (D / 8);
+    bwd_delta_kernel<D><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
+        static_cast<const uint4*>(o), static_cast<const uint4*>(d_o), delta, rows);
+    if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
+    p.delta = delta;
+    const unsigned tiles = static_cast<unsigned>((sh->S + 127) / 128);
+    af_status st;
+    p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32;
+    dim3 gkv(sh->B * sh->Hkv, tiles, 1);
+    st = p.R > 0 ? launch_bwd_variant<D, true, true>(tk, tv, tq, tdo, p, gkv, stream)
+                 : launch_bwd_variant<D, true, false>(tk, tv, tq, tdo, p, gkv, stream);
+    if (st != AF_OK) return st;
+    p.out1 = dq; p.out2 = nullptr; p.out_f32 = dq_f32;
+    dim3 gq(sh->B * sh->Hq, tiles, 1);
+    return p.R > 0 ? launch_bwd_variant<D, false, true>(tq, tdo, tk, tv, p, gq, stream)
+                   : launch_bwd_variant<D, false, false>(tq, tdo, tk, tv, p, gq, stream);
+}
+
 }  // namespace
 
 extern "C" {
@@ -294,8 +332,29 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
     if ((st = resolve_strides(skv, shape->Hkv, shape->S, shape->D, &stkv)) != AF_OK) return st;
     resolve_strides(nullptr, shape->Hq, shape->S, shape->D, &stc);
     if ((st = check_arch()) != AF_OK) return st;
-    (void)stc;
-    return AF_ERR_SPEC;  // backward kernels not wired yet
+    CUtensorMap tq, tk, tv, tdo;
+    if ((st = make_tmap(&tq, q, shape->B, shape->Hq, shape->S, shape->D, stq, 128)) != AF_OK) return st;
+    if ((st = make_tmap(&tk, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, 128)) != AF_OK) return st;
+    if ((st = make_tmap(&tv, v, shape->B, shape->Hkv, shape->S, shape->D, stkv, 128)) != AF_OK) return st;
+    if ((st = make_tmap(&tdo, d_o, shape->B, shape->Hq, shape->S, shape->D, stc, 128)) != AF_OK) return st;
+    BwdParams p;
+    p.B = shape->B; p.Hq = shape->Hq; p.Hkv = shape->Hkv; p.S = shape->S; p.group = gqa_group;
+    p.R = rope->rotary_dim;
+    p.causal = mask->causal ? 1 : 0;
+    p.window = mask->window < 0 ? -1 : (mask->window > shape->S ? shape->S : mask->window);
+    p.scale = softmax_scale;
+    p.scale_log2 = softmax_scale * 1.4426950408889634f;
+    p.slopes = mask->alibi_slopes;
+    p.table = static_cast<const float2*>(rope_table);
+    p.lse = lse;
+    p.delta = nullptr; p.out1 = nullptr; p.out2 = nullptr; p.out_f32 = 0;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    float* delta = static_cast<float*>(workspace);
+    return shape->D == 128
+               ? launch_bwd<128>(shape, tq, tk, tv, tdo, o, d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32,
+                                 delta, stream)
+               : launch_bwd<64>(shape, tq, tk, tv, tdo, o, d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32,
+                                delta, stream);
 }
 
 }  // extern "C"

@@ -1,4 +1,381 @@
-// Backward kernels (Section 4.4).
+// Backward kernels (Section 4.4, FlashAttention-2 decomposition):
+//   1. bwd_delta_kernel      delta_i = sum_d dO_id * O_id             (row-reduced gradients)
+//   2. attn_bwd_kernel<DKV>  per key tile: dV += P^T dO, dK' += dS^T Q'   (no atomics: one CTA owns the tile)
+//   3. attn_bwd_kernel<DQ>   per query tile: dQ' += dS K'
+// Both MMA kernels recompute P from the saved L, recompute the RoPE rotation on chip, and rotate
+// the accumulated gradient back (transpose rotation) in the epilogue.
+//
+// One template covers 2 and 3.  A CTA keeps a stationary pair of tiles (X, Y) and streams pairs
+// (A, Bc):      DKV: X = K', Y = V,  A = Q', Bc = dO   (TMEM lane = key row,   column = query row)
+//               DQ : X = Q', Y = dO, A = K', Bc = V    (TMEM lane = query row, column = key row)
+//   T1 = X A^T  (scores or their transpose),  T2 = Y Bc^T  (dP or its transpose)
+//   P = 2^(c2 T1 + bias - L2), dS = P (T2 - delta); P, dS go back to TMEM as bf16 over T1, T2
+//   DKV: acc1 += P Bc, acc2 += dS A.      DQ: acc1 += dS A.
 #pragma once
 #include <cuda.h>
+#include <type_traits>
 #include "common.cuh"
+
+namespace af {
+
+struct BwdParams {
+    int B, Hq, Hkv, S, group;
+    int R;
+    int causal, window;
+    float scale, scale_log2;
+    const float* slopes;
+    const float2* table;
+    const float* lse;     // [B,Hq,S]
+    const float* delta;   // [B,Hq,S]
+    void* out1;           // DKV: dV   DQ: dQ
+    void* out2;           // DKV: dK   DQ: unused
+    int out_f32;
+};
+
+// delta[row] = <dO[row], O[row]>; one 16-byte chunk per thread, D/8 threads per row.
+template <int D>
+__global__ void __launch_bounds__(256) bwd_delta_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o,
+                                                        float* __restrict__ delta, long long rows) {
+    constexpr int TPR = D / 8;
+    const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+    const long long row = idx / TPR;
+    float acc = 0.f;
+    if (row < rows) {
+        const uint4 a = __ldg(o + idx), b = __ldg(d_o + idx);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            acc += bf16lo_to_f32(aw[u]) * bf16lo_to_f32(bw[u]) + bf16hi_to_f32(aw[u]) * bf16hi_to_f32(bw[u]);
+    }
+#pragma unroll
+    for (int off = TPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (row < rows && (threadIdx.x % TPR) == 0) delta[row] = acc;
+}
+
+template <int D>
+struct BwdSmem {
+    static constexpr int TILE = 128 * D * 2;
+    static constexpr int NST = 2;                 // stream stages
+    static constexpr int OFF_X = 0, OFF_Y = TILE;
+    static constexpr int OFF_A = 2 * TILE;        // NST tiles
+    static constexpr int OFF_B = OFF_A + NST * TILE;
+    static constexpr int OFF_STATS = OFF_B + NST * TILE;      // float [2][2][128]: L2 and delta of the streamed tile
+    static constexpr int OFF_BAR = OFF_STATS + 2 * 2 * 128 * 4;
+    static constexpr int B_XFULL = 0, B_XROT = 1, B_YFULL = 2, B_AFULL = 3, B_AROT = B_AFULL + NST,
+                         B_BFULL = B_AROT + NST, B_EMPTY = B_BFULL + NST, B_TFULL = B_EMPTY + NST,
+                         B_PDS = B_TFULL + 1, B_DONE = B_PDS + 1, N_BARS = B_DONE + 1;
+    static constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;
+    static constexpr int BYTES = OFF_MISC + 16 + 1024;
+    static constexpr int STG_STRIDE = D + 4;      // floats per staged row (padding keeps 16-byte stores conflict-free)
+    static_assert(128 * STG_STRIDE * 4 <= 2 * NST * TILE, "staging buffer must fit in the stream stages");
+};
+
+__device__ __forceinline__ void wg_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Barrier over the 128 threads of the gradient warpgroup that also ANDs a flag, so that a wait
+// that gave up in one thread ends the loop in all of them (nobody is left alone at a barrier).
+__device__ __forceinline__ bool wg_all(bool v) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.and.pred q, 1, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"(static_cast<uint32_t>(v))
+        : "memory");
+    return r != 0;
+}
+
+// Epilogue helper: the 128 threads of the gradient warpgroup move a [128 x D] fp32 accumulator
+// from TMEM (one row per thread) through shared memory to global memory, scaling it and, when
+// R > 0, applying the transpose rotation for positions row0.. (gradients w.r.t. rotated rows are
+// rotated back).  Global writes are coalesced along D.
+template <int D>
+__device__ __forceinline__ void store_acc_rotated(uint32_t t_acc, float* stg, int tid, float mul, int R,
+                                                  const float2* table, int row0, int S, void* out, size_t out_row0,
+                                                  int out_f32) {
+    constexpr int STRIDE = BwdSmem<D>::STG_STRIDE;
+#pragma unroll 1
+    for (int c = 0; c < D / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld32(t_acc + c * 32, v);
+        tmem_wait_ld();
+        float4* dst = reinterpret_cast<float4*>(stg + tid * STRIDE + c * 32);
+#pragma unroll
+        for (int e = 0; e < 32; e += 4)
+            dst[e >> 2] = make_float4(__uint_as_float(v[e]) * mul, __uint_as_float(v[e + 1]) * mul,
+                                      __uint_as_float(v[e + 2]) * mul, __uint_as_float(v[e + 3]) * mul);
+    }
+    wg_sync();
+    constexpr int RPP = 128 / D;  // rows per pass (1 for D = 128, 2 for D = 64)
+    const int d = tid % D, rsub = tid / D;
+    const int half = R >> 1;
+    const int fi = d < half ? d : d - half;
+    for (int r = rsub; r < 128; r += RPP) {
+        const int row = row0 + r;
+        if (row >= S) break;
+        float y = stg[r * STRIDE + d];
+        if (d < R) {
+            const float2 cs = __ldg(table + static_cast<size_t>(row) * half + fi);
+            const float other = stg[r * STRIDE + (d < half ? d + half : d - half)];
+            y = d < half ? fmaf(y, cs.x, other * cs.y) : fmaf(y, cs.x, -other * cs.y);
+        }
+        const size_t o = (out_row0 + r) * D + d;
+        if (out_f32) static_cast<float*>(out)[o] = y;
+        else static_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(y);
+    }
+    wg_sync();
+}
+
+template <int D, bool DKV, bool ROPE>
+__global__ void __launch_bounds__(384, 1)
+attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_y,
+                const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                const BwdParams p) {
+    using L = BwdSmem<D>;
+    constexpr int TILE = L::TILE, NST = L::NST;
+    constexpr int NBOX = D / BOX_COLS;
+    constexpr uint32_t TMEM_COLS = 512;
+    constexpr uint32_t T1 = 0, T2 = 128, ACC1 = 256, ACC2 = 256 + D;
+    constexpr uint32_t IDESC_T = idesc_bf16_f32(128, 128, 0, 0);
+    constexpr uint32_t IDESC_ACC = idesc_bf16_f32(128, D, 0, 1);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *sX = smem + L::OFF_X, *sY = smem + L::OFF_Y, *sA = smem + L::OFF_A, *sB = smem + L::OFF_B;
+    float* sStats = reinterpret_cast<float*>(smem + L::OFF_STATS);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_MISC + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const MaskSpec ms{p.S, p.causal, p.window};
+    // stationary tile: DKV -> key tile of kv head (b, hk); DQ -> query tile of head (b, h)
+    const int xh_count = DKV ? p.Hkv : p.Hq;
+    const int b = blockIdx.x / xh_count, xh = blockIdx.x - b * xh_count;
+    // heaviest tiles first: under a causal mask early key tiles and late query tiles see the most work
+    const int x0 = (DKV ? static_cast<int>(blockIdx.y) : static_cast<int>(gridDim.y - 1 - blockIdx.y)) * 128;
+    int lo, hi;  // streamed tile range
+    if (DKV) qtile_range(ms, x0, lo, hi);
+    else tile_range(ms, x0, lo, hi);
+    const int per_head = hi - lo + 1;
+    const int n_it = DKV ? per_head * p.group : per_head;
+    // iteration n -> (streamed head, streamed row0)
+    auto stream_head = [&](int n) { return DKV ? xh * p.group + n / per_head : xh / p.group; };
+    auto stream_row0 = [&](int n) { return (lo + (DKV ? n % per_head : n)) * 128; };
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < L::N_BARS; ++i) {
+            uint32_t cnt = 1;
+            if (i == L::B_XROT || (i >= L::B_AROT && i < L::B_AROT + NST) || i == L::B_PDS) cnt = 128;
+            mbar_init(&bars[i], cnt);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            prefetch_tmap(&tm_x); prefetch_tmap(&tm_y); prefetch_tmap(&tm_a); prefetch_tmap(&tm_b);
+            mbar_arrive_expect_tx(&bars[L::B_XFULL], TILE);
+            mbar_arrive_expect_tx(&bars[L::B_YFULL], TILE);
+#pragma unroll
+            for (int bx = 0; bx < NBOX; ++bx) {
+                tma_load_4d(sX + bx * BOX_BYTES, &tm_x, &bars[L::B_XFULL], bx * BOX_COLS, x0, xh, b);
+                tma_load_4d(sY + bx * BOX_BYTES, &tm_y, &bars[L::B_YFULL], bx * BOX_COLS, x0, xh, b);
+            }
+            for (int n = 0; n < n_it; ++n) {
+                const int st = n % NST, ah = stream_head(n), a0 = stream_row0(n);
+                if (!mbar_wait(&bars[L::B_EMPTY + st], ((n / NST) & 1) ^ 1, abort_flag, 21)) break;
+                mbar_arrive_expect_tx(&bars[L::B_AFULL + st], TILE);
+                mbar_arrive_expect_tx(&bars[L::B_BFULL + st], TILE);
+#pragma unroll
+                for (int bx = 0; bx < NBOX; ++bx) {
+                    tma_load_4d(sA + st * TILE + bx * BOX_BYTES, &tm_a, &bars[L::B_AFULL + st], bx * BOX_COLS, a0, ah, b);
+                    tma_load_4d(sB + st * TILE + bx * BOX_BYTES, &tm_b, &bars[L::B_BFULL + st], bx * BOX_COLS, a0, ah, b);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr int B_XREADY = ROPE ? L::B_XROT : L::B_XFULL;
+            constexpr int B_AREADY = ROPE ? L::B_AROT : L::B_AFULL;
+            bool ok = mbar_wait(&bars[B_XREADY], 0, abort_flag, 22);
+            if (ok) ok = mbar_wait(&bars[L::B_YFULL], 0, abort_flag, 23);
+            const uint32_t xa = smem_u32(sX), ya = smem_u32(sY);
+            for (int n = 0; ok && n < n_it; ++n) {
+                const int st = n % NST;
+                const uint32_t aa = smem_u32(sA + st * TILE), ba = smem_u32(sB + st * TILE);
+                ok = mbar_wait(&bars[B_AREADY + st], (n / NST) & 1, abort_flag, 24);
+                if (ok) ok = mbar_wait(&bars[L::B_BFULL + st], (n / NST) & 1, abort_flag, 25);
+                if (!ok) break;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
+                    mma_ss(tmem_base + T1, smem_desc_sw128(xa + off, 16, 1024), smem_desc_sw128(aa + off, 16, 1024),
+                           IDESC_T, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
+                    mma_ss(tmem_base + T2, smem_desc_sw128(ya + off, 16, 1024), smem_desc_sw128(ba + off, 16, 1024),
+                           IDESC_T, kk > 0);
+                }
+                mma_commit(&bars[L::B_TFULL]);
+                ok = mbar_wait(&bars[L::B_PDS], n & 1, abort_flag, 26);
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (DKV) {
+#pragma unroll
+                    for (int kk = 0; kk < 128 / 16; ++kk)   // acc1 (dV) += P^T dO: dO is the MN-major B operand
+                        mma_ts(tmem_base + ACC1, tmem_base + T1 + kk * 8, smem_desc_sw128(ba + kk * 2048, BOX_BYTES, 1024),
+                               IDESC_ACC, (n > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+                    for (int kk = 0; kk < 128 / 16; ++kk)   // acc2 (dK') += dS^T Q'
+                        mma_ts(tmem_base + ACC2, tmem_base + T2 + kk * 8, smem_desc_sw128(aa + kk * 2048, BOX_BYTES, 1024),
+                               IDESC_ACC, (n > 0 || kk > 0) ? 1u : 0u);
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < 128 / 16; ++kk)   // acc1 (dQ') += dS K'
+                        mma_ts(tmem_base + ACC1, tmem_base + T1 + kk * 8, smem_desc_sw128(aa + kk * 2048, BOX_BYTES, 1024),
+                               IDESC_ACC, (n > 0 || kk > 0) ? 1u : 0u);
+                }
+                mma_commit(&bars[L::B_EMPTY + st]);
+                if (n == n_it - 1) mma_commit(&bars[L::B_DONE]);
+            }
+        }
+    } else if (warp >= 4 && warp < 8) {
+        // ------------------------------------------------------------ rotation warpgroup: X once, every A tile
+        if (ROPE) {
+            const int t = threadIdx.x - 128;
+            auto run = [&](auto cp_tag) {
+                constexpr int CP = decltype(cp_tag)::value;
+                constexpr int CPT = CP > 0 ? CP : 1;
+                float4 step[4];
+                RotState<CPT> st;
+                if (CP > 0) {
+                    rotate_load_step<CPT>(p.table, p.S, p.R, t, step);
+                    rotate_prefetch(st, p.table, x0, p.S, p.R, t);
+                }
+                bool ok = mbar_wait(&bars[L::B_XFULL], 0, abort_flag, 27);
+                if (!ok) return;
+                if (CP > 0) rotate_tile_fast(sX, st, step, t);
+                else rotate_tile_smem(sX, x0, p.S, p.R, p.table, t, 128);
+                fence_proxy_async_smem();
+                mbar_arrive(&bars[L::B_XROT]);
+                for (int n = 0; n < n_it; ++n) {
+                    const int sg = n % NST, a0 = stream_row0(n);
+                    if (CP > 0) rotate_prefetch(st, p.table, a0, p.S, p.R, t);
+                    if (!mbar_wait(&bars[L::B_AFULL + sg], (n / NST) & 1, abort_flag, 28)) return;
+                    if (CP > 0) rotate_tile_fast(sA + sg * TILE, st, step, t);
+                    else rotate_tile_smem(sA + sg * TILE, a0, p.S, p.R, p.table, t, 128);
+                    fence_proxy_async_smem();
+                    mbar_arrive(&bars[L::B_AROT + sg]);
+                }
+            };
+            if (p.R == 128) run(std::integral_constant<int, 8>{});
+            else if (p.R == 64) run(std::integral_constant<int, 4>{});
+            else if (p.R == 32) run(std::integral_constant<int, 2>{});
+            else if (p.R == 16) run(std::integral_constant<int, 1>{});
+            else run(std::integral_constant<int, 0>{});
+        }
+    } else if (warp >= 8) {
+        // ------------------------------------------------------------ gradient warpgroup (one TMEM lane per thread)
+        const int tid = threadIdx.x - 256;
+        const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tb = tmem_base + lane_addr;
+        const int xrow = x0 + tid;  // DKV: key row j; DQ: query row i
+        const bool alibi = p.slopes != nullptr;
+        constexpr float kLog2e = 1.4426950408889634f;
+        float my_l2 = 0.f, my_delta = 0.f, my_slope2 = 0.f;
+        if (!DKV) {
+            const size_t r = (static_cast<size_t>(b) * p.Hq + xh) * p.S + xrow;
+            my_l2 = xrow < p.S ? p.lse[r] * kLog2e : INFINITY;
+            my_delta = xrow < p.S ? p.delta[r] : 0.f;
+            my_slope2 = alibi ? p.slopes[xh] * kLog2e : 0.f;
+        }
+        bool ok = true;
+        for (int n = 0; ok && n < n_it; ++n) {
+            const int ah = stream_head(n), a0 = stream_row0(n);
+            float* sL2 = sStats + (n & 1) * 256;
+            float* sDl = sL2 + 128;
+            if (DKV) {
+                // per-column statistics of the streamed query tile
+                const int qi = a0 + tid;
+                const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + qi;
+                sL2[tid] = qi < p.S ? p.lse[r] * kLog2e : INFINITY;
+                sDl[tid] = qi < p.S ? p.delta[r] : 0.f;
+                my_slope2 = alibi ? p.slopes[ah] * kLog2e : 0.f;
+            }
+            const int i0 = DKV ? a0 : x0, j0 = DKV ? x0 : a0;
+            const bool need_mask = tile_needs_mask(ms, i0, j0);
+            ok = wg_all(mbar_wait(&bars[L::B_TFULL], n & 1, abort_flag, 29));  // also publishes the statistics
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t s[32], dp[32], pk[16], dk[16];
+                tmem_ld32(tb + T1 + c * 32, s);
+                tmem_ld32(tb + T2 + c * 32, dp);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    float pv[2], dv[2];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int col = c * 32 + e + u;
+                        const int i = DKV ? a0 + col : xrow, j = DKV ? xrow : a0 + col;
+                        const float l2 = DKV ? sL2[col] : my_l2, dl = DKV ? sDl[col] : my_delta;
+                        float t = fmaf(__uint_as_float(s[e + u]), p.scale_log2, -l2);
+                        if (alibi) t = fmaf(my_slope2, static_cast<float>(j - i), t);
+                        float pe = ex2(t);
+                        if (need_mask && !pair_kept(ms, i, j)) pe = 0.f;
+                        pv[u] = pe;
+                        dv[u] = pe * (__uint_as_float(dp[e + u]) - dl);
+                    }
+                    pk[e >> 1] = pack_bf16x2(pv[0], pv[1]);
+                    dk[e >> 1] = pack_bf16x2(dv[0], dv[1]);
+                }
+                if (DKV) {
+                    tmem_st16(tb + T1 + c * 16, pk);
+                    tmem_st16(tb + T2 + c * 16, dk);
+                } else {
+                    tmem_st16(tb + T1 + c * 16, dk);
+                }
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(&bars[L::B_PDS]);
+        }
+        // epilogue: stage through shared memory (the stream stages are idle now), rotate back, store
+        if (ok && n_it > 0) ok = wg_all(mbar_wait(&bars[L::B_DONE], 0, abort_flag, 30));
+        if (ok && n_it > 0) {
+            tc_fence_after_sync();
+            float* stg = reinterpret_cast<float*>(sA);
+            const size_t out_row0 = (static_cast<size_t>(b) * xh_count + xh) * p.S + x0;
+            if (DKV) {
+                store_acc_rotated<D>(tb + ACC1, stg, tid, 1.f, 0, p.table, x0, p.S, p.out1, out_row0, p.out_f32);
+                store_acc_rotated<D>(tb + ACC2, stg, tid, p.scale, p.R, p.table, x0, p.S, p.out2, out_row0, p.out_f32);
+            } else {
+                store_acc_rotated<D>(tb + ACC1, stg, tid, p.scale, p.R, p.table, x0, p.S, p.out1, out_row0, p.out_f32);
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace af

@@ -157,3 +157,33 @@ def test_rope_table_against_fp64_formula():
 def test_config1_tiny_and_config2_full():
     for w in synth.CONFIGS[:2]:
         run_case(w)
+
+
+def test_config3_composed_variant_sampled_heads():
+    """Config 3 at full size (window 1024 + ALiBi): all rows of sampled heads (steepest and flattest slope)."""
+    w = synth.CONFIGS[2]
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    o, lse = pu.gpu_fwd(w, dev)
+    sl = w.alibi_slopes()
+    for b, h in ((0, 0), (1, 7), (1, 15)):
+        sub = {k: v[b:b + 1, h:h + 1] for k, v in t.items()}
+        want_o, want_l = oracle.fwd(sub["q"], sub["k"], sub["v"], theta=w.theta, rotary_dim=w.R, window=w.window,
+                                    slopes=sl[h:h + 1], scale=w.scale)
+        pu.assert_close("c3 O head %d" % h, pu.to_np(o[b:b + 1, h:h + 1]), want_o)
+        assert np.abs(pu.to_np(lse[b:b + 1, h:h + 1]) - want_l).max() <= pu.LSE_TOL
+
+
+def test_config4_long_context_sampled_rows():
+    """Config 4 at full size: a stratified subset of query rows of every head (first rows, tile
+    boundaries, every 509th row, the last rows), each computed one by one by the oracle."""
+    w = synth.CONFIGS[3]
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    o, lse = pu.gpu_fwd(w, dev)
+    rows = sorted(set([0, 1, 2, 127, 128, 129, 255, 256, 257] + list(range(300, w.S, 509)) +
+                      list(range(w.S - 3, w.S))))
+    want_o, want_l = oracle.run_workload(w, t, rows=rows)
+    idx = torch.tensor(rows, device="cuda")
+    pu.assert_close("c4 O", pu.to_np(o[:, :, idx]), want_o)
+    assert np.abs(pu.to_np(lse[:, :, idx]) - want_l).max() <= pu.LSE_TOL
