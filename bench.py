@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark of the fused RoPE + causal attention path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--extras 0|1]
+
+Prints ONE JSON line.  A step is one fused forward pass (rotate Q and K on chip, QK^T, causal
+mask, online softmax, PV, O and L written) over the Llama-3-8B attention shape (B=1, Hq=32,
+Hkv=8, S=4096, D=128, bf16); `value` is algorithmic TFLOP/s (two contractions over the kept
+(query, key) pairs only).  The cos/sin table is set-up, built once before the timed region.
+
+Inputs are seeded synthetic N(0,1) tensors of that shape, resident in HBM; the timed steps rotate
+over several independent input sets whose total size exceeds L2, so no step finds its inputs
+cached.  `e2e` measures the same step through the host-buffer entry point (pinned host memory,
+copies inside the timed region).  `--impl reference` times the fp64 CPU oracle on the host cores.
+With N > 1 (torchrun) every rank runs the same per-GPU workload (the path shards over independent
+(batch, kv-head) units with no exchange step); times are the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2609_13612_b200 import synth  # noqa: E402
+
+METRIC = "fused RoPE+causal attention TFLOP/s (bf16 fwd/bwd) and % of B200 tensor peak"
+UNIT = "TFLOP/s"
+L2_BYTES = 126 * 1024 * 1024
+# DRAM bytes per launch of the forward kernel on this workload, from the ncu capture summarised in
+# profiles/attn_fwd_kernel_c2_llama3_8b.md (dram__bytes_read.sum + dram__bytes_write.sum).
+FWD_TRAFFIC_BYTES_PER_LAUNCH = None
+PAPER_CONTEXT = {
+    "rtx3090_fused_vs_flex_prerotate_rope_causal": "2.10x (RTX 3090, fp16, B=4 H=12 D=64, N=4096)",
+    "h100_llama3_8b_training_step_vs_sdpa": "within ~5% (H100 NVL, fp16, N=2048: 7.65 ms vs 7.27 ms)",
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_tflops": float(d["bf16_tflops"]), "bf16_tflops_sustained": float(d["bf16_tflops_sustained"]),
+                "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4,
+                 "hw_power_brake_slowdown": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_rate(w: synth.Workload, budget_s: float):
+    """Time the oracle (as it stands) on a row sample of workload w sized for about budget_s."""
+    import oracle
+    t = synth.draw_all(w)
+    pilot_rows = list(range(w.S - 1, -1, -max(1, w.S // 64)))
+    t0 = time.perf_counter()
+    oracle.run_workload(w, t, rows=pilot_rows)
+    dt = max(time.perf_counter() - t0, 1e-6)
+    pairs = lambda rows: float(sum(min(i + 1, (w.window + 1) if w.window >= 0 else i + 1) for i in rows))
+    rate = pairs(pilot_rows) / dt
+    total = float(w.kept_pairs_per_head())
+    stride = max(1, int(math.ceil(total / (rate * budget_s))))
+    rows = list(range(w.S - 1, -1, -stride))
+    t0 = time.perf_counter()
+    oracle.run_workload(w, t, rows=rows)
+    dt = time.perf_counter() - t0
+    flops = 4.0 * w.D * pairs(rows) * w.B * w.Hq
+    return flops / dt / 1e12, "every %d-th query row of every head (%d rows, %.1f s)" % (stride, len(rows), dt), dt
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0))
+    per_step = max(1.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
+    vals, sample = [], ""
+    for i in range(args.warmup + args.steps):
+        v, sample, _ = oracle_rate(w, per_step)
+        if i >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": None, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "S": w.S, "D": w.D,
+                                        "variant": "rope(theta=%g)+causal" % w.theta},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--extras", type=int, default=1, help="also time configs 3-5, the separate-RoPE arm and the sweep")
+    ap.add_argument("--cpu-baseline", type=int, default=1)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = synth.CONFIGS[1]
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import paper_2609_13612_b200 as af
+    from paper_2609_13612_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    peaks = measured_peaks()
+
+    def to_dev(x):
+        return torch.from_numpy(synth.bf16_bits(x).view(np.int16)).view(torch.bfloat16).to(dev)
+
+    def make_sets(wl, n_sets):
+        base = {k: to_dev(v) for k, v in synth.draw_all(wl).items()}
+        sets = [base]
+        for s in range(1, n_sets):
+            sets.append({k: torch.roll(v, shifts=s, dims=1).contiguous() for k, v in base.items()})
+        return sets
+
+    def specs(wl):
+        rope = af.RopeSpec(theta=wl.theta, rotary_dim=wl.R, pos_offset=wl.pos_offset)
+        sl = wl.alibi_slopes()
+        mask = af.MaskSpec(causal=wl.causal, window=wl.window,
+                           alibi_slopes=torch.from_numpy(sl).to(dev) if sl is not None else None)
+        return rope, mask, af.rope_table(rope, wl.S, device=dev)
+
+    def input_bytes(wl):
+        return 2 * wl.B * wl.S * wl.D * (wl.Hq + 2 * wl.Hkv)
+
+    def n_sets_for(wl):
+        return max(2, int(math.ceil(2.0 * L2_BYTES / input_bytes(wl))) + 1) if input_bytes(wl) < 2 * L2_BYTES else 1
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        """K steps between barrier+sync, plus per-launch CUDA-event durations on the launching stream."""
+        for i in range(warmup):
+            fn(i)
+        barrier()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        t0 = time.perf_counter()
+        start = torch.cuda.Event(enable_timing=True)
+        stop = torch.cuda.Event(enable_timing=True)
+        start.record()
+        for i in range(steps):
+            evs[i][0].record()
+            fn(i)
+            evs[i][1].record()
+        stop.record()
+        barrier()
+        wall_ms = (time.perf_counter() - t0) * 1e3
+        total_ms = start.elapsed_time(stop)
+        per = [a.elapsed_time(b) for a, b in evs]
+        if dist is not None:
+            tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            total_ms = float(tt.item())
+        return total_ms, per, wall_ms
+
+    # ------------------------------------------------------------------ headline: fused forward, config 2
+    rope, mask, table = specs(w)
+    sets = make_sets(w, n_sets_for(w))
+    o = torch.empty((w.B, w.Hq, w.S, w.D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((w.B, w.Hq, w.S), dtype=torch.float32, device=dev)
+
+    def step(i):
+        s = sets[i % len(sets)]
+        af.fwd(s["q"], s["k"], s["v"], rope, table, mask, w.scale, out=o, lse=lse)
+
+    with ClockSampler(local) as clk:
+        total_ms, per, _ = timed(step, args.steps, args.warmup)
+    code, detail = af.device_status()
+    if code != 0:
+        raise SystemExit("device-side wait ran out (0x%x): numbers invalid" % detail)
+    ms_per_step = total_ms / args.steps
+    flops = w.fwd_flops()
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    kern_ms = float(np.mean(per))
+    achieved = flops / (kern_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "attn_fwd_kernel<128,2,rope>", "achieved": achieved,
+                "peak": peaks["bf16_tflops"], "peak_kind": "burst bf16 dense, %s" % peaks["source"], "unit": UNIT,
+                "frac": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
+                "traffic": FWD_TRAFFIC_BYTES_PER_LAUNCH, "kernel_ms": kern_ms,
+                "algorithmic_flops_per_launch": flops}
+
+    # ------------------------------------------------------------------ e2e: host buffers through the C-ABI
+    hq, hk, hv = (sets[0][k].cpu().pin_memory() for k in ("q", "k", "v"))
+    ho = torch.empty_like(hq).pin_memory()
+    hl = torch.empty((w.B, w.Hq, w.S), dtype=torch.float32).pin_memory()
+    staging = torch.empty(binding.fwd_host_staging_bytes(w.B, w.Hq, w.Hkv, w.S, w.D), dtype=torch.uint8, device=dev)
+
+    def step_host(i):
+        af.fwd_host(hq, hk, hv, rope, table, mask, w.scale, ho, hl, staging)
+
+    e2e_steps = max(3, min(args.steps, 50))
+    e2e_ms, _, _ = timed(step_host, e2e_steps, 3)
+    e2e_val = world * flops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    h2d = int(hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2)
+    d2h = int(ho.numel() * 2 + hl.numel() * 4)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "S": w.S, "D": w.D,
+                   "variant": "rope(theta=%g, all dims)+causal, scale 1/sqrt(D), forward" % w.theta,
+                   "l2": "inputs rotate over %d independent sets (%.0f MB total > 126 MB L2)" % (
+                       len(sets), len(sets) * input_bytes(w) / 1e6),
+                   "sharding": "replicated per-GPU workload, no collective" if world > 1 else "single GPU"},
+        "clocks": clk.summary(),
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": args.steps,
+        "roofline": roofline,
+        "pct_of_tensor_peak": {"measured_burst_%.0f" % peaks["bf16_tflops"]: 100 * value / world / peaks["bf16_tflops"],
+                               "measured_sustained_%.0f" % peaks["bf16_tflops_sustained"]:
+                                   100 * value / world / peaks["bf16_tflops_sustained"],
+                               "nominal_2250": 100 * value / world / 2250.0},
+        "paper_context": PAPER_CONTEXT,
+    }
+
+    # ------------------------------------------------------------------ extras (rank 0's GPU only, short runs)
+    if args.extras and rank == 0:
+        ex = {}
+        k_ex, w_ex = 20, 5
+
+        def fwd_ms(wl, fused=True, sets_=None):
+            r, m, tb = specs(wl)
+            ss = sets_ or make_sets(wl, n_sets_for(wl))
+            oo = torch.empty((wl.B, wl.Hq, wl.S, wl.D), dtype=torch.bfloat16, device=dev)
+            ll = torch.empty((wl.B, wl.Hq, wl.S), dtype=torch.float32, device=dev)
+            norope = af.RopeSpec()
+            if fused:
+                f = lambda i: af.fwd(ss[i % len(ss)]["q"], ss[i % len(ss)]["k"], ss[i % len(ss)]["v"], r, tb, m,
+                                     wl.scale, out=oo, lse=ll)
+            else:
+                qr = torch.empty_like(ss[0]["q"])
+                kr = torch.empty_like(ss[0]["k"])
+
+                def f(i):
+                    s = ss[i % len(ss)]
+                    af.rope(s["q"], r, tb, out=qr)
+                    af.rope(s["k"], r, tb, out=kr)
+                    af.fwd(qr, kr, s["v"], norope, None, m, wl.scale, out=oo, lse=ll)
+            t, _, _ = timed(f, k_ex, w_ex)
+            return t / k_ex, ss
+
+        for wl in synth.CONFIGS[2:4]:
+            ms_f, ss = fwd_ms(wl, True)
+            ms_s, _ = fwd_ms(wl, False, ss)
+            ex[wl.name] = {"fused_fwd_ms": ms_f, "fused_fwd_tflops": wl.fwd_flops() / ms_f / 1e9,
+                           "separate_rope_fwd_ms": ms_s, "separate_rope_fwd_tflops": wl.fwd_flops() / ms_s / 1e9,
+                           "fused_over_separate_speedup": ms_s / ms_f}
+            del ss
+            torch.cuda.empty_cache()
+        # config 5: forward + backward
+        w5 = synth.CONFIGS[4]
+        r5, m5, t5 = specs(w5)
+        s5 = make_sets(w5, n_sets_for(w5))
+        o5, l5 = af.fwd(s5[0]["q"], s5[0]["k"], s5[0]["v"], r5, t5, m5, w5.scale)
+        ws = torch.empty(af.lib().attnfuse_bwd_workspace_bytes(
+            __import__("ctypes").byref(binding._Shape(w5.B, w5.Hq, w5.Hkv, w5.S, w5.D))), dtype=torch.uint8, device=dev)
+
+        def fb(i):
+            s = s5[i % len(s5)]
+            af.fwd(s["q"], s["k"], s["v"], r5, t5, m5, w5.scale, out=o5, lse=l5)
+            af.bwd(s["q"], s["k"], s["v"], o5, l5, s["do"], r5, t5, m5, w5.scale, workspace=ws)
+
+        def bonly(i):
+            s = s5[i % len(s5)]
+            af.bwd(s["q"], s["k"], s["v"], o5, l5, s["do"], r5, t5, m5, w5.scale, workspace=ws)
+
+        t_fb, _, _ = timed(fb, k_ex, w_ex)
+        t_b, _, _ = timed(bonly, k_ex, w_ex)
+        ex[w5.name] = {"fwd_bwd_ms": t_fb / k_ex,
+                       "fwd_bwd_tflops": (w5.fwd_flops() + w5.bwd_flops()) / (t_fb / k_ex) / 1e9,
+                       "bwd_ms": t_b / k_ex, "bwd_tflops": w5.bwd_flops() / (t_b / k_ex) / 1e9,
+                       "bwd_pct_of_measured_peak": 100 * w5.bwd_flops() / (t_b / k_ex) / 1e9 / peaks["bf16_tflops"]}
+        del s5
+        torch.cuda.empty_cache()
+        # Rotation Calculus sweep (Section 5.3): fused vs separate RoPE at constant B*S = 32768 tokens
+        sweep = []
+        for S in (512, 1024, 2048, 4096, 8192, 16384, 32768):
+            wl = synth.Workload("sweep_S%d" % S, 32768 // S, 32, 8, S, 128, theta=5.0e5, seed_id=50)
+            ms_f, ss = fwd_ms(wl, True)
+            ms_s, _ = fwd_ms(wl, False, ss)
+            sweep.append({"S": S, "B": wl.B, "fused_ms": ms_f, "separate_ms": ms_s, "speedup_fused": ms_s / ms_f,
+                          "fused_tflops": wl.fwd_flops() / ms_f / 1e9})
+            del ss
+            torch.cuda.empty_cache()
+        ex["rotation_calculus_sweep"] = sweep
+        # separate RoPE kernel alone on a larger-than-L2 buffer (HBM roofline)
+        wl = synth.CONFIGS[3]
+        x = torch.randn((wl.B, wl.Hq, wl.S, wl.D), device=dev).to(torch.bfloat16)
+        y = torch.empty_like(x)
+        rr, _, tb = specs(wl)
+        t_r, _, _ = timed(lambda i: af.rope(x, rr, tb, out=y), k_ex, w_ex)
+        gbs = 2 * x.numel() * 2 / (t_r / k_ex * 1e-3) / 1e9
+        ex["rope_apply_kernel"] = {"bytes": 2 * x.numel() * 2, "ms": t_r / k_ex, "GB/s": gbs,
+                                   "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]}
+        line["extras"] = ex
+
+    if rank == 0 and world == 1 and args.cpu_baseline:
+        v, sample, _ = oracle_rate(w, 12.0)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+                                "sample": sample}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
