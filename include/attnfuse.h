@@ -36,7 +36,8 @@ typedef enum {
     AF_ERR_WORKSPACE = 6,       /* workspace missing or too small */
     AF_ERR_ARCH = 7,            /* current device is not compute capability 10.x */
     AF_ERR_CUDA = 8,            /* a CUDA runtime / driver call failed */
-    AF_ERR_DEVICE_TIMEOUT = 9   /* a bounded device-side wait ran out in an earlier launch */
+    AF_ERR_DEVICE_TIMEOUT = 9,  /* a bounded device-side wait ran out in an earlier launch */
+    AF_ERR_STATIC_LIMIT = 10    /* attnfuse_bwd_static: B*Hq*S exceeds AF_BWD_STATIC_MAX_ROWS */
 } af_status;
 
 typedef enum { AF_BF16 = 0, AF_F32 = 1 } af_dtype;
@@ -117,6 +118,31 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
                        int gqa_group, float softmax_scale,
                        void* dq, af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---- backward without a caller workspace (the paper has no counterpart) ---------------------------
+ * Some callers are not allowed to obtain device memory at the point where they need the backward:
+ * a plug-in that runs inside another framework's enqueue hook, a serving loop whose memory pool was
+ * frozen at start-up, code that runs while the allocator is locked by someone else.  For them this
+ * variant of attnfuse_bwd keeps the one piece of scratch the backward needs (delta, one fp32 per
+ * query row) in a fixed array inside the library instead of a caller workspace.  Inputs and outputs
+ * are still the caller's, exactly as for attnfuse_bwd, and the results are the same.
+ *
+ *  - Limit: B*Hq*S <= AF_BWD_STATIC_MAX_ROWS (4 MiB of scratch, which every GPU that loads the library
+ *    holds until the process exits).  Larger problems return AF_ERR_STATIC_LIMIT and launch nothing.
+ *  - The call allocates and frees nothing, on the host side of CUDA or through any library.
+ *  - The first call on each device looks up the device address of the array (with that device
+ *    current) and remembers it; make that first call outside any stream capture.
+ *  - All calls on a device share the array and it keeps whatever the previous call left there.  Nothing
+ *    in it has to start at zero (each call overwrites the part it reads), but two calls that overlap
+ *    on the GPU (different streams, no ordering between them) race on it: order them. */
+#define AF_BWD_STATIC_MAX_ROWS (1 << 20)
+af_status attnfuse_bwd_static(const af_shape* shape, const void* q, const void* k, const void* v,
+                              const void* o, const float* lse, const void* d_o,
+                              const af_strides* sq, const af_strides* skv,
+                              const af_rope* rope, const void* rope_table, const af_mask* mask,
+                              int gqa_group, float softmax_scale,
+                              void* dq, af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
+                              void* cuda_stream);
 
 #ifdef __cplusplus
 }

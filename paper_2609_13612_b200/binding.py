@@ -86,6 +86,9 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_bwd.restype = i
         L.attnfuse_bwd.argtypes = [P(_Shape), vp, vp, vp, vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp,
                                    P(_Mask), i, f, vp, i, vp, vp, i, vp, sz, vp]
+        L.attnfuse_bwd_static.restype = i
+        L.attnfuse_bwd_static.argtypes = [P(_Shape), vp, vp, vp, vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp,
+                                          P(_Mask), i, f, vp, i, vp, vp, i, vp]
         _lib = L
     return _lib
 
@@ -231,4 +234,32 @@ def bwd(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softma
                               table.data_ptr() if table is not None else None, ctypes.byref(m), Hq // Hkv,
                               float(softmax_scale), dq.data_ptr(), code(dq_dtype), dk.data_ptr(), dv.data_ptr(),
                               code(dkv_dtype), workspace.data_ptr(), workspace.numel(), _stream()))
+    return dq, dk, dv
+
+
+BWD_STATIC_MAX_ROWS = 1 << 20
+
+
+def bwd_static(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softmax_scale: float,
+               dq: torch.Tensor, dk: torch.Tensor, dv: torch.Tensor):
+    """Backward for callers that must not allocate: no workspace argument, the scratch lives inside
+    the library (B*Hq*S <= BWD_STATIC_MAX_ROWS).  The caller passes the output tensors; this wrapper
+    creates no tensor either.  Calls on one device share that scratch, so do not let two of them
+    overlap on the GPU."""
+    _need_cuda(q, k, v, o, lse, d_o, table, dq, dk, dv)
+    B, Hq, S, D = q.shape
+    Hkv = k.shape[1]
+    assert o.is_contiguous() and d_o.is_contiguous() and lse.is_contiguous()
+    assert dq.is_contiguous() and dk.is_contiguous() and dv.is_contiguous() and dk.dtype == dv.dtype
+    assert dq.shape == q.shape and dk.shape == k.shape and dv.shape == v.shape
+    sh = _Shape(B, Hq, Hkv, S, D)
+    sq, skv = _strides(q), _strides(k)
+    r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
+    m = _mask_struct(mask)
+    code = lambda dt: AF_F32 if dt == torch.float32 else AF_BF16
+    _check(lib().attnfuse_bwd_static(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                     lse.data_ptr(), d_o.data_ptr(), ctypes.byref(sq), ctypes.byref(skv),
+                                     ctypes.byref(r), table.data_ptr() if table is not None else None,
+                                     ctypes.byref(m), Hq // Hkv, float(softmax_scale), dq.data_ptr(), code(dq.dtype),
+                                     dk.data_ptr(), dv.data_ptr(), code(dk.dtype), _stream()))
     return dq, dk, dv

@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>
+#include <mutex>
 #include <stdlib.h>
 #include <string.h>
 
@@ -177,6 +178,8 @@ const char* attnfuse_strerror(af_status st) {
         case AF_ERR_ARCH: return "device is not compute capability 10.x";
         case AF_ERR_CUDA: return "CUDA call failed";
         case AF_ERR_DEVICE_TIMEOUT: return "bounded device-side wait ran out";
+        case AF_ERR_STATIC_LIMIT:
+            return "attnfuse_bwd_static: B*Hq*S exceeds AF_BWD_STATIC_MAX_ROWS (use attnfuse_bwd with a workspace)";
     }
     return "unknown status";
 }
@@ -358,3 +361,44 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------
+// Backward for callers that cannot obtain device memory when they call: the scratch (delta) lives in
+// a fixed device array of this library.  In host code the array's name is only a stand-in for the
+// symbol, not a device address, so its address is looked up once per device and passed on as a
+// pointer.  Every call on a device shares the array; see the header for the rules.
+static __device__ __align__(256) unsigned char g_bwd_static_scratch[AF_BWD_STATIC_MAX_ROWS * sizeof(float) + 256];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_bwd_static_ptr[kMaxDevices] = {};
+std::mutex g_bwd_static_mutex;
+}  // namespace
+
+extern "C" af_status attnfuse_bwd_static(const af_shape* shape, const void* q, const void* k, const void* v,
+                                         const void* o, const float* lse, const void* d_o, const af_strides* sq,
+                                         const af_strides* skv, const af_rope* rope, const void* rope_table,
+                                         const af_mask* mask, int gqa_group, float softmax_scale, void* dq,
+                                         af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
+                                         void* cuda_stream) {
+    if (!shape) return AF_ERR_NULL;
+    if (shape->B < 1 || shape->Hq < 1 || shape->S < 1) return AF_ERR_SHAPE;
+    const long long rows = static_cast<long long>(shape->B) * shape->Hq * shape->S;
+    if (rows > AF_BWD_STATIC_MAX_ROWS) return AF_ERR_STATIC_LIMIT;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return AF_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return AF_ERR_CUDA;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_bwd_static_mutex);
+        if (!g_bwd_static_ptr[dev]) {
+            // once per device, with that device current
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_bwd_static_scratch) != cudaSuccess || !ptr) return AF_ERR_CUDA;
+            g_bwd_static_ptr[dev] = ptr;
+        }
+        scratch = g_bwd_static_ptr[dev];
+    }
+    return attnfuse_bwd(shape, q, k, v, o, lse, d_o, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, dq,
+                        dq_dtype, dk, dv, dkv_dtype, scratch, sizeof(g_bwd_static_scratch), cuda_stream);
+}
