@@ -271,14 +271,17 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 else rotate_tile_smem(sX, x0, p.S, p.R, p.table, t, 128);
                 fence_proxy_async_smem();
                 mbar_arrive(&bars[L::B_XROT]);
+                RotState<CPT> nx;
+                if (CP > 0 && n_it > 0) rotate_prefetch(st, p.table, stream_row0(0), p.S, p.R, t);
                 for (int n = 0; n < n_it; ++n) {
                     const int sg = n % NST, a0 = stream_row0(n);
-                    if (CP > 0) rotate_prefetch(st, p.table, a0, p.S, p.R, t);
+                    if (CP > 0 && n + 1 < n_it) rotate_prefetch(nx, p.table, stream_row0(n + 1), p.S, p.R, t);
                     if (!mbar_wait(&bars[L::B_AFULL + sg], (n / NST) & 1, abort_flag, 28)) return;
                     if (CP > 0) rotate_tile_fast(sA + sg * TILE, st, step, t);
                     else rotate_tile_smem(sA + sg * TILE, a0, p.S, p.R, p.table, t, 128);
                     fence_proxy_async_smem();
                     mbar_arrive(&bars[L::B_AROT + sg]);
+                    if (CP > 0) st = nx;
                 }
             };
             if (p.R == 128) run(std::integral_constant<int, 8>{});
@@ -317,6 +320,15 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             }
             const int i0 = DKV ? a0 : x0, j0 = DKV ? x0 : a0;
             const bool need_mask = tile_needs_mask(ms, i0, j0);
+            int mlo = 0;
+            uint32_t mn = 128;
+            if (need_mask) {
+                if (DKV) kept_queries_of_key(ms, xrow, a0, mlo, mn);
+                else kept_keys_of_query(ms, xrow, a0, mlo, mn);
+            }
+            // ALiBi: slope2 * (j - i) = sb * (col + base), sb = +-slope2
+            const float sb = DKV ? -my_slope2 : my_slope2;
+            const float bias_base = sb * static_cast<float>(DKV ? a0 - xrow : a0 - xrow);
             ok = wg_all(mbar_wait(&bars[L::B_TFULL], n & 1, abort_flag, 29));  // also publishes the statistics
             if (!ok) break;
             tc_fence_after_sync();
@@ -326,18 +338,18 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 tmem_ld32(tb + T1 + c * 32, s);
                 tmem_ld32(tb + T2 + c * 32, dp);
                 tmem_wait_ld();
+                const float cbias = fmaf(sb, static_cast<float>(c * 32), bias_base);
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
                     float pv[2], dv[2];
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         const int col = c * 32 + e + u;
-                        const int i = DKV ? a0 + col : xrow, j = DKV ? xrow : a0 + col;
                         const float l2 = DKV ? sL2[col] : my_l2, dl = DKV ? sDl[col] : my_delta;
-                        float t = fmaf(__uint_as_float(s[e + u]), p.scale_log2, -l2);
-                        if (alibi) t = fmaf(my_slope2, static_cast<float>(j - i), t);
+                        float t = fmaf(__uint_as_float(s[e + u]), p.scale_log2, cbias - l2);
+                        if (alibi) t = fmaf(sb, static_cast<float>(e + u), t);
                         float pe = ex2(t);
-                        if (need_mask && !pair_kept(ms, i, j)) pe = 0.f;
+                        if (need_mask) pe = (static_cast<uint32_t>(col - mlo) < mn) ? pe : 0.f;
                         pv[u] = pe;
                         dv[u] = pe * (__uint_as_float(dp[e + u]) - dl);
                     }

@@ -57,6 +57,34 @@ __device__ __forceinline__ bool pair_kept(const MaskSpec& m, int i, int j) {
     return true;
 }
 
+// For a fixed row of a tile pair the kept columns form one interval (causal, window and the sequence
+// end are all half-lines in the column index).  Returns lo and the width n: column e (0..127) is kept
+// iff (unsigned)(e - lo) < n.
+//   Query-major tiles (lane = query i, column = key j0 + e):     kept_keys_of_query
+//   Key-major tiles   (lane = key j,   column = query i0 + e):   kept_queries_of_key
+__device__ __forceinline__ void kept_keys_of_query(const MaskSpec& m, int i, int j0, int& lo, uint32_t& n) {
+    const int d = i - j0;
+    int hi = min(BN - 1, m.S - 1 - j0);
+    lo = 0;
+    if (m.causal) hi = min(hi, d);
+    if (m.window >= 0) {
+        lo = max(lo, d - m.window);
+        if (!m.causal) hi = min(hi, d + m.window);
+    }
+    n = hi >= lo ? static_cast<uint32_t>(hi - lo + 1) : 0u;
+}
+__device__ __forceinline__ void kept_queries_of_key(const MaskSpec& m, int j, int i0, int& lo, uint32_t& n) {
+    const int d = j - i0;
+    int hi = BM - 1;
+    lo = 0;
+    if (m.causal) lo = max(lo, d);
+    if (m.window >= 0) {
+        hi = min(hi, d + m.window);
+        if (!m.causal) lo = max(lo, d - m.window);
+    }
+    n = (hi >= lo && j < m.S) ? static_cast<uint32_t>(hi - lo + 1) : 0u;
+}
+
 // Byte offset of the 16-byte chunk `chunk` (8 bf16 columns) of row `r` inside a tile made of
 // D/64 TMA boxes, each [128 rows][64 cols] with the 128-byte swizzle.
 __device__ __forceinline__ uint32_t swz_chunk_offset(int r, int chunk) {

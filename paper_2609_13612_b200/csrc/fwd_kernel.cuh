@@ -42,14 +42,14 @@ struct FwdSmem {
 
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the row max grows by more
 
-// One key tile of the online softmax for one query row (this thread's TMEM lane):
-// reads the 128 raw scores, applies scale / ALiBi / mask in the log2 domain, updates the running
-// max and sum, writes P (bf16) over S and, when the reference max moved, rescales O.
+// One key tile of the online softmax for one query row (this thread's TMEM lane): reads the 128
+// raw scores, adds ALiBi and the mask in the raw domain, updates the running max and sum in the
+// log2 domain, writes P (bf16) over S and, when the reference max moved, rescales O.
 // MASKED / ALIBI select straight-line code: interior tiles carry no mask logic at all.
+//   score (log2 domain) t_e = c2 * (S_e + kb * e) + bias0,  kb = slope2 / c2, bias0 = slope2 * (j0 - i)
 template <int D, bool MASKED, bool ALIBI>
-__device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, float scale_log2, float slope2,
-                                             float bias0, int i, int j0, const MaskSpec& ms, float& m_run,
-                                             float& l_run) {
+__device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, float scale_log2, float kb,
+                                             float bias0, int mlo, uint32_t mn, float& m_run, float& l_run) {
     uint32_t v[BN];
     tmem_ld32(tS, v);
     tmem_ld32(tS + 32, v + 32);
@@ -57,21 +57,16 @@ __device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, fl
     tmem_ld32(tS + 96, v + 96);
     tmem_wait_ld();
     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-    if (!MASKED && !ALIBI) {
 #pragma unroll
-        for (int e = 0; e < BN; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(v[e]));
-    } else {
-#pragma unroll
-        for (int e = 0; e < BN; ++e) {
-            float t = __uint_as_float(v[e]) * scale_log2;
-            if (ALIBI) t = fmaf(slope2, static_cast<float>(e), t + bias0);
-            if (MASKED) t = pair_kept(ms, i, j0 + e) ? t : -INFINITY;
-            v[e] = __float_as_uint(t);
-            mx4[e & 3] = fmaxf(mx4[e & 3], t);
-        }
+    for (int e = 0; e < BN; ++e) {
+        float sv = __uint_as_float(v[e]);
+        if (ALIBI) sv = fmaf(kb, static_cast<float>(e), sv);
+        if (MASKED) sv = (static_cast<uint32_t>(e - mlo) < mn) ? sv : -INFINITY;
+        if (ALIBI || MASKED) v[e] = __float_as_uint(sv);
+        mx4[e & 3] = fmaxf(mx4[e & 3], sv);
     }
-    float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-    if (!MASKED && !ALIBI) mx *= scale_log2;  // scale > 0: max commutes with it
+    // scale > 0, so the max commutes with it
+    const float mx = fmaf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])), scale_log2, bias0);
     // lazy rescale: keep the old reference max unless it grew by more than the threshold
     const bool upd = mx > m_run + kRescaleThreshold;
     float alpha = 1.f;
@@ -79,20 +74,13 @@ __device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, fl
         alpha = ex2(m_run - mx);  // m_run = -inf -> 0
         m_run = mx;
     }
-    const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+    const float sub = bias0 - ((m_run == -INFINITY) ? 0.f : m_run);
     float ps4[4] = {0.f, 0.f, 0.f, 0.f};
     uint32_t pk[BN / 2];
 #pragma unroll
     for (int e = 0; e < BN; e += 2) {
-        float t0, t1;
-        if (!MASKED && !ALIBI) {
-            t0 = fmaf(__uint_as_float(v[e]), scale_log2, -m_use);
-            t1 = fmaf(__uint_as_float(v[e + 1]), scale_log2, -m_use);
-        } else {
-            t0 = __uint_as_float(v[e]) - m_use;
-            t1 = __uint_as_float(v[e + 1]) - m_use;
-        }
-        const float p0 = ex2(t0), p1 = ex2(t1);
+        const float p0 = ex2(fmaf(__uint_as_float(v[e]), scale_log2, sub));
+        const float p1 = ex2(fmaf(__uint_as_float(v[e + 1]), scale_log2, sub));
         ps4[(e >> 1) & 3] += p0 + p1;
         pk[e >> 1] = pack_bf16x2(p0, p1);
     }
@@ -177,7 +165,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // Register budget: the softmax warpgroups hold a full row of 128 scores; the others need little.
     constexpr int kSoftmaxRegs = NQ == 2 ? 176 : 232;
 
-    if (warp < 4) setmaxnreg_dec<56>();
+    if (warp < 4) setmaxnreg_dec<64>();
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -282,7 +270,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------ rotation warpgroup (Section 4.1)
-        setmaxnreg_dec<104>();
+        setmaxnreg_dec<96>();
         if (ROPE) {
             const int t = threadIdx.x - 128;
             auto run = [&](auto cp_tag) {
@@ -302,15 +290,20 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     fence_proxy_async_smem();
                     mbar_arrive(&bars[L::B_QROT + q]);
                 }
+                // K tiles: the table row of tile it+1 is fetched before tile it is rotated, so its
+                // latency never sits between a tile landing and its rotation
+                RotState<(CP > 0 ? CP : 1)> nx;
+                if (CP > 0 && ok && n_it > 0) rotate_prefetch(st, p.table, jlo_c * BN, p.S, p.R, t);
                 for (int it = 0; ok && it < n_it; ++it) {
                     const int ks = it % KS;
-                    if (CP > 0) rotate_prefetch(st, p.table, (jlo_c + it) * BN, p.S, p.R, t);
+                    if (CP > 0 && it + 1 < n_it) rotate_prefetch(nx, p.table, (jlo_c + it + 1) * BN, p.S, p.R, t);
                     ok = mbar_wait(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
                     if (!ok) break;
                     if (CP > 0) rotate_tile_fast(sK + ks * TILE, st, step, t);
                     else rotate_tile_smem(sK + ks * TILE, (jlo_c + it) * BN, p.S, p.R, p.table, t, 128);
                     fence_proxy_async_smem();
                     mbar_arrive(&bars[L::B_KROT + ks]);
+                    if (CP > 0) st = nx;
                 }
             };
             if (p.R == 128) run(std::integral_constant<int, 8>{});
@@ -330,6 +323,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int i = i0[q] + row;
         const float slope2 = p.slopes ? p.slopes[h] * 1.4426950408889634f : 0.f;
         const bool alibi = p.slopes != nullptr;
+        const float kb = slope2 / p.scale_log2;
         float m_run = -INFINITY, l_run = 0.f;
         bool ok = true;
         int n = 0;
@@ -340,12 +334,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tc_fence_after_sync();
             const bool need_mask = tile_needs_mask(ms, i0[q], j0);
             const float bias0 = slope2 * static_cast<float>(j0 - i);
+            int mlo = 0;
+            uint32_t mn = BN;
+            if (need_mask) kept_keys_of_query(ms, i, j0, mlo, mn);
             if (alibi) {
-                if (need_mask) softmax_tile<D, true, true>(tS, tO, n, p.scale_log2, slope2, bias0, i, j0, ms, m_run, l_run);
-                else softmax_tile<D, false, true>(tS, tO, n, p.scale_log2, slope2, bias0, i, j0, ms, m_run, l_run);
+                if (need_mask) softmax_tile<D, true, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
+                else softmax_tile<D, false, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
             } else {
-                if (need_mask) softmax_tile<D, true, false>(tS, tO, n, p.scale_log2, slope2, bias0, i, j0, ms, m_run, l_run);
-                else softmax_tile<D, false, false>(tS, tO, n, p.scale_log2, slope2, bias0, i, j0, ms, m_run, l_run);
+                if (need_mask) softmax_tile<D, true, false>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
+                else softmax_tile<D, false, false>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
             }
             tc_fence_before_sync();
             mbar_arrive(&bars[L::B_PREADY + q]);
