@@ -271,6 +271,9 @@ af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, cons
     p.table = static_cast<const float2*>(rope_table);
     p.o = o; p.o_f32 = (o_dtype == AF_F32); p.lse = lse;
     p.n_row_blocks = 0;
+#ifdef AF_TRACE
+    p.trace = reinterpret_cast<long long*>(getenv("AF_TRACE_PTR") ? strtoull(getenv("AF_TRACE_PTR"), nullptr, 0) : 0ull);
+#endif
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     return shape->D == 128 ? launch_fwd<128>(tq, tk, tv, p, stream) : launch_fwd<64>(tq, tk, tv, p, stream);
 }

@@ -164,7 +164,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::N_BARS; ++i) {
             uint32_t cnt = 1;
-            if (i == L::B_XROT || (i >= L::B_AROT && i < L::B_AROT + NST) || i == L::B_PDS) cnt = 128;
+            if (i == L::B_XROT || (i >= L::B_AROT && i < L::B_AROT + NST) || i == L::B_PDS) cnt = 4;  // per-warp arrives
             mbar_init(&bars[i], cnt);
         }
         *abort_flag = 0;
@@ -265,23 +265,24 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                     rotate_load_step<CPT>(p.table, p.S, p.R, t, step);
                     rotate_prefetch(st, p.table, x0, p.S, p.R, t);
                 }
-                bool ok = mbar_wait(&bars[L::B_XFULL], 0, abort_flag, 27);
+                bool ok = mbar_wait_warp(&bars[L::B_XFULL], 0, abort_flag, 27);
                 if (!ok) return;
                 if (CP > 0) rotate_tile_fast(sX, st, step, t);
                 else rotate_tile_smem(sX, x0, p.S, p.R, p.table, t, 128);
                 fence_proxy_async_smem();
-                mbar_arrive(&bars[L::B_XROT]);
-                RotState<CPT> nx;
-                if (CP > 0 && n_it > 0) rotate_prefetch(st, p.table, stream_row0(0), p.S, p.R, t);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[L::B_XROT]);
+                // streamed tiles are consecutive within a head: the recurrence carries the state along
                 for (int n = 0; n < n_it; ++n) {
                     const int sg = n % NST, a0 = stream_row0(n);
-                    if (CP > 0 && n + 1 < n_it) rotate_prefetch(nx, p.table, stream_row0(n + 1), p.S, p.R, t);
-                    if (!mbar_wait(&bars[L::B_AFULL + sg], (n / NST) & 1, abort_flag, 28)) return;
+                    const int run_pos = DKV ? n % per_head : n;
+                    if (CP > 0 && (run_pos % kRotResync) == 0) rotate_prefetch(st, p.table, a0, p.S, p.R, t);
+                    if (!mbar_wait_warp(&bars[L::B_AFULL + sg], (n / NST) & 1, abort_flag, 28)) return;
                     if (CP > 0) rotate_tile_fast(sA + sg * TILE, st, step, t);
                     else rotate_tile_smem(sA + sg * TILE, a0, p.S, p.R, p.table, t, 128);
                     fence_proxy_async_smem();
-                    mbar_arrive(&bars[L::B_AROT + sg]);
-                    if (CP > 0) st = nx;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars[L::B_AROT + sg]);
                 }
             };
             if (p.R == 128) run(std::integral_constant<int, 8>{});
@@ -365,7 +366,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             }
             tmem_wait_st();
             tc_fence_before_sync();
-            mbar_arrive(&bars[L::B_PDS]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars[L::B_PDS]);
         }
         // epilogue: stage through shared memory (the stream stages are idle now), rotate back, store
         if (ok && n_it > 0) ok = wg_all(mbar_wait(&bars[L::B_DONE], 0, abort_flag, 30));

@@ -133,7 +133,11 @@ __device__ __forceinline__ void rotate_tile_smem(uint8_t* tile, int row0, int S,
 // (RP = 128 / CP).  It reads the table once, for its first row, and walks to the next rows with the
 // angle-addition recurrence (cos, sin)(a + d) from (cos, sin)(a) and the constant (cos, sin)(d),
 // d = RP * theta_i, which the table carries as a trailer row.  The first-row read is split off
-// (rotate_prefetch) so that it can be issued before waiting for the tile to land.
+// (rotate_prefetch) so that it can be issued before waiting for the tile to land.  After a tile the
+// state has advanced by 128 rows, i.e. to the thread's first row of the next consecutive tile, so a
+// run of consecutive tiles needs no table read at all; callers re-read the table every
+// kRotResync tiles to keep the accumulated rounding of the recurrence far below bf16 resolution.
+constexpr int kRotResync = 16;
 template <int CP>
 struct RotState {
     float4 t[4];     // {cos, sin} x 8 frequencies at the current row
@@ -183,12 +187,11 @@ __device__ __forceinline__ void rotate_tile_fast(uint8_t* tile, RotState<CP>& st
             rotate_word(lo[u].y, hi[u].y, st.t[1].x, st.t[1].y, st.t[1].z, st.t[1].w);
             rotate_word(lo[u].z, hi[u].z, st.t[2].x, st.t[2].y, st.t[2].z, st.t[2].w);
             rotate_word(lo[u].w, hi[u].w, st.t[3].x, st.t[3].y, st.t[3].z, st.t[3].w);
-            if (k0 + u + 1 < CP) {
+            // after the last row the state sits RP * CP = 128 rows further: the same row of the next tile
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    advance_cs(st.t[w].x, st.t[w].y, step[w].x, step[w].y);
-                    advance_cs(st.t[w].z, st.t[w].w, step[w].z, step[w].w);
-                }
+            for (int w = 0; w < 4; ++w) {
+                advance_cs(st.t[w].x, st.t[w].y, step[w].x, step[w].y);
+                advance_cs(st.t[w].z, st.t[w].w, step[w].z, step[w].w);
             }
         }
 #pragma unroll

@@ -22,6 +22,9 @@ struct FwdParams {
     int o_f32;
     float* lse;         // nullable
     int n_row_blocks;   // ceil(S / (128 * NQ))
+#ifdef AF_TRACE
+    long long* trace;
+#endif
 };
 
 template <int D, int NQ, int KS, int VS>
@@ -39,6 +42,18 @@ struct FwdSmem {
     static constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;
     static constexpr int BYTES = OFF_MISC + 16 + 1024;  // + alignment slack
 };
+
+// Optional timeline instrumentation for tuning (compiled out unless AF_TRACE is defined): one CTA
+// records SM-clock stamps per role, iteration and phase into a caller-provided buffer.
+#ifdef AF_TRACE
+#define AF_STAMP(role, it, ph)                                                                         \
+    do {                                                                                               \
+        if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && (it) < 64)     \
+            p.trace[((role) * 64 + (it)) * 8 + (ph)] = clock64();                                      \
+    } while (0)
+#else
+#define AF_STAMP(role, it, ph) do { } while (0)
+#endif
 
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the row max grows by more
 
@@ -141,13 +156,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     }
     const int n_it = jhi_c - jlo_c + 1;
+    AF_STAMP(0, 63, 0);  // kernel entry
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::N_BARS; ++i) {
             uint32_t cnt = 1;
             if ((i >= L::B_QROT && i < L::B_QROT + NQ) || (i >= L::B_KROT && i < L::B_KROT + KS) ||
                 (i >= L::B_PREADY && i < L::B_PREADY + NQ))
-                cnt = 128;
+                cnt = 4;  // one elected arrive per warp of the producing warpgroup
             mbar_init(&bars[i], cnt);
         }
         *abort_flag = 0;
@@ -229,7 +245,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
             for (int q = 0; q < NQ; ++q)
                 if (ok && jhi[q] >= jlo[q]) ok = mbar_wait(&bars[B_QREADY + q], 0, abort_flag, 3);
+            AF_STAMP(0, 63, 2);  // Q ready
             if (ok) ok = mbar_wait(&bars[B_KREADY + 0], 0, abort_flag, 4);
+            AF_STAMP(0, 63, 3);  // first K ready
             if (ok) {
                 tc_fence_after_sync();
 #pragma unroll
@@ -241,14 +259,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const int j = jlo_c + it, vs = it % VS, ks1 = (it + 1) % KS;
                 const bool next = it + 1 < n_it;
                 bool kwaited = false;
+                AF_STAMP(0, it, 0);
                 ok = mbar_wait(&bars[L::B_VFULL + vs], (it / VS) & 1, abort_flag, 5);
+                AF_STAMP(0, it, 1);
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
                     if (ok && j >= jlo[q] && j <= jhi[q]) {
                         ok = mbar_wait(&bars[L::B_PREADY + q], cnt[q] & 1, abort_flag, 6);
+                        AF_STAMP(0, it, 2 + 3 * q);
                         if (ok) {
                             tc_fence_after_sync();
                             issue_O(q, vs, cnt[q] > 0);
+                            AF_STAMP(0, it, 3 + 3 * q);
                             ++cnt[q];
                             if (j == jhi[q]) mma_commit(&bars[L::B_ODONE + q]);
                         }
@@ -260,6 +282,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             kwaited = true;
                         }
                         if (ok) issue_S(q, ks1);
+                        AF_STAMP(0, it, 4 + 3 * q);
                     }
                 }
                 if (ok) {
@@ -283,27 +306,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int q = 0; q < NQ; ++q) {
                     if (!ok || jhi[q] < jlo[q]) continue;
                     if (CP > 0) rotate_prefetch(st, p.table, i0[q], p.S, p.R, t);
-                    ok = mbar_wait(&bars[L::B_QFULL + q], 0, abort_flag, 8);
+                    ok = mbar_wait_warp(&bars[L::B_QFULL + q], 0, abort_flag, 8);
                     if (!ok) break;
                     if (CP > 0) rotate_tile_fast(sQ + q * TILE, st, step, t);
                     else rotate_tile_smem(sQ + q * TILE, i0[q], p.S, p.R, p.table, t, 128);
                     fence_proxy_async_smem();
-                    mbar_arrive(&bars[L::B_QROT + q]);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars[L::B_QROT + q]);
                 }
-                // K tiles: the table row of tile it+1 is fetched before tile it is rotated, so its
-                // latency never sits between a tile landing and its rotation
-                RotState<(CP > 0 ? CP : 1)> nx;
-                if (CP > 0 && ok && n_it > 0) rotate_prefetch(st, p.table, jlo_c * BN, p.S, p.R, t);
+                // K tiles are consecutive: the recurrence carries the cos/sin state from tile to tile
                 for (int it = 0; ok && it < n_it; ++it) {
                     const int ks = it % KS;
-                    if (CP > 0 && it + 1 < n_it) rotate_prefetch(nx, p.table, (jlo_c + it + 1) * BN, p.S, p.R, t);
-                    ok = mbar_wait(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
+                    if (CP > 0 && (it % kRotResync) == 0) rotate_prefetch(st, p.table, (jlo_c + it) * BN, p.S, p.R, t);
+                    AF_STAMP(1, it, 0);
+                    ok = mbar_wait_warp(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
+                    AF_STAMP(1, it, 1);
                     if (!ok) break;
                     if (CP > 0) rotate_tile_fast(sK + ks * TILE, st, step, t);
                     else rotate_tile_smem(sK + ks * TILE, (jlo_c + it) * BN, p.S, p.R, p.table, t, 128);
                     fence_proxy_async_smem();
-                    mbar_arrive(&bars[L::B_KROT + ks]);
-                    if (CP > 0) st = nx;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars[L::B_KROT + ks]);
+                    AF_STAMP(1, it, 2);
                 }
             };
             if (p.R == 128) run(std::integral_constant<int, 8>{});
@@ -329,7 +353,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         int n = 0;
         for (int j = jlo[q]; ok && j <= jhi[q]; ++j, ++n) {
             const int j0 = j * BN;
-            ok = mbar_wait(&bars[L::B_SFULL + q], n & 1, abort_flag, 10);
+            AF_STAMP(2 + q, n, 0);
+            ok = mbar_wait_warp(&bars[L::B_SFULL + q], n & 1, abort_flag, 10);
+            AF_STAMP(2 + q, n, 1);
             if (!ok) break;
             tc_fence_after_sync();
             const bool need_mask = tile_needs_mask(ms, i0[q], j0);
@@ -345,10 +371,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 else softmax_tile<D, false, false>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
             }
             tc_fence_before_sync();
-            mbar_arrive(&bars[L::B_PREADY + q]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars[L::B_PREADY + q]);
+            AF_STAMP(2 + q, n, 2);
         }
         // epilogue (Section 4.4: save L = m + ln l)
-        if (ok && jhi[q] >= jlo[q]) ok = mbar_wait(&bars[L::B_ODONE + q], 0, abort_flag, 11);
+        if (ok && jhi[q] >= jlo[q]) ok = mbar_wait_warp(&bars[L::B_ODONE + q], 0, abort_flag, 11);
+        AF_STAMP(2 + q, 63, 0);  // O complete
         if (ok && jhi[q] >= jlo[q]) {
             tc_fence_after_sync();
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
@@ -385,6 +414,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     tc_fence_before_sync();
     __syncthreads();
+    AF_STAMP(0, 63, 1);  // all roles done
     if (warp == 1) {
         __syncwarp();
         tmem_dealloc(tmem_base, TMEM_COLS);

@@ -66,6 +66,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
 }
 
+// Warp-uniform variant for roles whose warps synchronise internally (__syncwarp, elected arrives,
+// warp-collective tcgen05.ld/st): all 32 lanes wait, and all of them give up if any of them did.
+// (Letting only lane 0 poll was measured slower: the warp woke up later.)
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                               uint32_t code) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, code));
+}
+
 // ---------------------------------------------------------------- proxies and fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
