@@ -38,7 +38,7 @@ UNIT = "TFLOP/s"
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes per launch of the forward kernel on this workload, from the ncu capture summarised in
 # profiles/attn_fwd_kernel_c2_llama3_8b.md (dram__bytes_read.sum + dram__bytes_write.sum).
-FWD_TRAFFIC_BYTES_PER_LAUNCH = None
+FWD_TRAFFIC_BYTES_PER_LAUNCH = 54.0e6
 PAPER_CONTEXT = {
     "rtx3090_fused_vs_flex_prerotate_rope_causal": "2.10x (RTX 3090, fp16, B=4 H=12 D=64, N=4096)",
     "h100_llama3_8b_training_step_vs_sdpa": "within ~5% (H100 NVL, fp16, N=2048: 7.65 ms vs 7.27 ms)",
@@ -159,6 +159,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--extras", type=int, default=1, help="also time configs 3-5, the separate-RoPE arm and the sweep")
     ap.add_argument("--cpu-baseline", type=int, default=1)
+    ap.add_argument("--profile", default="", choices=["", "fwd", "bwd", "rope"],
+                    help="run only a few launches of one path (for ncu captures) and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = synth.CONFIGS[1]
@@ -236,6 +238,22 @@ def main():
             dist.all_reduce(tt, op=dist.ReduceOp.MAX)
             total_ms = float(tt.item())
         return total_ms, per, wall_ms
+
+    if args.profile:
+        # a handful of launches of one path on its configuration, nothing else: the target of ncu captures
+        wl = {"fwd": synth.CONFIGS[1], "bwd": synth.CONFIGS[4], "rope": synth.CONFIGS[3]}[args.profile]
+        r, m, tb = specs(wl)
+        t = {k: to_dev(v) for k, v in synth.draw_all(wl).items()}
+        for _ in range(3):
+            if args.profile == "rope":
+                af.rope(t["q"], r, tb)
+            else:
+                o_, l_ = af.fwd(t["q"], t["k"], t["v"], r, tb, m, wl.scale)
+                if args.profile == "bwd":
+                    af.bwd(t["q"], t["k"], t["v"], o_, l_, t["do"], r, tb, m, wl.scale)
+        torch.cuda.synchronize()
+        print(json.dumps({"profile": args.profile, "workload": wl.name, "device_status": af.device_status()[0]}))
+        return
 
     # ------------------------------------------------------------------ headline: fused forward, config 2
     rope, mask, table = specs(w)
