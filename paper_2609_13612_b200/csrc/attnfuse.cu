@@ -133,7 +133,7 @@ af_status launch_bwd_variant(const CUtensorMap& tx, const CUtensorMap& ty, const
             return AF_ERR_CUDA;
         configured = true;
     }
-    kern<<<grid, 384, L::BYTES, stream>>>(tx, ty, ta, tb, p);
+    kern<<<grid, 512, L::BYTES, stream>>>(tx, ty, ta, tb, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 

@@ -11,6 +11,9 @@
 //   T1 = X A^T  (scores or their transpose),  T2 = Y Bc^T  (dP or its transpose)
 //   P = 2^(c2 T1 + bias - L2), dS = P (T2 - delta); P, dS go back to TMEM as bf16 over T1, T2
 //   DKV: acc1 += P Bc, acc2 += dS A.      DQ: acc1 += dS A.
+// Warp roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-7 rotation, warps 8-11 and
+// 12-15 two gradient warpgroups: each owns 64 of the 128 columns of T1/T2 (all 128 lanes), so the
+// accumulator MMAs of the first half of the contraction start while nothing waits for the second.
 #pragma once
 #include <cuda.h>
 #include <type_traits>
@@ -63,69 +66,73 @@ struct BwdSmem {
     static constexpr int OFF_BAR = OFF_STATS + 2 * 2 * 128 * 4;
     static constexpr int B_XFULL = 0, B_XROT = 1, B_YFULL = 2, B_AFULL = 3, B_AROT = B_AFULL + NST,
                          B_BFULL = B_AROT + NST, B_EMPTY = B_BFULL + NST, B_TFULL = B_EMPTY + NST,
-                         B_PDS = B_TFULL + 1, B_DONE = B_PDS + 1, N_BARS = B_DONE + 1;
+                         B_PDS = B_TFULL + 1, B_DONE = B_PDS + 2, N_BARS = B_DONE + 1;   // B_PDS: one per column half
     static constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;
     static constexpr int BYTES = OFF_MISC + 16 + 1024;
     static constexpr int STG_STRIDE = D + 4;      // floats per staged row (padding keeps 16-byte stores conflict-free)
     static_assert(128 * STG_STRIDE * 4 <= 2 * NST * TILE, "staging buffer must fit in the stream stages");
 };
 
-__device__ __forceinline__ void wg_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-// Barrier over the 128 threads of the gradient warpgroup that also ANDs a flag, so that a wait
+__device__ __forceinline__ void wg_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// Barrier over the 256 threads of the two gradient warpgroups that also ANDs a flag, so that a wait
 // that gave up in one thread ends the loop in all of them (nobody is left alone at a barrier).
 __device__ __forceinline__ bool wg_all(bool v) {
     uint32_t r;
     asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.and.pred q, 1, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.and.pred q, 1, 256, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(r)
         : "r"(static_cast<uint32_t>(v))
         : "memory");
     return r != 0;
 }
 
-// Epilogue helper: the 128 threads of the gradient warpgroup move a [128 x D] fp32 accumulator
-// from TMEM (one row per thread) through shared memory to global memory, scaling it and, when
-// R > 0, applying the transpose rotation for positions row0.. (gradients w.r.t. rotated rows are
-// rotated back).  Global writes are coalesced along D.
+// Epilogue helper: the 256 threads of the two gradient warpgroups move a [128 x D] fp32 accumulator
+// from TMEM (thread gtid reads lane gtid % 128, column half gtid / 128) through shared memory to
+// global memory, scaling it and, when R > 0, applying the transpose rotation for positions row0..
+// (gradients w.r.t. rotated rows are rotated back).  Global writes are coalesced along D.
 template <int D>
-__device__ __forceinline__ void store_acc_rotated(uint32_t t_acc, float* stg, int tid, float mul, int R,
+__device__ __forceinline__ void store_acc_rotated(uint32_t t_acc, float* stg, int gtid, float mul, int R,
                                                   const float2* table, int row0, int S, void* out, size_t out_row0,
                                                   int out_f32) {
     constexpr int STRIDE = BwdSmem<D>::STG_STRIDE;
+    const int lane_row = gtid & 127, chalf = gtid >> 7;
 #pragma unroll 1
-    for (int c = 0; c < D / 32; ++c) {
+    for (int c = 0; c < D / 64; ++c) {
+        const int col = chalf * (D / 2) + c * 32;
         uint32_t v[32];
-        tmem_ld32(t_acc + c * 32, v);
+        tmem_ld32(t_acc + col, v);
         tmem_wait_ld();
-        float4* dst = reinterpret_cast<float4*>(stg + tid * STRIDE + c * 32);
+        float4* dst = reinterpret_cast<float4*>(stg + lane_row * STRIDE + col);
 #pragma unroll
         for (int e = 0; e < 32; e += 4)
             dst[e >> 2] = make_float4(__uint_as_float(v[e]) * mul, __uint_as_float(v[e + 1]) * mul,
                                       __uint_as_float(v[e + 2]) * mul, __uint_as_float(v[e + 3]) * mul);
     }
     wg_sync();
-    constexpr int RPP = 128 / D;  // rows per pass (1 for D = 128, 2 for D = 64)
-    const int d = tid % D, rsub = tid / D;
+    constexpr int RPP = 256 / D;  // rows per pass (2 for D = 128, 4 for D = 64)
+    const int d = gtid % D, rsub = gtid / D;
     const int half = R >> 1;
     const int fi = d < half ? d : d - half;
+#pragma unroll 4
     for (int r = rsub; r < 128; r += RPP) {
         const int row = row0 + r;
-        if (row >= S) break;
-        float y = stg[r * STRIDE + d];
-        if (d < R) {
-            const float2 cs = __ldg(table + static_cast<size_t>(row) * half + fi);
-            const float other = stg[r * STRIDE + (d < half ? d + half : d - half)];
-            y = d < half ? fmaf(y, cs.x, other * cs.y) : fmaf(y, cs.x, -other * cs.y);
+        if (row < S) {
+            float y = stg[r * STRIDE + d];
+            if (d < R) {
+                const float2 cs = __ldg(table + static_cast<size_t>(row) * half + fi);
+                const float other = stg[r * STRIDE + (d < half ? d + half : d - half)];
+                y = d < half ? fmaf(y, cs.x, other * cs.y) : fmaf(y, cs.x, -other * cs.y);
+            }
+            const size_t o = (out_row0 + r) * D + d;
+            if (out_f32) static_cast<float*>(out)[o] = y;
+            else static_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(y);
         }
-        const size_t o = (out_row0 + r) * D + d;
-        if (out_f32) static_cast<float*>(out)[o] = y;
-        else static_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(y);
     }
     wg_sync();
 }
 
 template <int D, bool DKV, bool ROPE>
-__global__ void __launch_bounds__(384, 1)
+__global__ void __launch_bounds__(512, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_y,
                 const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                 const BwdParams p) {
@@ -164,7 +171,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::N_BARS; ++i) {
             uint32_t cnt = 1;
-            if (i == L::B_XROT || (i >= L::B_AROT && i < L::B_AROT + NST) || i == L::B_PDS) cnt = 4;  // per-warp arrives
+            if (i == L::B_XROT || (i >= L::B_AROT && i < L::B_AROT + NST) || i == L::B_PDS || i == L::B_PDS + 1)
+                cnt = 4;  // per-warp arrives
             mbar_init(&bars[i], cnt);
         }
         *abort_flag = 0;
@@ -230,24 +238,32 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                            IDESC_T, kk > 0);
                 }
                 mma_commit(&bars[L::B_TFULL]);
-                ok = mbar_wait(&bars[L::B_PDS], n & 1, abort_flag, 26);
-                if (!ok) break;
-                tc_fence_after_sync();
-                if (DKV) {
+                // the contraction runs over the 128 columns of T1/T2; each gradient warpgroup delivers 64 of
+                // them (4 K = 16 steps), its bf16 results sitting at the start of its own column half
 #pragma unroll
-                    for (int kk = 0; kk < 128 / 16; ++kk)   // acc1 (dV) += P^T dO: dO is the MN-major B operand
-                        mma_ts(tmem_base + ACC1, tmem_base + T1 + kk * 8, smem_desc_sw128(ba + kk * 2048, BOX_BYTES, 1024),
-                               IDESC_ACC, (n > 0 || kk > 0) ? 1u : 0u);
+                for (int hf = 0; hf < 2; ++hf) {
+                    ok = mbar_wait(&bars[L::B_PDS + hf], n & 1, abort_flag, 26);
+                    if (!ok) break;
+                    tc_fence_after_sync();
 #pragma unroll
-                    for (int kk = 0; kk < 128 / 16; ++kk)   // acc2 (dK') += dS^T Q'
-                        mma_ts(tmem_base + ACC2, tmem_base + T2 + kk * 8, smem_desc_sw128(aa + kk * 2048, BOX_BYTES, 1024),
-                               IDESC_ACC, (n > 0 || kk > 0) ? 1u : 0u);
-                } else {
-#pragma unroll
-                    for (int kk = 0; kk < 128 / 16; ++kk)   // acc1 (dQ') += dS K'
-                        mma_ts(tmem_base + ACC1, tmem_base + T1 + kk * 8, smem_desc_sw128(aa + kk * 2048, BOX_BYTES, 1024),
-                               IDESC_ACC, (n > 0 || kk > 0) ? 1u : 0u);
+                    for (int k4 = 0; k4 < 4; ++k4) {
+                        const int kk = hf * 4 + k4;
+                        const uint32_t a_off = hf * 64 + k4 * 8;
+                        const uint32_t acc_on = (n > 0 || kk > 0) ? 1u : 0u;
+                        if (DKV) {
+                            // acc1 (dV) += P^T dO, acc2 (dK') += dS^T Q': dO and Q' are MN-major B operands
+                            mma_ts(tmem_base + ACC1, tmem_base + T1 + a_off, smem_desc_sw128(ba + kk * 2048, BOX_BYTES, 1024),
+                                   IDESC_ACC, acc_on);
+                            mma_ts(tmem_base + ACC2, tmem_base + T2 + a_off, smem_desc_sw128(aa + kk * 2048, BOX_BYTES, 1024),
+                                   IDESC_ACC, acc_on);
+                        } else {
+                            // acc1 (dQ') += dS K'
+                            mma_ts(tmem_base + ACC1, tmem_base + T1 + a_off, smem_desc_sw128(aa + kk * 2048, BOX_BYTES, 1024),
+                                   IDESC_ACC, acc_on);
+                        }
+                    }
                 }
+                if (!ok) break;
                 mma_commit(&bars[L::B_EMPTY + st]);
                 if (n == n_it - 1) mma_commit(&bars[L::B_DONE]);
             }
@@ -292,8 +308,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             else run(std::integral_constant<int, 0>{});
         }
     } else if (warp >= 8) {
-        // ------------------------------------------------------------ gradient warpgroup (one TMEM lane per thread)
-        const int tid = threadIdx.x - 256;
+        // ------------------------------------------------------------ gradient warpgroups (one TMEM lane per thread)
+        const int gtid = threadIdx.x - 256;          // 0..255 over both warpgroups
+        const int hf = gtid >> 7;                    // column half owned by this warpgroup
+        const int tid = gtid & 127;                  // == TMEM lane
         const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tb = tmem_base + lane_addr;
         const int xrow = x0 + tid;  // DKV: key row j; DQ: query row i
@@ -312,11 +330,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             float* sL2 = sStats + (n & 1) * 256;
             float* sDl = sL2 + 128;
             if (DKV) {
-                // per-column statistics of the streamed query tile
-                const int qi = a0 + tid;
-                const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + qi;
-                sL2[tid] = qi < p.S ? p.lse[r] * kLog2e : INFINITY;
-                sDl[tid] = qi < p.S ? p.delta[r] : 0.f;
+                // per-column statistics of the streamed query tile (written by the first warpgroup)
+                if (hf == 0) {
+                    const int qi = a0 + tid;
+                    const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + qi;
+                    sL2[tid] = qi < p.S ? p.lse[r] * kLog2e : INFINITY;
+                    sDl[tid] = qi < p.S ? p.delta[r] : 0.f;
+                }
                 my_slope2 = alibi ? p.slopes[ah] * kLog2e : 0.f;
             }
             const int i0 = DKV ? a0 : x0, j0 = DKV ? x0 : a0;
@@ -329,45 +349,57 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             }
             // ALiBi: slope2 * (j - i) = sb * (col + base), sb = +-slope2
             const float sb = DKV ? -my_slope2 : my_slope2;
-            const float bias_base = sb * static_cast<float>(DKV ? a0 - xrow : a0 - xrow);
+            const float bias_base = sb * static_cast<float>(a0 - xrow);
             ok = wg_all(mbar_wait(&bars[L::B_TFULL], n & 1, abort_flag, 29));  // also publishes the statistics
             if (!ok) break;
             tc_fence_after_sync();
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
+#pragma unroll
+            for (int qt = 0; qt < 2; ++qt) {
+                const int col0 = hf * 64 + qt * 32;
                 uint32_t s[32], dp[32], pk[16], dk[16];
-                tmem_ld32(tb + T1 + c * 32, s);
-                tmem_ld32(tb + T2 + c * 32, dp);
+                tmem_ld32(tb + T1 + col0, s);
+                tmem_ld32(tb + T2 + col0, dp);
                 tmem_wait_ld();
-                const float cbias = fmaf(sb, static_cast<float>(c * 32), bias_base);
+                const float cbias = fmaf(sb, static_cast<float>(col0), bias_base);
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float pv[2], dv[2];
+                for (int e = 0; e < 32; e += 4) {
+                    float l2v[4], dlv[4];
+                    if (DKV) {
+                        const float4 a4 = *reinterpret_cast<const float4*>(sL2 + col0 + e);
+                        const float4 b4 = *reinterpret_cast<const float4*>(sDl + col0 + e);
+                        l2v[0] = a4.x; l2v[1] = a4.y; l2v[2] = a4.z; l2v[3] = a4.w;
+                        dlv[0] = b4.x; dlv[1] = b4.y; dlv[2] = b4.z; dlv[3] = b4.w;
+                    } else {
 #pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int col = c * 32 + e + u;
-                        const float l2 = DKV ? sL2[col] : my_l2, dl = DKV ? sDl[col] : my_delta;
-                        float t = fmaf(__uint_as_float(s[e + u]), p.scale_log2, cbias - l2);
+                        for (int u = 0; u < 4; ++u) { l2v[u] = my_l2; dlv[u] = my_delta; }
+                    }
+                    float pv[4], dv[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        float t = fmaf(__uint_as_float(s[e + u]), p.scale_log2, cbias - l2v[u]);
                         if (alibi) t = fmaf(sb, static_cast<float>(e + u), t);
                         float pe = ex2(t);
-                        if (need_mask) pe = (static_cast<uint32_t>(col - mlo) < mn) ? pe : 0.f;
+                        if (need_mask) pe = (static_cast<uint32_t>(col0 + e + u - mlo) < mn) ? pe : 0.f;
                         pv[u] = pe;
-                        dv[u] = pe * (__uint_as_float(dp[e + u]) - dl);
+                        dv[u] = pe * (__uint_as_float(dp[e + u]) - dlv[u]);
                     }
                     pk[e >> 1] = pack_bf16x2(pv[0], pv[1]);
+                    pk[(e >> 1) + 1] = pack_bf16x2(pv[2], pv[3]);
                     dk[e >> 1] = pack_bf16x2(dv[0], dv[1]);
+                    dk[(e >> 1) + 1] = pack_bf16x2(dv[2], dv[3]);
                 }
+                // bf16 results go to the start of this warpgroup's own column half (already read)
                 if (DKV) {
-                    tmem_st16(tb + T1 + c * 16, pk);
-                    tmem_st16(tb + T2 + c * 16, dk);
+                    tmem_st16(tb + T1 + hf * 64 + qt * 16, pk);
+                    tmem_st16(tb + T2 + hf * 64 + qt * 16, dk);
                 } else {
-                    tmem_st16(tb + T1 + c * 16, dk);
+                    tmem_st16(tb + T1 + hf * 64 + qt * 16, dk);
                 }
             }
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars[L::B_PDS]);
+            if (lane == 0) mbar_arrive(&bars[L::B_PDS + hf]);
         }
         // epilogue: stage through shared memory (the stream stages are idle now), rotate back, store
         if (ok && n_it > 0) ok = wg_all(mbar_wait(&bars[L::B_DONE], 0, abort_flag, 30));
@@ -376,10 +408,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             float* stg = reinterpret_cast<float*>(sA);
             const size_t out_row0 = (static_cast<size_t>(b) * xh_count + xh) * p.S + x0;
             if (DKV) {
-                store_acc_rotated<D>(tb + ACC1, stg, tid, 1.f, 0, p.table, x0, p.S, p.out1, out_row0, p.out_f32);
-                store_acc_rotated<D>(tb + ACC2, stg, tid, p.scale, p.R, p.table, x0, p.S, p.out2, out_row0, p.out_f32);
+                store_acc_rotated<D>(tb + ACC1, stg, gtid, 1.f, 0, p.table, x0, p.S, p.out1, out_row0, p.out_f32);
+                store_acc_rotated<D>(tb + ACC2, stg, gtid, p.scale, p.R, p.table, x0, p.S, p.out2, out_row0, p.out_f32);
             } else {
-                store_acc_rotated<D>(tb + ACC1, stg, tid, p.scale, p.R, p.table, x0, p.S, p.out1, out_row0, p.out_f32);
+                store_acc_rotated<D>(tb + ACC1, stg, gtid, p.scale, p.R, p.table, x0, p.S, p.out1, out_row0, p.out_f32);
             }
         }
     }
