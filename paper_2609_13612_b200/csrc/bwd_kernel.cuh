@@ -275,7 +275,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             auto run = [&](auto cp_tag) {
                 constexpr int CP = decltype(cp_tag)::value;
                 constexpr int CPT = CP > 0 ? CP : 1;
-                float4 step[4];
+                RotStep step;
                 RotState<CPT> st;
                 if (CP > 0) {
                     rotate_load_step<CPT>(p.table, p.S, p.R, t, step);

@@ -138,17 +138,27 @@ __device__ __forceinline__ void rotate_tile_smem(uint8_t* tile, int row0, int S,
 // run of consecutive tiles needs no table read at all; callers re-read the table every
 // kRotResync tiles to keep the accumulated rounding of the recurrence far below bf16 resolution.
 constexpr int kRotResync = 16;
+// The arithmetic uses the packed fp32 instructions of sm_100 (two lanes per instruction): a bf16x2
+// word holds two adjacent columns, i.e. two frequencies, so cos and sin are kept as float2 pairs.
 template <int CP>
 struct RotState {
-    float4 t[4];     // {cos, sin} x 8 frequencies at the current row
+    float2 c[4], s[4];   // cos / sin of the 8 frequencies (4 column pairs) at the current row
+};
+struct RotStep {
+    float2 c[4], s[4], ns[4];   // cos, sin, -sin of the row-to-row step angle
 };
 
 template <int CP>
-__device__ __forceinline__ void rotate_load_step(const float2* table, int S, int R, int tid, float4 (&step)[4]) {
+__device__ __forceinline__ void rotate_load_step(const float2* table, int S, int R, int tid, RotStep& step) {
     const int cp = tid % CP;
     const float4* tb = reinterpret_cast<const float4*>(table + static_cast<size_t>(S) * (R >> 1) + cp * 8);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) step[u] = __ldg(tb + u);
+    for (int u = 0; u < 4; ++u) {
+        const float4 t = __ldg(tb + u);   // {cos0, sin0, cos1, sin1}
+        step.c[u] = make_float2(t.x, t.z);
+        step.s[u] = make_float2(t.y, t.w);
+        step.ns[u] = make_float2(-t.y, -t.w);
+    }
 }
 
 template <int CP>
@@ -158,17 +168,26 @@ __device__ __forceinline__ void rotate_prefetch(RotState<CP>& st, const float2* 
     const int prow = min(row0 + rg, S - 1);
     const float4* tb = reinterpret_cast<const float4*>(table + static_cast<size_t>(prow) * (R >> 1) + cp * 8);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) st.t[u] = __ldg(tb + u);
+    for (int u = 0; u < 4; ++u) {
+        const float4 t = __ldg(tb + u);
+        st.c[u] = make_float2(t.x, t.z);
+        st.s[u] = make_float2(t.y, t.w);
+    }
 }
 
-__device__ __forceinline__ void advance_cs(float& c, float& s, float C, float Sn) {
-    const float nc = fmaf(c, C, -s * Sn), ns = fmaf(s, C, c * Sn);
-    c = nc;
-    s = ns;
+// (a, b): bf16x2 words at column pairs (d, d+1) and (d + R/2, d + R/2 + 1); c, s: their cos / sin.
+__device__ __forceinline__ void rotate_word2(uint32_t& a, uint32_t& b, float2 c, float2 s) {
+    const float2 A = make_float2(bf16lo_to_f32(a), bf16hi_to_f32(a));
+    const float2 B = make_float2(bf16lo_to_f32(b), bf16hi_to_f32(b));
+    const float2 ns = make_float2(-s.x, -s.y);
+    const float2 na = __ffma2_rn(B, ns, __fmul2_rn(A, c));   // a cos - b sin
+    const float2 nb = __ffma2_rn(A, s, __fmul2_rn(B, c));    // b cos + a sin
+    a = pack_bf16x2(na.x, na.y);
+    b = pack_bf16x2(nb.x, nb.y);
 }
 
 template <int CP>
-__device__ __forceinline__ void rotate_tile_fast(uint8_t* tile, RotState<CP>& st, const float4 (&step)[4], int tid) {
+__device__ __forceinline__ void rotate_tile_fast(uint8_t* tile, RotState<CP>& st, const RotStep& step, int tid) {
     constexpr int RP = 128 / CP;
     constexpr int NB = CP < 4 ? CP : 4;  // rows in flight per thread: all loads of a batch are issued first
     const int rg = tid / CP, cp = tid % CP;
@@ -183,15 +202,17 @@ __device__ __forceinline__ void rotate_tile_fast(uint8_t* tile, RotState<CP>& st
         }
 #pragma unroll
         for (int u = 0; u < NB; ++u) {
-            rotate_word(lo[u].x, hi[u].x, st.t[0].x, st.t[0].y, st.t[0].z, st.t[0].w);
-            rotate_word(lo[u].y, hi[u].y, st.t[1].x, st.t[1].y, st.t[1].z, st.t[1].w);
-            rotate_word(lo[u].z, hi[u].z, st.t[2].x, st.t[2].y, st.t[2].z, st.t[2].w);
-            rotate_word(lo[u].w, hi[u].w, st.t[3].x, st.t[3].y, st.t[3].z, st.t[3].w);
+            rotate_word2(lo[u].x, hi[u].x, st.c[0], st.s[0]);
+            rotate_word2(lo[u].y, hi[u].y, st.c[1], st.s[1]);
+            rotate_word2(lo[u].z, hi[u].z, st.c[2], st.s[2]);
+            rotate_word2(lo[u].w, hi[u].w, st.c[3], st.s[3]);
             // after the last row the state sits RP * CP = 128 rows further: the same row of the next tile
 #pragma unroll
             for (int w = 0; w < 4; ++w) {
-                advance_cs(st.t[w].x, st.t[w].y, step[w].x, step[w].y);
-                advance_cs(st.t[w].z, st.t[w].w, step[w].z, step[w].w);
+                const float2 nc = __ffma2_rn(st.s[w], step.ns[w], __fmul2_rn(st.c[w], step.c[w]));
+                const float2 nsn = __ffma2_rn(st.c[w], step.s[w], __fmul2_rn(st.s[w], step.c[w]));
+                st.c[w] = nc;
+                st.s[w] = nsn;
             }
         }
 #pragma unroll

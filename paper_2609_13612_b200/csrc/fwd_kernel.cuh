@@ -90,18 +90,20 @@ __device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, fl
         m_run = mx;
     }
     const float sub = bias0 - ((m_run == -INFINITY) ? 0.f : m_run);
-    float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+    const float2 sc2 = make_float2(scale_log2, scale_log2), sub2 = make_float2(sub, sub);
+    float2 ps2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
     uint32_t pk[BN / 2];
 #pragma unroll
     for (int e = 0; e < BN; e += 2) {
-        const float p0 = ex2(fmaf(__uint_as_float(v[e]), scale_log2, sub));
-        const float p1 = ex2(fmaf(__uint_as_float(v[e + 1]), scale_log2, sub));
-        ps4[(e >> 1) & 3] += p0 + p1;
-        pk[e >> 1] = pack_bf16x2(p0, p1);
+        // packed fp32: one instruction scales and shifts two scores, one adds two probabilities
+        const float2 t = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), sc2, sub2);
+        const float2 pe = make_float2(ex2(t.x), ex2(t.y));
+        ps2[(e >> 1) & 1] = __fadd2_rn(ps2[(e >> 1) & 1], pe);
+        pk[e >> 1] = pack_bf16x2(pe.x, pe.y);
     }
     tmem_st32(tS, pk);
     tmem_st32(tS + 32, pk + 32);
-    l_run = l_run * alpha + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
+    l_run = l_run * alpha + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
     if (n > 0 && __any_sync(0xffffffffu, upd)) {
 #pragma unroll 1
         for (int c = 0; c < D / 32; ++c) {
@@ -299,7 +301,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             auto run = [&](auto cp_tag) {
                 constexpr int CP = decltype(cp_tag)::value;  // 0: generic path (table read per row)
                 bool ok = true;
-                float4 step[4];
+                RotStep step;
                 RotState<(CP > 0 ? CP : 1)> st;
                 if (CP > 0) rotate_load_step<(CP > 0 ? CP : 1)>(p.table, p.S, p.R, t, step);
 #pragma unroll
