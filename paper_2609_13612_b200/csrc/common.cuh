@@ -189,7 +189,7 @@ __device__ __forceinline__ void rotate_word2(uint32_t& a, uint32_t& b, float2 c,
 template <int CP>
 __device__ __forceinline__ void rotate_tile_fast(uint8_t* tile, RotState<CP>& st, const RotStep& step, int tid) {
     constexpr int RP = 128 / CP;
-    constexpr int NB = CP < 4 ? CP : 4;  // rows in flight per thread: all loads of a batch are issued first
+    constexpr int NB = CP < 2 ? CP : 2;  // rows in flight per thread (more would spill at this role's register budget)
     const int rg = tid / CP, cp = tid % CP;
 #pragma unroll
     for (int k0 = 0; k0 < CP; k0 += NB) {

@@ -243,20 +243,20 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
             };
 
-            // prologue: S of the first key tile
-#pragma unroll
-            for (int q = 0; q < NQ; ++q)
-                if (ok && jhi[q] >= jlo[q]) ok = mbar_wait(&bars[B_QREADY + q], 0, abort_flag, 3);
-            AF_STAMP(0, 63, 2);  // Q ready
+            // prologue: S of the first key tile, each query tile as soon as it is ready (the rotation
+            // warpgroup delivers Q tile 0, K tile 0, Q tile 1 in that order)
             if (ok) ok = mbar_wait(&bars[B_KREADY + 0], 0, abort_flag, 4);
             AF_STAMP(0, 63, 3);  // first K ready
-            if (ok) {
-                tc_fence_after_sync();
 #pragma unroll
-                for (int q = 0; q < NQ; ++q)
-                    if (jlo_c >= jlo[q] && jlo_c <= jhi[q]) issue_S(q, 0);
-                mma_commit(&bars[L::B_KEMPTY + 0]);
+            for (int q = 0; q < NQ; ++q) {
+                if (ok && jhi[q] >= jlo[q]) {
+                    ok = mbar_wait(&bars[B_QREADY + q], 0, abort_flag, 3);
+                    tc_fence_after_sync();
+                    if (ok && jlo_c >= jlo[q] && jlo_c <= jhi[q]) issue_S(q, 0);
+                }
             }
+            AF_STAMP(0, 63, 2);  // Q ready
+            if (ok) mma_commit(&bars[L::B_KEMPTY + 0]);
             for (int it = 0; ok && it < n_it; ++it) {
                 const int j = jlo_c + it, vs = it % VS, ks1 = (it + 1) % KS;
                 const bool next = it + 1 < n_it;
@@ -304,22 +304,24 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 RotStep step;
                 RotState<(CP > 0 ? CP : 1)> st;
                 if (CP > 0) rotate_load_step<(CP > 0 ? CP : 1)>(p.table, p.S, p.R, t, step);
-#pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    if (!ok || jhi[q] < jlo[q]) continue;
+                auto rotate_q = [&](int q) {
+                    if (!ok || jhi[q] < jlo[q]) return;
                     if (CP > 0) rotate_prefetch(st, p.table, i0[q], p.S, p.R, t);
                     ok = mbar_wait_warp(&bars[L::B_QFULL + q], 0, abort_flag, 8);
-                    if (!ok) break;
+                    if (!ok) return;
                     if (CP > 0) rotate_tile_fast(sQ + q * TILE, st, step, t);
                     else rotate_tile_smem(sQ + q * TILE, i0[q], p.S, p.R, p.table, t, 128);
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars[L::B_QROT + q]);
-                }
+                };
+                // order: Q tile 0, K tile 0, remaining Q tiles, K tiles 1.. - the first S MMA needs only the first two
+                rotate_q(0);
                 // K tiles are consecutive: the recurrence carries the cos/sin state from tile to tile
                 for (int it = 0; ok && it < n_it; ++it) {
                     const int ks = it % KS;
-                    if (CP > 0 && (it % kRotResync) == 0) rotate_prefetch(st, p.table, (jlo_c + it) * BN, p.S, p.R, t);
+                    if (CP > 0 && ((it % kRotResync) == 0 || it == 1))   // it == 1: the Q tiles in between used the state
+                        rotate_prefetch(st, p.table, (jlo_c + it) * BN, p.S, p.R, t);
                     AF_STAMP(1, it, 0);
                     ok = mbar_wait_warp(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
                     AF_STAMP(1, it, 1);
@@ -330,6 +332,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars[L::B_KROT + ks]);
                     AF_STAMP(1, it, 2);
+                    if (it == 0) {
+#pragma unroll
+                        for (int q = 1; q < NQ; ++q) rotate_q(q);
+                    }
                 }
             };
             if (p.R == 128) run(std::integral_constant<int, 8>{});
