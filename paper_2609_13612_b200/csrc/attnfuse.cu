@@ -104,8 +104,11 @@ af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const
             return AF_ERR_CUDA;
         configured = true;
     }
-    p.n_row_blocks = (p.S + BM * NQ - 1) / (BM * NQ);
-    dim3 grid(p.B * p.Hq, p.n_row_blocks, 1);
+    // an even GQA group lets the two query tiles of a CTA be two heads of one kv head (same key range)
+    p.pair_heads = (NQ == 2 && (p.group % 2) == 0 && env_int("AF_FWD_PAIR", 1)) ? 1 : 0;
+    const int rows_per_cta = p.pair_heads ? BM : BM * NQ;
+    p.n_row_blocks = (p.S + rows_per_cta - 1) / rows_per_cta;
+    dim3 grid(p.pair_heads ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
     kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
@@ -271,6 +274,7 @@ af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, cons
     p.table = static_cast<const float2*>(rope_table);
     p.o = o; p.o_f32 = (o_dtype == AF_F32); p.lse = lse;
     p.n_row_blocks = 0;
+    p.pair_heads = 0;
 #ifdef AF_TRACE
     p.trace = reinterpret_cast<long long*>(getenv("AF_TRACE_PTR") ? strtoull(getenv("AF_TRACE_PTR"), nullptr, 0) : 0ull);
 #endif

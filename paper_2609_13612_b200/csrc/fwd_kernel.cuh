@@ -21,7 +21,8 @@ struct FwdParams {
     void* o;
     int o_f32;
     float* lse;         // nullable
-    int n_row_blocks;   // ceil(S / (128 * NQ))
+    int n_row_blocks;   // ceil(S / (128 * NQ)), or ceil(S / 128) with pair_heads
+    int pair_heads;     // NQ = 2 only: the two query tiles are the same 128 rows of two heads of one kv group
 #ifdef AF_TRACE
     long long* trace;
 #endif
@@ -139,7 +140,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_MISC + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bh = blockIdx.x, b = bh / p.Hq, h = bh - b * p.Hq, hk = h / p.group;
+    // blockIdx.x: a head, or with pair_heads (even GQA group) a pair of adjacent heads that share a kv head.
+    // Pairing heads gives both query tiles the same key range, so the two softmax warpgroups stay in
+    // step down to the last tile; without it the tiles are rows [256 rb, +128) and [256 rb + 128, +128).
+    const int upb = p.pair_heads ? p.Hq / 2 : p.Hq;   // units per batch
+    const int b = static_cast<int>(blockIdx.x) / upb, u = static_cast<int>(blockIdx.x) - b * upb;
+    int hq[NQ];
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) hq[q] = p.pair_heads ? 2 * u + q : u;
+    const int hk = hq[0] / p.group;
     const int rb = p.n_row_blocks - 1 - static_cast<int>(blockIdx.y);  // heaviest (last) row blocks first
     const MaskSpec ms{p.S, p.causal, p.window};
 
@@ -147,7 +156,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     int jlo_c = 0x7fffffff, jhi_c = -1;
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
-        i0[q] = (rb * NQ + q) * BM;
+        i0[q] = p.pair_heads ? rb * BM : (rb * NQ + q) * BM;
         if (i0[q] < p.S) {
             tile_range(ms, i0[q], jlo[q], jhi[q]);
             jlo_c = min(jlo_c, jlo[q]);
@@ -196,7 +205,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 mbar_arrive_expect_tx(&bars[L::B_QFULL + q], TILE);
 #pragma unroll
                 for (int bx = 0; bx < NBOX; ++bx)
-                    tma_load_4d(sQ + q * TILE + bx * BOX_BYTES, &tm_q, &bars[L::B_QFULL + q], bx * BOX_COLS, i0[q], h, b);
+                    tma_load_4d(sQ + q * TILE + bx * BOX_BYTES, &tm_q, &bars[L::B_QFULL + q], bx * BOX_COLS, i0[q], hq[q], b);
             }
             for (int it = 0; it < n_it; ++it) {
                 const int j0 = (jlo_c + it) * BN;
@@ -353,7 +362,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t tS = tmem_base + lane_addr + q * BN;      // S (fp32) and, over it, P (bf16x2)
         const uint32_t tO = tmem_base + lane_addr + NQ * BN + q * D;
         const int i = i0[q] + row;
-        const float slope2 = p.slopes ? p.slopes[h] * 1.4426950408889634f : 0.f;
+        const int bh = b * p.Hq + hq[q];
+        const float slope2 = p.slopes ? p.slopes[hq[q]] * 1.4426950408889634f : 0.f;
         const bool alibi = p.slopes != nullptr;
         const float kb = slope2 / p.scale_log2;
         float m_run = -INFINITY, l_run = 0.f;
