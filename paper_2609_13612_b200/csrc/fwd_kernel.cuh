@@ -74,15 +74,19 @@ __device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, fl
     tmem_wait_ld();
     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-    for (int e = 0; e < BN; ++e) {
-        float sv = __uint_as_float(v[e]);
-        if (ALIBI) sv = fmaf(kb, static_cast<float>(e), sv);
-        if (MASKED) sv = (static_cast<uint32_t>(e - mlo) < mn) ? sv : -INFINITY;
-        if (ALIBI || MASKED) v[e] = __float_as_uint(sv);
-        mx4[e & 3] = fmaxf(mx4[e & 3], sv);
+    for (int e = 0; e < BN; e += 2) {
+        float sv[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            sv[u] = __uint_as_float(v[e + u]);
+            if (ALIBI) sv[u] = fmaf(kb, static_cast<float>(e + u), sv[u]);
+            if (MASKED) sv[u] = (static_cast<uint32_t>(e + u - mlo) < mn) ? sv[u] : -INFINITY;
+            if (ALIBI || MASKED) v[e + u] = __float_as_uint(sv[u]);
+        }
+        mx4[(e >> 1) & 3] = fmax3(mx4[(e >> 1) & 3], sv[0], sv[1]);   // two scores per instruction
     }
     // scale > 0, so the max commutes with it
-    const float mx = fmaf(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])), scale_log2, bias0);
+    const float mx = fmaf(fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]), scale_log2, bias0);
     // lazy rescale: keep the old reference max unless it grew by more than the threshold
     const bool upd = mx > m_run + kRescaleThreshold;
     float alpha = 1.f;
@@ -252,8 +256,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
             };
 
-            // prologue: S of the first key tile, each query tile as soon as it is ready (the rotation
-            // warpgroup delivers Q tile 0, K tile 0, Q tile 1 in that order)
+            // prologue: S of the first key tile, each query tile as soon as it is ready (the softmax
+            // warpgroups rotate their Q tiles while the rotation warpgroup rotates K tile 0)
             if (ok) ok = mbar_wait(&bars[B_KREADY + 0], 0, abort_flag, 4);
             AF_STAMP(0, 63, 3);  // first K ready
 #pragma unroll
@@ -313,24 +317,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 RotStep step;
                 RotState<(CP > 0 ? CP : 1)> st;
                 if (CP > 0) rotate_load_step<(CP > 0 ? CP : 1)>(p.table, p.S, p.R, t, step);
-                auto rotate_q = [&](int q) {
-                    if (!ok || jhi[q] < jlo[q]) return;
-                    if (CP > 0) rotate_prefetch(st, p.table, i0[q], p.S, p.R, t);
-                    ok = mbar_wait_warp(&bars[L::B_QFULL + q], 0, abort_flag, 8);
-                    if (!ok) return;
-                    if (CP > 0) rotate_tile_fast(sQ + q * TILE, st, step, t);
-                    else rotate_tile_smem(sQ + q * TILE, i0[q], p.S, p.R, p.table, t, 128);
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars[L::B_QROT + q]);
-                };
-                // order: Q tile 0, K tile 0, remaining Q tiles, K tiles 1.. - the first S MMA needs only the first two
-                rotate_q(0);
+                // (each Q tile is rotated by its own softmax warpgroup, which has nothing else to do yet)
                 // K tiles are consecutive: the recurrence carries the cos/sin state from tile to tile
                 for (int it = 0; ok && it < n_it; ++it) {
                     const int ks = it % KS;
-                    if (CP > 0 && ((it % kRotResync) == 0 || it == 1))   // it == 1: the Q tiles in between used the state
-                        rotate_prefetch(st, p.table, (jlo_c + it) * BN, p.S, p.R, t);
+                    if (CP > 0 && (it % kRotResync) == 0) rotate_prefetch(st, p.table, (jlo_c + it) * BN, p.S, p.R, t);
                     AF_STAMP(1, it, 0);
                     ok = mbar_wait_warp(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
                     AF_STAMP(1, it, 1);
@@ -341,10 +332,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars[L::B_KROT + ks]);
                     AF_STAMP(1, it, 2);
-                    if (it == 0) {
-#pragma unroll
-                        for (int q = 1; q < NQ; ++q) rotate_q(q);
-                    }
                 }
             };
             if (p.R == 128) run(std::integral_constant<int, 8>{});
@@ -369,6 +356,32 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         float m_run = -INFINITY, l_run = 0.f;
         bool ok = true;
         int n = 0;
+        if (ROPE && jhi[q] >= jlo[q]) {
+            // Section 4.1: the query tile is rotated once, before the key loop - by this warpgroup, which
+            // would otherwise idle until the first scores arrive (the rotation warpgroup starts on K at once)
+            auto rot_q = [&](auto cp_tag) {
+                constexpr int CP = decltype(cp_tag)::value;
+                constexpr int CPT = CP > 0 ? CP : 1;
+                RotStep step;
+                RotState<CPT> st;
+                if (CP > 0) {
+                    rotate_load_step<CPT>(p.table, p.S, p.R, row, step);
+                    rotate_prefetch(st, p.table, i0[q], p.S, p.R, row);
+                }
+                ok = mbar_wait_warp(&bars[L::B_QFULL + q], 0, abort_flag, 8);
+                if (!ok) return;
+                if (CP > 0) rotate_tile_fast(sQ + q * TILE, st, step, row);
+                else rotate_tile_smem(sQ + q * TILE, i0[q], p.S, p.R, p.table, row, 128);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[L::B_QROT + q]);
+            };
+            if (p.R == 128) rot_q(std::integral_constant<int, 8>{});
+            else if (p.R == 64) rot_q(std::integral_constant<int, 4>{});
+            else if (p.R == 32) rot_q(std::integral_constant<int, 2>{});
+            else if (p.R == 16) rot_q(std::integral_constant<int, 1>{});
+            else rot_q(std::integral_constant<int, 0>{});
+        }
         for (int j = jlo[q]; ok && j <= jhi[q]; ++j, ++n) {
             const int j0 = j * BN;
             AF_STAMP(2 + q, n, 0);
