@@ -109,7 +109,10 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
  * on chip and gradients w.r.t. rotated rows are rotated back in the epilogues.
  * o, d_o: [B,Hq,S,D] bf16 contiguous; lse from the forward.
  * dq [B,Hq,S,D] (dq_dtype), dk, dv [B,Hkv,S,D] (dkv_dtype), contiguous; dk/dv sum over the group.
- * workspace: at least attnfuse_bwd_workspace_bytes(shape) bytes (holds delta). */
+ * workspace: attnfuse_bwd_workspace_bytes(shape) bytes hold delta (4 bytes per query row, rounded up to
+ * 256) followed by a cache of the rotated K (B*Hkv*S*D bf16) that the dK/dV kernel fills and the dQ
+ * kernel reads, so K is rotated once per key tile instead of once per (query tile, key tile).  A smaller
+ * workspace is accepted down to the delta part alone; the dQ kernel then rotates K on chip itself. */
 size_t    attnfuse_bwd_workspace_bytes(const af_shape* shape);
 af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, const void* v,
                        const void* o, const float* lse, const void* d_o,

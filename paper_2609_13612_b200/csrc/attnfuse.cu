@@ -125,25 +125,27 @@ af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
                    : launch_fwd_variant<D, 2, false, 2, 2>(tq, tk, tv, p, stream);
 }
 
-template <int D, bool DKV, bool ROPE>
+template <int D, bool DKV, bool ROT_X, bool ROT_A>
 af_status launch_bwd_variant(const CUtensorMap& tx, const CUtensorMap& ty, const CUtensorMap& ta, const CUtensorMap& tb,
-                             const BwdParams& p, dim3 grid, cudaStream_t stream) {
+                             const CUtensorMap& ts, const BwdParams& p, dim3 grid, cudaStream_t stream) {
     using L = BwdSmem<D>;
-    auto kern = attn_bwd_kernel<D, DKV, ROPE>;
+    auto kern = attn_bwd_kernel<D, DKV, ROT_X, ROT_A>;
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
             return AF_ERR_CUDA;
         configured = true;
     }
-    kern<<<grid, 512, L::BYTES, stream>>>(tx, ty, ta, tb, p);
+    kern<<<grid, 512, L::BYTES, stream>>>(tx, ty, ta, tb, ts, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
+// delta, then the dK/dV kernel, then the dQ kernel.  tkp: tensor map over the rotated-K cache in the
+// workspace, or nullptr when the workspace has no room for it (then the dQ kernel rotates K itself).
 template <int D>
 af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                     const CUtensorMap& tdo, const void* o, const void* d_o, BwdParams p, void* dq, int dq_f32,
-                     void* dk, void* dv, int dkv_f32, float* delta, cudaStream_t stream) {
+                     const CUtensorMap& tdo, const CUtensorMap* tkp, const void* o, const void* d_o, BwdParams p,
+                     void* dq, int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, cudaStream_t stream) {
     const long long rows = static_cast<long long>(sh->B) * sh->Hq * sh->S;
     const long long threads = rows * (D / 8);
     bwd_delta_kernel<D><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
@@ -152,15 +154,26 @@ af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMa
     p.delta = delta;
     const unsigned tiles = static_cast<unsigned>((sh->S + 127) / 128);
     af_status st;
-    p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32;
+    const int only = env_int("AF_BWD_ONLY", 0);   // tuning aid: 1 = dK/dV kernel only, 2 = dQ kernel only
+    const bool cache = p.R > 0 && tkp != nullptr && only != 2;
+    p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32; p.store_x = cache ? 1 : 0;
     dim3 gkv(sh->B * sh->Hkv, tiles, 1);
-    st = p.R > 0 ? launch_bwd_variant<D, true, true>(tk, tv, tq, tdo, p, gkv, stream)
-                 : launch_bwd_variant<D, true, false>(tk, tv, tq, tdo, p, gkv, stream);
-    if (st != AF_OK) return st;
-    p.out1 = dq; p.out2 = nullptr; p.out_f32 = dq_f32;
+    st = only == 2 ? AF_OK
+         : p.R > 0 ? launch_bwd_variant<D, true, true, true>(tk, tv, tq, tdo, cache ? *tkp : tk, p, gkv, stream)
+                   : launch_bwd_variant<D, true, false, false>(tk, tv, tq, tdo, tk, p, gkv, stream);
+    if (st != AF_OK || only == 1) return st;
+    p.out1 = dq; p.out2 = nullptr; p.out_f32 = dq_f32; p.store_x = 0;
     dim3 gq(sh->B * sh->Hq, tiles, 1);
-    return p.R > 0 ? launch_bwd_variant<D, false, true>(tq, tdo, tk, tv, p, gq, stream)
-                   : launch_bwd_variant<D, false, false>(tq, tdo, tk, tv, p, gq, stream);
+    if (p.R == 0) return launch_bwd_variant<D, false, false, false>(tq, tdo, tk, tv, tk, p, gq, stream);
+    return cache ? launch_bwd_variant<D, false, true, false>(tq, tdo, *tkp, tv, tk, p, gq, stream)
+                 : launch_bwd_variant<D, false, true, true>(tq, tdo, tk, tv, tk, p, gq, stream);
+}
+
+size_t bwd_delta_bytes(const af_shape* sh) {
+    return (static_cast<size_t>(sh->B) * sh->Hq * sh->S * sizeof(float) + 255) / 256 * 256;
+}
+size_t bwd_kcache_bytes(const af_shape* sh) {
+    return static_cast<size_t>(sh->B) * sh->Hkv * sh->S * sh->D * 2;
 }
 
 }  // namespace
@@ -319,7 +332,7 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
 
 size_t attnfuse_bwd_workspace_bytes(const af_shape* shape) {
     if (!shape) return 0;
-    return static_cast<size_t>(shape->B) * shape->Hq * shape->S * sizeof(float) + 256;
+    return bwd_delta_bytes(shape) + bwd_kcache_bytes(shape);   // delta + rotated-K cache
 }
 
 af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,
@@ -332,7 +345,7 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
     if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv) return AF_ERR_NULL;
     if ((dq_dtype != AF_BF16 && dq_dtype != AF_F32) || (dkv_dtype != AF_BF16 && dkv_dtype != AF_F32))
         return AF_ERR_DTYPE;
-    if (!workspace || workspace_bytes < attnfuse_bwd_workspace_bytes(shape)) return AF_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < bwd_delta_bytes(shape)) return AF_ERR_WORKSPACE;   // the cache is optional
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv) || !aligned16(workspace) || !aligned16(lse))
         return AF_ERR_ALIGN;
@@ -357,14 +370,23 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
     p.slopes = mask->alibi_slopes;
     p.table = static_cast<const float2*>(rope_table);
     p.lse = lse;
-    p.delta = nullptr; p.out1 = nullptr; p.out2 = nullptr; p.out_f32 = 0;
+    p.delta = nullptr; p.out1 = nullptr; p.out2 = nullptr; p.out_f32 = 0; p.store_x = 0;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     float* delta = static_cast<float*>(workspace);
+    // rotated-K cache: used when there is a rotation and the workspace has room behind delta
+    CUtensorMap tkp;
+    const bool have_cache = p.R > 0 && workspace_bytes >= bwd_delta_bytes(shape) + bwd_kcache_bytes(shape);
+    if (have_cache) {
+        af_strides stk;
+        resolve_strides(nullptr, shape->Hkv, shape->S, shape->D, &stk);
+        void* kc = static_cast<uint8_t*>(workspace) + bwd_delta_bytes(shape);
+        if ((st = make_tmap(&tkp, kc, shape->B, shape->Hkv, shape->S, shape->D, stk, 128)) != AF_OK) return st;
+    }
     return shape->D == 128
-               ? launch_bwd<128>(shape, tq, tk, tv, tdo, o, d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32,
-                                 delta, stream)
-               : launch_bwd<64>(shape, tq, tk, tv, tdo, o, d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32,
-                                delta, stream);
+               ? launch_bwd<128>(shape, tq, tk, tv, tdo, have_cache ? &tkp : nullptr, o, d_o, p, dq, dq_dtype == AF_F32, dk,
+                                 dv, dkv_dtype == AF_F32, delta, stream)
+               : launch_bwd<64>(shape, tq, tk, tv, tdo, have_cache ? &tkp : nullptr, o, d_o, p, dq, dq_dtype == AF_F32, dk,
+                                dv, dkv_dtype == AF_F32, delta, stream);
 }
 
 }  // extern "C"
@@ -374,7 +396,7 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
 // a fixed device array of this library.  In host code the array's name is only a stand-in for the
 // symbol, not a device address, so its address is looked up once per device and passed on as a
 // pointer.  Every call on a device shares the array; see the header for the rules.
-static __device__ __align__(256) unsigned char g_bwd_static_scratch[AF_BWD_STATIC_MAX_ROWS * sizeof(float) + 256];
+static __device__ __align__(256) unsigned char g_bwd_static_scratch[AF_BWD_STATIC_MAX_ROWS * sizeof(float) + 256];   // delta only
 
 namespace {
 constexpr int kMaxDevices = 64;

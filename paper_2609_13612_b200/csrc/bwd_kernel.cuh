@@ -33,6 +33,7 @@ struct BwdParams {
     void* out1;           // DKV: dV   DQ: dQ
     void* out2;           // DKV: dK   DQ: unused
     int out_f32;
+    int store_x;          // DKV role: write the rotated X tile through tm_s
 };
 
 // delta[row] = <dO[row], O[row]>; one 16-byte chunk per thread, D/8 threads per row.
@@ -113,29 +114,49 @@ __device__ __forceinline__ void store_acc_rotated(uint32_t t_acc, float* stg, in
     const int d = gtid % D, rsub = gtid / D;
     const int half = R >> 1;
     const int fi = d < half ? d : d - half;
+    // This thread writes column d of rows rsub, rsub + RPP, ...: one frequency, positions RPP apart.  Its
+    // cos/sin come from the table once (first row, and the next one to get the step angle as a
+    // difference of angles) and then walk by the angle-addition recurrence: no table read in the loop.
+    float c = 1.f, sn = 0.f, cst = 1.f, sst = 0.f;
+    if (d < R) {
+        const int r0 = min(row0 + rsub, S - 1), r1 = min(row0 + rsub + RPP, S - 1);
+        const float2 t0 = __ldg(table + static_cast<size_t>(r0) * half + fi);
+        const float2 t1 = __ldg(table + static_cast<size_t>(r1) * half + fi);
+        c = t0.x;
+        sn = t0.y;
+        cst = fmaf(t1.x, t0.x, t1.y * t0.y);    // cos(a1 - a0)
+        sst = fmaf(t1.y, t0.x, -t1.x * t0.y);   // sin(a1 - a0)
+    }
+    const bool upper = d >= half;
+    const int partner = d < half ? d + half : d - half;
 #pragma unroll 4
     for (int r = rsub; r < 128; r += RPP) {
-        const int row = row0 + r;
-        if (row < S) {
+        if (row0 + r < S) {
             float y = stg[r * STRIDE + d];
             if (d < R) {
-                const float2 cs = __ldg(table + static_cast<size_t>(row) * half + fi);
-                const float other = stg[r * STRIDE + (d < half ? d + half : d - half)];
-                y = d < half ? fmaf(y, cs.x, other * cs.y) : fmaf(y, cs.x, -other * cs.y);
+                const float other = stg[r * STRIDE + partner];
+                y = upper ? fmaf(y, c, -other * sn) : fmaf(y, c, other * sn);   // transpose rotation
             }
             const size_t o = (out_row0 + r) * D + d;
             if (out_f32) static_cast<float*>(out)[o] = y;
             else static_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(y);
         }
+        const float nc = fmaf(c, cst, -sn * sst), ns = fmaf(sn, cst, c * sst);
+        c = nc;
+        sn = ns;
     }
     wg_sync();
 }
 
-template <int D, bool DKV, bool ROPE>
+// ROT_X / ROT_A: rotate the stationary tile X / every streamed tile A on chip.  The dK/dV role rotates
+// both (K' once, every Q' tile) and, when the caller's workspace has room (p.store_x), writes its rotated
+// K' tile to that workspace through tm_s; the dQ role then streams those rows and rotates only its own
+// Q' tile, instead of rotating every K tile again for every query tile.
+template <int D, bool DKV, bool ROT_X, bool ROT_A>
 __global__ void __launch_bounds__(512, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_y,
                 const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                const BwdParams p) {
+                const __grid_constant__ CUtensorMap tm_s, const BwdParams p) {
     using L = BwdSmem<D>;
     constexpr int TILE = L::TILE, NST = L::NST;
     constexpr int NBOX = D / BOX_COLS;
@@ -171,8 +192,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::N_BARS; ++i) {
             uint32_t cnt = 1;
-            if (i == L::B_XROT || (i >= L::B_AROT && i < L::B_AROT + NST) || i == L::B_PDS || i == L::B_PDS + 1)
-                cnt = 4;  // per-warp arrives
+            if ((i >= L::B_AROT && i < L::B_AROT + NST) || i == L::B_PDS || i == L::B_PDS + 1) cnt = 4;  // per-warp arrives
+            if (i == L::B_XROT) cnt = 8;  // both gradient warpgroups
             mbar_init(&bars[i], cnt);
         }
         *abort_flag = 0;
@@ -213,9 +234,15 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr int B_XREADY = ROPE ? L::B_XROT : L::B_XFULL;
-            constexpr int B_AREADY = ROPE ? L::B_AROT : L::B_AFULL;
+            constexpr int B_XREADY = ROT_X ? L::B_XROT : L::B_XFULL;
+            constexpr int B_AREADY = ROT_A ? L::B_AROT : L::B_AFULL;
             bool ok = mbar_wait(&bars[B_XREADY], 0, abort_flag, 22);
+            if (ok && DKV && ROT_X && p.store_x) {
+                // publish the rotated K' tile (rows past S are clipped by the tensor map)
+#pragma unroll
+                for (int bx = 0; bx < NBOX; ++bx) tma_store_4d(&tm_s, sX + bx * BOX_BYTES, bx * BOX_COLS, x0, xh, b);
+                tma_store_commit();
+            }
             if (ok) ok = mbar_wait(&bars[L::B_YFULL], 0, abort_flag, 23);
             const uint32_t xa = smem_u32(sX), ya = smem_u32(sY);
             for (int n = 0; ok && n < n_it; ++n) {
@@ -267,27 +294,20 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 mma_commit(&bars[L::B_EMPTY + st]);
                 if (n == n_it - 1) mma_commit(&bars[L::B_DONE]);
             }
+            if (DKV && ROT_X && p.store_x) tma_store_wait_all();   // the tile must stay in place until it has been read
         }
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------ rotation warpgroup: X once, every A tile
-        if (ROPE) {
+        if (ROT_A) {
             const int t = threadIdx.x - 128;
             auto run = [&](auto cp_tag) {
                 constexpr int CP = decltype(cp_tag)::value;
                 constexpr int CPT = CP > 0 ? CP : 1;
                 RotStep step;
                 RotState<CPT> st;
-                if (CP > 0) {
-                    rotate_load_step<CPT>(p.table, p.S, p.R, t, step);
-                    rotate_prefetch(st, p.table, x0, p.S, p.R, t);
-                }
-                bool ok = mbar_wait_warp(&bars[L::B_XFULL], 0, abort_flag, 27);
-                if (!ok) return;
-                if (CP > 0) rotate_tile_fast(sX, st, step, t);
-                else rotate_tile_smem(sX, x0, p.S, p.R, p.table, t, 128);
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars[L::B_XROT]);
+                if (CP > 0) rotate_load_step<CPT>(p.table, p.S, p.R, t, step);
+                // (the stationary tile X is rotated by the two gradient warpgroups, idle at that point)
+                if (!ROT_A) return;
                 // streamed tiles are consecutive within a head: the recurrence carries the state along
                 for (int n = 0; n < n_it; ++n) {
                     const int sg = n % NST, a0 = stream_row0(n);
@@ -325,6 +345,30 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             my_slope2 = alibi ? p.slopes[xh] * kLog2e : 0.f;
         }
         bool ok = true;
+        if (ROT_X) {
+            // the stationary tile is rotated once, by these two warpgroups (half of the rows each): they
+            // have nothing else to do until the first scores arrive
+            auto rot_x = [&](auto cp_tag) {
+                constexpr int CP = decltype(cp_tag)::value;
+                ok = wg_all(mbar_wait(&bars[L::B_XFULL], 0, abort_flag, 27));
+                if (!ok) return;
+                if constexpr (CP > 0) {
+                    RotStep step;
+                    rotate_load_step<CP>(p.table, p.S, p.R, tid, step);
+                    rotate_tile_share<CP, 2>(sX, p.table, x0, p.S, p.R, step, tid, hf);
+                } else {
+                    rotate_tile_smem(sX, x0, p.S, p.R, p.table, gtid, 256);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[L::B_XROT]);
+            };
+            if (p.R == 128) rot_x(std::integral_constant<int, 8>{});
+            else if (p.R == 64) rot_x(std::integral_constant<int, 4>{});
+            else if (p.R == 32) rot_x(std::integral_constant<int, 2>{});
+            else if (p.R == 16) rot_x(std::integral_constant<int, 1>{});
+            else rot_x(std::integral_constant<int, 0>{});
+        }
         for (int n = 0; ok && n < n_it; ++n) {
             const int ah = stream_head(n), a0 = stream_row0(n);
             float* sL2 = sStats + (n & 1) * 256;

@@ -224,6 +224,52 @@ __device__ __forceinline__ void rotate_tile_fast(uint8_t* tile, RotState<CP>& st
     }
 }
 
+// The same walk restricted to a share of the rows: with PARTS warpgroups working on one tile, part p
+// takes the rows rg + RP * k for k in [p * CP / PARTS, (p + 1) * CP / PARTS).  Used where otherwise idle
+// warpgroups rotate a stationary tile together.  (CP < PARTS: part 0 does everything.)
+template <int CP, int PARTS>
+__device__ __forceinline__ void rotate_tile_share(uint8_t* tile, const float2* table, int row0, int S, int R,
+                                                  const RotStep& step, int tid, int part) {
+    constexpr int RP = 128 / CP;
+    constexpr int KC = CP >= PARTS ? CP / PARTS : CP;
+    if (CP < PARTS && part != 0) return;
+    const int kb = CP >= PARTS ? part * KC : 0;
+    const int rg = tid / CP, cp = tid % CP;
+    RotState<CP> st;
+    {
+        const int prow = min(row0 + rg + RP * kb, S - 1);
+        const float4* tb = reinterpret_cast<const float4*>(table + static_cast<size_t>(prow) * (R >> 1) + cp * 8);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float4 t = __ldg(tb + u);
+            st.c[u] = make_float2(t.x, t.z);
+            st.s[u] = make_float2(t.y, t.w);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < KC; ++k) {
+        const int r = rg + RP * (kb + k);
+        uint4* pl = reinterpret_cast<uint4*>(tile + swz_chunk_offset(r, cp));
+        uint4* ph = reinterpret_cast<uint4*>(tile + swz_chunk_offset(r, cp + CP));
+        uint4 lo = *pl, hi = *ph;
+        rotate_word2(lo.x, hi.x, st.c[0], st.s[0]);
+        rotate_word2(lo.y, hi.y, st.c[1], st.s[1]);
+        rotate_word2(lo.z, hi.z, st.c[2], st.s[2]);
+        rotate_word2(lo.w, hi.w, st.c[3], st.s[3]);
+        *pl = lo;
+        *ph = hi;
+        if (k + 1 < KC) {
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                const float2 nc = __ffma2_rn(st.s[w], step.ns[w], __fmul2_rn(st.c[w], step.c[w]));
+                const float2 nsn = __ffma2_rn(st.c[w], step.s[w], __fmul2_rn(st.s[w], step.c[w]));
+                st.c[w] = nc;
+                st.s[w] = nsn;
+            }
+        }
+    }
+}
+
 // Rows of the trailer: the recurrence stride for a given rotary dim (0: no fast path).
 __host__ __device__ constexpr int rope_fast_stride(int R) {
     return (R == 16 || R == 32 || R == 64 || R == 128) ? 128 / (R / 16) : 0;
