@@ -12,8 +12,11 @@
 //   P = 2^(c2 T1 + bias - L2), dS = P (T2 - delta); P, dS go back to TMEM as bf16 over T1, T2
 //   DKV: acc1 += P Bc, acc2 += dS A.      DQ: acc1 += dS A.
 // Warp roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 4-7 rotation, warps 8-11 and
-// 12-15 two gradient warpgroups: each owns 64 of the 128 columns of T1/T2 (all 128 lanes), so the
-// accumulator MMAs of the first half of the contraction start while nothing waits for the second.
+// 12-15 two gradient warpgroups: each owns 64 of the 128 columns of T1/T2 (all 128 lanes).  The MMAs are
+// issued per column half (N = 64 for T1/T2, 4 of the 8 K-steps for the accumulators) in the order
+//   T(a,n) T(b,n) | acc(a,n) T(a,n+1) | acc(b,n) T(b,n+1) | acc(a,n+1) ...
+// so that while one warpgroup turns its half of (S, dP) into (P, dS), the tensor pipe works on the other
+// half and on the next streamed tile: nothing in the loop waits for a whole tile.
 #pragma once
 #include <cuda.h>
 #include <type_traits>
@@ -67,25 +70,27 @@ struct BwdSmem {
     static constexpr int OFF_BAR = OFF_STATS + 2 * 2 * 128 * 4;
     static constexpr int B_XFULL = 0, B_XROT = 1, B_YFULL = 2, B_AFULL = 3, B_AROT = B_AFULL + NST,
                          B_BFULL = B_AROT + NST, B_EMPTY = B_BFULL + NST, B_TFULL = B_EMPTY + NST,
-                         B_PDS = B_TFULL + 1, B_DONE = B_PDS + 2, N_BARS = B_DONE + 1;   // B_PDS: one per column half
+                         B_PDS = B_TFULL + 2, B_DONE = B_PDS + 2, N_BARS = B_DONE + 1;   // TFULL, PDS: one per column half
     static constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;
     static constexpr int BYTES = OFF_MISC + 16 + 1024;
     static constexpr int STG_STRIDE = D + 4;      // floats per staged row (padding keeps 16-byte stores conflict-free)
     static_assert(128 * STG_STRIDE * 4 <= 2 * NST * TILE, "staging buffer must fit in the stream stages");
 };
 
-__device__ __forceinline__ void wg_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-// Barrier over the 256 threads of the two gradient warpgroups that also ANDs a flag, so that a wait
-// that gave up in one thread ends the loop in all of them (nobody is left alone at a barrier).
-__device__ __forceinline__ bool wg_all(bool v) {
+// Named barriers of the gradient warpgroups: id 3 joins both (256 threads), ids 1 and 2 one each.
+__device__ __forceinline__ void wg_sync() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
+// Barrier that also ANDs a flag, so that a wait that gave up in one thread ends the loop in all of
+// them (nobody is left alone at a barrier).  id/count: 3/256 for both warpgroups, 1+hf/128 for one.
+__device__ __forceinline__ bool bar_all(bool v, int id, int count) {
     uint32_t r;
     asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.and.pred q, 1, 256, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.and.pred q, %2, %3, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(r)
-        : "r"(static_cast<uint32_t>(v))
+        : "r"(static_cast<uint32_t>(v)), "r"(id), "r"(count)
         : "memory");
     return r != 0;
 }
+__device__ __forceinline__ bool wg_all(bool v) { return bar_all(v, 3, 256); }
 
 // Epilogue helper: the 256 threads of the two gradient warpgroups move a [128 x D] fp32 accumulator
 // from TMEM (thread gtid reads lane gtid % 128, column half gtid / 128) through shared memory to
@@ -146,6 +151,59 @@ __device__ __forceinline__ void store_acc_rotated(uint32_t t_acc, float* stg, in
         sn = ns;
     }
     wg_sync();
+}
+
+// One 32-column pass of a gradient warpgroup over its lane's row of T1 (scores) and T2 (dP):
+//   p = 2^(c2 * s + bias - L2),  ds = p * (dP - delta),  masked entries give 0;
+// p (DKV role only) and ds go back to TMEM as bf16 pairs at `out_col` of T1 / T2.
+// nl2 / ndl: -L2 and -delta, either per column from shared memory (DKV: the columns are query rows) or
+// the thread's own (DQ).  MASKED / ALIBI select straight-line code; arithmetic is packed fp32 (f32x2).
+template <bool DKV, bool MASKED, bool ALIBI>
+__device__ __forceinline__ void grad_pass32(uint32_t t1, uint32_t t2, int col0, uint32_t out_col, float scale_log2,
+                                            float cbias, float sb, const float* s_nl2, const float* s_ndl, float my_nl2,
+                                            float my_ndl, int mlo, uint32_t mn) {
+    uint32_t s[32], dp[32], pk[16], dk[16];
+    tmem_ld32(t1 + col0, s);
+    tmem_ld32(t2 + col0, dp);
+    tmem_wait_ld();
+    const float2 sc2 = make_float2(scale_log2, scale_log2), cb2 = make_float2(cbias, cbias);
+#pragma unroll
+    for (int e = 0; e < 32; e += 4) {
+        float2 nl[2], nd[2];
+        if (DKV) {
+            const float4 a4 = *reinterpret_cast<const float4*>(s_nl2 + col0 + e);
+            const float4 b4 = *reinterpret_cast<const float4*>(s_ndl + col0 + e);
+            nl[0] = make_float2(a4.x, a4.y); nl[1] = make_float2(a4.z, a4.w);
+            nd[0] = make_float2(b4.x, b4.y); nd[1] = make_float2(b4.z, b4.w);
+        } else {
+            nl[0] = nl[1] = make_float2(my_nl2, my_nl2);
+            nd[0] = nd[1] = make_float2(my_ndl, my_ndl);
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int c = e + 2 * u;
+            float2 t = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2,
+                                  __fadd2_rn(cb2, nl[u]));
+            if (ALIBI) {
+                t.x = fmaf(sb, static_cast<float>(c), t.x);
+                t.y = fmaf(sb, static_cast<float>(c + 1), t.y);
+            }
+            float2 pe = make_float2(ex2(t.x), ex2(t.y));
+            if (MASKED) {
+                pe.x = (static_cast<uint32_t>(col0 + c - mlo) < mn) ? pe.x : 0.f;
+                pe.y = (static_cast<uint32_t>(col0 + c + 1 - mlo) < mn) ? pe.y : 0.f;
+            }
+            const float2 ds = __fmul2_rn(pe, __fadd2_rn(make_float2(__uint_as_float(dp[c]), __uint_as_float(dp[c + 1])), nd[u]));
+            pk[c >> 1] = pack_bf16x2(pe.x, pe.y);
+            dk[c >> 1] = pack_bf16x2(ds.x, ds.y);
+        }
+    }
+    if (DKV) {
+        tmem_st16(t1 + out_col, pk);
+        tmem_st16(t2 + out_col, dk);
+    } else {
+        tmem_st16(t1 + out_col, dk);
+    }
 }
 
 // ROT_X / ROT_A: rotate the stationary tile X / every streamed tile A on chip.  The dK/dV role rotates
@@ -245,30 +303,45 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             }
             if (ok) ok = mbar_wait(&bars[L::B_YFULL], 0, abort_flag, 23);
             const uint32_t xa = smem_u32(sX), ya = smem_u32(sY);
+            constexpr uint32_t IDESC_TH = idesc_bf16_f32(128, 64, 0, 0);   // half tile: 64 streamed rows
+            // T1/T2 half hf of streamed tile n: rows [64 hf, 64 hf + 64) of A and Bc are the N index
+            auto issue_T = [&](int n, int hf) {
+                const int st = n % NST;
+                const uint32_t aa = smem_u32(sA + st * TILE) + hf * 64 * 128, ba = smem_u32(sB + st * TILE) + hf * 64 * 128;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
+                    mma_ss(tmem_base + T1 + hf * 64, smem_desc_sw128(xa + off, 16, 1024), smem_desc_sw128(aa + off, 16, 1024),
+                           IDESC_TH, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
+                    mma_ss(tmem_base + T2 + hf * 64, smem_desc_sw128(ya + off, 16, 1024), smem_desc_sw128(ba + off, 16, 1024),
+                           IDESC_TH, kk > 0);
+                }
+                mma_commit(&bars[L::B_TFULL + hf]);
+            };
+            auto wait_stream = [&](int n) {
+                const int st = n % NST;
+                bool r = mbar_wait(&bars[B_AREADY + st], (n / NST) & 1, abort_flag, 24);
+                if (r) r = mbar_wait(&bars[L::B_BFULL + st], (n / NST) & 1, abort_flag, 25);
+                tc_fence_after_sync();
+                return r;
+            };
+            if (ok && n_it > 0) ok = wait_stream(0);
+            if (ok && n_it > 0) {
+                issue_T(0, 0);
+                issue_T(0, 1);
+            }
             for (int n = 0; ok && n < n_it; ++n) {
                 const int st = n % NST;
                 const uint32_t aa = smem_u32(sA + st * TILE), ba = smem_u32(sB + st * TILE);
-                ok = mbar_wait(&bars[B_AREADY + st], (n / NST) & 1, abort_flag, 24);
-                if (ok) ok = mbar_wait(&bars[L::B_BFULL + st], (n / NST) & 1, abort_flag, 25);
-                if (!ok) break;
-                tc_fence_after_sync();
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
-                    mma_ss(tmem_base + T1, smem_desc_sw128(xa + off, 16, 1024), smem_desc_sw128(aa + off, 16, 1024),
-                           IDESC_T, kk > 0);
-                }
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
-                    mma_ss(tmem_base + T2, smem_desc_sw128(ya + off, 16, 1024), smem_desc_sw128(ba + off, 16, 1024),
-                           IDESC_T, kk > 0);
-                }
-                mma_commit(&bars[L::B_TFULL]);
-                // the contraction runs over the 128 columns of T1/T2; each gradient warpgroup delivers 64 of
-                // them (4 K = 16 steps), its bf16 results sitting at the start of its own column half
+                const bool next = n + 1 < n_it;
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
+                    // accumulate this half: 4 K = 16 steps over its 64 streamed rows; the bf16 operands sit at
+                    // the start of the half's own columns
                     ok = mbar_wait(&bars[L::B_PDS + hf], n & 1, abort_flag, 26);
                     if (!ok) break;
                     tc_fence_after_sync();
@@ -289,10 +362,16 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                                    IDESC_ACC, acc_on);
                         }
                     }
+                    if (hf == 1) mma_commit(&bars[L::B_EMPTY + st]);   // the stage is free once both halves are consumed
+                    // the same half of the next streamed tile may overwrite T1/T2 right behind (in-order pipe)
+                    if (next) {
+                        if (hf == 0) ok = wait_stream(n + 1);
+                        if (!ok) break;
+                        issue_T(n + 1, hf);
+                    }
                 }
                 if (!ok) break;
-                mma_commit(&bars[L::B_EMPTY + st]);
-                if (n == n_it - 1) mma_commit(&bars[L::B_DONE]);
+                if (!next) mma_commit(&bars[L::B_DONE]);
             }
             if (DKV && ROT_X && p.store_x) tma_store_wait_all();   // the tile must stay in place until it has been read
         }
@@ -340,8 +419,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
         float my_l2 = 0.f, my_delta = 0.f, my_slope2 = 0.f;
         if (!DKV) {
             const size_t r = (static_cast<size_t>(b) * p.Hq + xh) * p.S + xrow;
-            my_l2 = xrow < p.S ? p.lse[r] * kLog2e : INFINITY;
-            my_delta = xrow < p.S ? p.delta[r] : 0.f;
+            my_l2 = xrow < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // kept negated
+            my_delta = xrow < p.S ? -p.delta[r] : 0.f;
             my_slope2 = alibi ? p.slopes[xh] * kLog2e : 0.f;
         }
         bool ok = true;
@@ -374,12 +453,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             float* sL2 = sStats + (n & 1) * 256;
             float* sDl = sL2 + 128;
             if (DKV) {
-                // per-column statistics of the streamed query tile (written by the first warpgroup)
-                if (hf == 0) {
-                    const int qi = a0 + tid;
+                // per-column statistics of the streamed query tile: each warpgroup stages its own 64 columns
+                if (tid < 64) {
+                    const int qi = a0 + hf * 64 + tid;
                     const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + qi;
-                    sL2[tid] = qi < p.S ? p.lse[r] * kLog2e : INFINITY;
-                    sDl[tid] = qi < p.S ? p.delta[r] : 0.f;
+                    sL2[hf * 64 + tid] = qi < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // stored negated
+                    sDl[hf * 64 + tid] = qi < p.S ? -p.delta[r] : 0.f;
                 }
                 my_slope2 = alibi ? p.slopes[ah] * kLog2e : 0.f;
             }
@@ -394,50 +473,21 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             // ALiBi: slope2 * (j - i) = sb * (col + base), sb = +-slope2
             const float sb = DKV ? -my_slope2 : my_slope2;
             const float bias_base = sb * static_cast<float>(a0 - xrow);
-            ok = wg_all(mbar_wait(&bars[L::B_TFULL], n & 1, abort_flag, 29));  // also publishes the statistics
+            // this warpgroup's half of T1/T2; the barrier also publishes the statistics within the warpgroup
+            ok = bar_all(mbar_wait(&bars[L::B_TFULL + hf], n & 1, abort_flag, 29), 1 + hf, 128);
             if (!ok) break;
             tc_fence_after_sync();
 #pragma unroll
             for (int qt = 0; qt < 2; ++qt) {
                 const int col0 = hf * 64 + qt * 32;
-                uint32_t s[32], dp[32], pk[16], dk[16];
-                tmem_ld32(tb + T1 + col0, s);
-                tmem_ld32(tb + T2 + col0, dp);
-                tmem_wait_ld();
+                const uint32_t out_col = hf * 64 + qt * 16;   // bf16 results: start of this warpgroup's own half
                 const float cbias = fmaf(sb, static_cast<float>(col0), bias_base);
-#pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    float l2v[4], dlv[4];
-                    if (DKV) {
-                        const float4 a4 = *reinterpret_cast<const float4*>(sL2 + col0 + e);
-                        const float4 b4 = *reinterpret_cast<const float4*>(sDl + col0 + e);
-                        l2v[0] = a4.x; l2v[1] = a4.y; l2v[2] = a4.z; l2v[3] = a4.w;
-                        dlv[0] = b4.x; dlv[1] = b4.y; dlv[2] = b4.z; dlv[3] = b4.w;
-                    } else {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) { l2v[u] = my_l2; dlv[u] = my_delta; }
-                    }
-                    float pv[4], dv[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        float t = fmaf(__uint_as_float(s[e + u]), p.scale_log2, cbias - l2v[u]);
-                        if (alibi) t = fmaf(sb, static_cast<float>(e + u), t);
-                        float pe = ex2(t);
-                        if (need_mask) pe = (static_cast<uint32_t>(col0 + e + u - mlo) < mn) ? pe : 0.f;
-                        pv[u] = pe;
-                        dv[u] = pe * (__uint_as_float(dp[e + u]) - dlv[u]);
-                    }
-                    pk[e >> 1] = pack_bf16x2(pv[0], pv[1]);
-                    pk[(e >> 1) + 1] = pack_bf16x2(pv[2], pv[3]);
-                    dk[e >> 1] = pack_bf16x2(dv[0], dv[1]);
-                    dk[(e >> 1) + 1] = pack_bf16x2(dv[2], dv[3]);
-                }
-                // bf16 results go to the start of this warpgroup's own column half (already read)
-                if (DKV) {
-                    tmem_st16(tb + T1 + hf * 64 + qt * 16, pk);
-                    tmem_st16(tb + T2 + hf * 64 + qt * 16, dk);
+                if (alibi) {
+                    if (need_mask) grad_pass32<DKV, true, true>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, my_l2, my_delta, mlo, mn);
+                    else grad_pass32<DKV, false, true>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, my_l2, my_delta, mlo, mn);
                 } else {
-                    tmem_st16(tb + T1 + hf * 64 + qt * 16, dk);
+                    if (need_mask) grad_pass32<DKV, true, false>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, my_l2, my_delta, mlo, mn);
+                    else grad_pass32<DKV, false, false>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, my_l2, my_delta, mlo, mn);
                 }
             }
             tmem_wait_st();
