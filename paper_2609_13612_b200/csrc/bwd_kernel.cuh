@@ -305,20 +305,24 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             const uint32_t xa = smem_u32(sX), ya = smem_u32(sY);
             constexpr uint32_t IDESC_TH = idesc_bf16_f32(128, 64, 0, 0);   // half tile: 64 streamed rows
             // T1/T2 half hf of streamed tile n: rows [64 hf, 64 hf + 64) of A and Bc are the N index
+            const uint32_t dhi = desc_hi(1024);
+            const uint32_t x_lo = desc_lo(xa, 16), y_lo = desc_lo(ya, 16);
             auto issue_T = [&](int n, int hf) {
                 const int st = n % NST;
-                const uint32_t aa = smem_u32(sA + st * TILE) + hf * 64 * 128, ba = smem_u32(sB + st * TILE) + hf * 64 * 128;
+                const uint32_t a_lo = desc_lo(smem_u32(sA + st * TILE) + hf * 64 * 128, 16);
+                const uint32_t b_lo = desc_lo(smem_u32(sB + st * TILE) + hf * 64 * 128, 16);
+                const uint32_t d1 = tmem_base + T1 + hf * 64, d2 = tmem_base + T2 + hf * 64;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
-                    mma_ss(tmem_base + T1 + hf * 64, smem_desc_sw128(xa + off, 16, 1024), smem_desc_sw128(aa + off, 16, 1024),
-                           IDESC_TH, kk > 0);
+                    const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
+                    if (kk == 0) mma_ss_lo<false>(d1, x_lo + off, a_lo + off, dhi, IDESC_TH);
+                    else mma_ss_lo<true>(d1, x_lo + off, a_lo + off, dhi, IDESC_TH);
                 }
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
-                    mma_ss(tmem_base + T2 + hf * 64, smem_desc_sw128(ya + off, 16, 1024), smem_desc_sw128(ba + off, 16, 1024),
-                           IDESC_TH, kk > 0);
+                    const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
+                    if (kk == 0) mma_ss_lo<false>(d2, y_lo + off, b_lo + off, dhi, IDESC_TH);
+                    else mma_ss_lo<true>(d2, y_lo + off, b_lo + off, dhi, IDESC_TH);
                 }
                 mma_commit(&bars[L::B_TFULL + hf]);
             };
@@ -336,7 +340,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             }
             for (int n = 0; ok && n < n_it; ++n) {
                 const int st = n % NST;
-                const uint32_t aa = smem_u32(sA + st * TILE), ba = smem_u32(sB + st * TILE);
+                // MN-major B operands of the accumulator MMAs: 16 streamed rows (2 KB) per K step
+                const uint32_t am_lo = desc_lo(smem_u32(sA + st * TILE), BOX_BYTES), bm_lo = desc_lo(smem_u32(sB + st * TILE), BOX_BYTES);
                 const bool next = n + 1 < n_it;
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
@@ -352,14 +357,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                         const uint32_t acc_on = (n > 0 || kk > 0) ? 1u : 0u;
                         if (DKV) {
                             // acc1 (dV) += P^T dO, acc2 (dK') += dS^T Q': dO and Q' are MN-major B operands
-                            mma_ts(tmem_base + ACC1, tmem_base + T1 + a_off, smem_desc_sw128(ba + kk * 2048, BOX_BYTES, 1024),
-                                   IDESC_ACC, acc_on);
-                            mma_ts(tmem_base + ACC2, tmem_base + T2 + a_off, smem_desc_sw128(aa + kk * 2048, BOX_BYTES, 1024),
-                                   IDESC_ACC, acc_on);
+                            mma_ts_lo(tmem_base + ACC1, tmem_base + T1 + a_off, bm_lo + kk * 128, dhi, IDESC_ACC, acc_on);
+                            mma_ts_lo(tmem_base + ACC2, tmem_base + T2 + a_off, am_lo + kk * 128, dhi, IDESC_ACC, acc_on);
                         } else {
                             // acc1 (dQ') += dS K'
-                            mma_ts(tmem_base + ACC1, tmem_base + T1 + a_off, smem_desc_sw128(aa + kk * 2048, BOX_BYTES, 1024),
-                                   IDESC_ACC, acc_on);
+                            mma_ts_lo(tmem_base + ACC1, tmem_base + T1 + a_off, am_lo + kk * 128, dhi, IDESC_ACC, acc_on);
                         }
                     }
                     if (hf == 1) mma_commit(&bars[L::B_EMPTY + st]);   // the stage is free once both halves are consumed
