@@ -236,24 +236,26 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
             for (int q = 0; q < NQ; ++q) cnt[q] = 0;
 
+            // descriptors differ only in their low word: one add per operand and step
+            const uint32_t dhi = desc_hi(1024);
             auto issue_S = [&](int q, int ks) {
-                const uint32_t qa = smem_u32(sQ + q * TILE), ka = smem_u32(sK + ks * TILE);
+                const uint32_t q_lo = desc_lo(smem_u32(sQ + q * TILE), 16), k_lo = desc_lo(smem_u32(sK + ks * TILE), 16);
+                const uint32_t d = tmem_base + q * BN;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * BOX_BYTES + (kk & 3) * 32;
-                    mma_ss(tmem_base + q * BN, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024),
-                           IDESC_S, kk > 0);
+                    const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
+                    if (kk == 0) mma_ss_lo<false>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
+                    else mma_ss_lo<true>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
                 }
                 mma_commit(&bars[L::B_SFULL + q]);
             };
             auto issue_O = [&](int q, int vs, bool acc) {
-                const uint32_t va = smem_u32(sV + vs * TILE);
+                // V is [BN key rows][D]: MN-major B operand; 16 key rows per step = 2 KB
+                const uint32_t v_lo = desc_lo(smem_u32(sV + vs * TILE), BOX_BYTES);
+                const uint32_t d = tmem_base + NQ * BN + q * D, a = tmem_base + q * BN;
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk) {
-                    // V is [BN key rows][D]: MN-major B operand; 16 key rows per step = 2 KB
-                    mma_ts(tmem_base + NQ * BN + q * D, tmem_base + q * BN + kk * 8,
-                           smem_desc_sw128(va + kk * 2048, BOX_BYTES, 1024), IDESC_O, (acc || kk > 0) ? 1u : 0u);
-                }
+                for (int kk = 0; kk < BN / 16; ++kk)
+                    mma_ts_lo(d, a + kk * 8, v_lo + kk * 128, dhi, IDESC_O, (acc || kk > 0) ? 1u : 0u);
             };
 
             // prologue: S of the first key tile, each query tile as soon as it is ready (the softmax
