@@ -10,6 +10,7 @@
 #include "../../include/attnfuse.h"
 #include "bwd_kernel.cuh"
 #include "fwd_kernel.cuh"
+#include "fwd2_kernel.cuh"
 #include "rope_kernels.cuh"
 
 namespace {
@@ -111,6 +112,37 @@ af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const
     dim3 grid(p.pair_heads ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
     kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+// CTA-pair variant (fwd2_kernel.cuh): clusters of two CTAs, one per (batch, head quad, 128-row block).
+// tk2: tensor map over K with 64-row boxes.
+template <bool ROPE>
+af_status launch_fwd2_variant(const CUtensorMap& tq, const CUtensorMap& tk2, const CUtensorMap& tv, FwdParams p,
+                              cudaStream_t stream) {
+    constexpr int KS = 3, VS = 3;
+    using L = Fwd2Smem<128, KS, VS>;
+    auto kern = attn_fwd2_kernel<128, ROPE, KS, VS>;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
+            return AF_ERR_CUDA;
+        configured = true;
+    }
+    p.pair_heads = 0;
+    p.n_row_blocks = (p.S + BM - 1) / BM;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2u * p.B * (p.Hq / 4), p.n_row_blocks, 1);
+    cfg.blockDim = dim3(512, 1, 1);
+    cfg.dynamicSmemBytes = L::BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, tq, tk2, tv, p) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
 template <int D>
@@ -292,6 +324,13 @@ af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, cons
     p.trace = reinterpret_cast<long long*>(getenv("AF_TRACE_PTR") ? strtoull(getenv("AF_TRACE_PTR"), nullptr, 0) : 0ull);
 #endif
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int R = rope->rotary_dim;
+    const bool pair_ok = shape->D == 128 && (gqa_group % 4) == 0 && (R == 0 || R == 16 || R == 32 || R == 64 || R == 128);
+    if (pair_ok && env_int("AF_FWD_2CTA", 0)) {
+        CUtensorMap tk2;
+        if ((st = make_tmap(&tk2, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, 64)) != AF_OK) return st;
+        return R > 0 ? launch_fwd2_variant<true>(tq, tk2, tv, p, stream) : launch_fwd2_variant<false>(tq, tk2, tv, p, stream);
+    }
     return shape->D == 128 ? launch_fwd<128>(tq, tk, tv, p, stream) : launch_fwd<64>(tq, tk, tv, p, stream);
 }
 
