@@ -56,6 +56,10 @@ struct FwdSmem {
 #define AF_STAMP(role, it, ph) do { } while (0)
 #endif
 
+#ifndef AF_POLY_EVERY
+#define AF_POLY_EVERY 0
+#endif
+constexpr int kPolyEvery = AF_POLY_EVERY;   // share of exps computed by polynomial: 1 in kPolyEvery pairs (0: none)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the row max grows by more
 
 // One key tile of the online softmax for one query row (this thread's TMEM lane): reads the 128
@@ -102,7 +106,9 @@ __device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, fl
     for (int e = 0; e < BN; e += 2) {
         // packed fp32: one instruction scales and shifts two scores, one adds two probabilities
         const float2 t = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), sc2, sub2);
-        const float2 pe = make_float2(ex2(t.x), ex2(t.y));
+        // every kPolyEvery-th pair takes the polynomial on the FMA pipe, the rest the special-function unit
+        const float2 pe = (kPolyEvery > 0 && ((e >> 1) % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) ? ex2_poly2(t)
+                                                                                               : make_float2(ex2(t.x), ex2(t.y));
         ps2[(e >> 1) & 1] = __fadd2_rn(ps2[(e >> 1) & 1], pe);
         pk[e >> 1] = pack_bf16x2(pe.x, pe.y);
     }
