@@ -322,6 +322,7 @@ af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, cons
     p.pair_heads = 0;
 #ifdef AF_TRACE
     p.trace = reinterpret_cast<long long*>(getenv("AF_TRACE_PTR") ? strtoull(getenv("AF_TRACE_PTR"), nullptr, 0) : 0ull);
+    cudaMemcpyToSymbol(af::g_trace, &p.trace, sizeof(p.trace));
 #endif
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int R = rope->rotary_dim;

@@ -38,7 +38,7 @@ struct FwdSmem {
     // barrier slots
     static constexpr int B_QFULL = 0, B_QROT = B_QFULL + NQ, B_KFULL = B_QROT + NQ, B_KROT = B_KFULL + KS,
                          B_KEMPTY = B_KROT + KS, B_VFULL = B_KEMPTY + KS, B_VEMPTY = B_VFULL + VS,
-                         B_SFULL = B_VEMPTY + VS, B_PREADY = B_SFULL + NQ, B_ODONE = B_PREADY + NQ,
+                         B_SFULL = B_VEMPTY + VS, B_PREADY = B_SFULL + 2 * NQ, B_ODONE = B_PREADY + 4 * NQ,   // SFULL: per column half; PREADY: per P part (up to 4)
                          N_BARS = B_ODONE + NQ;
     static constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;
     static constexpr int BYTES = OFF_MISC + 16 + 1024;  // + alignment slack
@@ -52,12 +52,22 @@ struct FwdSmem {
         if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && (it) < 64)     \
             p.trace[((role) * 64 + (it)) * 8 + (ph)] = clock64();                                      \
     } while (0)
+// fine-grained stamps inside softmax_tile: slots 3..7 of role 2 (query tile 0, warp 8 lane 0 only)
+#define AF_STAMP_SM(ph)                                                                                \
+    do {                                                                                               \
+        if (g_trace && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 256 && n < 64)             \
+            g_trace[(2 * 64 + n) * 8 + (ph)] = clock64();                                              \
+    } while (0)
 #else
 #define AF_STAMP(role, it, ph) do { } while (0)
+#define AF_STAMP_SM(ph) do { } while (0)
 #endif
 
 #ifndef AF_POLY_EVERY
 #define AF_POLY_EVERY 0
+#endif
+#ifdef AF_TRACE
+__device__ long long* g_trace = nullptr;
 #endif
 constexpr int kPolyEvery = AF_POLY_EVERY;   // share of exps computed by polynomial: 1 in kPolyEvery pairs (0: none)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the row max grows by more
@@ -76,6 +86,7 @@ __device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, fl
     tmem_ld32(tS + 64, v + 64);
     tmem_ld32(tS + 96, v + 96);
     tmem_wait_ld();
+    AF_STAMP_SM(3);
     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
     for (int e = 0; e < BN; e += 2) {
@@ -91,6 +102,7 @@ __device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, fl
     }
     // scale > 0, so the max commutes with it
     const float mx = fmaf(fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]), scale_log2, bias0);
+    AF_STAMP_SM(4);
     // lazy rescale: keep the old reference max unless it grew by more than the threshold
     const bool upd = mx > m_run + kRescaleThreshold;
     float alpha = 1.f;
@@ -114,6 +126,7 @@ __device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, fl
     }
     tmem_st32(tS, pk);
     tmem_st32(tS + 32, pk + 32);
+    AF_STAMP_SM(5);
     l_run = l_run * alpha + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
     if (n > 0 && __any_sync(0xffffffffu, upd)) {
 #pragma unroll 1
@@ -127,6 +140,112 @@ __device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, fl
         }
     }
     tmem_wait_st();
+    AF_STAMP_SM(6);
+}
+
+#ifndef AF_SPLIT_S
+#define AF_SPLIT_S 0
+#endif
+constexpr bool kSplitS = AF_SPLIT_S != 0;   // S tile produced as two N = 64 halves (measured slower: N = 64 MMAs are inefficient)
+#ifndef AF_P_PARTS
+#define AF_P_PARTS 2
+#endif
+constexpr int kPParts = AF_P_PARTS;          // P is handed to the MMA issuer in this many column parts (2 or 4)
+
+// The same tile step with the work handed over in column halves, so that less of it sits on the
+// S-MMA -> softmax -> PV-MMA dependency chain of a query tile:
+//  - with kSplitS the scores arrive as two 64-column halves (two barriers): the TMEM load of the first
+//    half overlaps the MMAs of the second;
+//  - P goes back in two halves, each announced on its own barrier (p_ready[0], p_ready[1]), so that the
+//    first four K-steps of O += P V run while the second half of the exponentials is computed.
+// P halves sit at the start of their own 64 score columns (bf16 pairs: 32 columns each).
+// Returns false if a bounded wait gave up.
+template <int D, bool MASKED, bool ALIBI>
+__device__ __forceinline__ bool softmax_tile_halves(uint32_t tS, uint32_t tO, int n, float scale_log2, float kb,
+                                                    float bias0, int mlo, uint32_t mn, uint64_t* s_full, uint64_t* p_ready,
+                                                    uint32_t parity, volatile uint32_t* abort_flag, int lane, float& m_run,
+                                                    float& l_run) {
+    uint32_t v[BN];
+    if (!mbar_wait_warp(&s_full[0], parity, abort_flag, 10)) return false;
+    tc_fence_after_sync();
+    tmem_ld32(tS, v);
+    tmem_ld32(tS + 32, v + 32);
+    if (kSplitS) {
+        if (!mbar_wait_warp(&s_full[1], parity, abort_flag, 10)) {
+            tmem_wait_ld();
+            return false;
+        }
+        tc_fence_after_sync();
+    }
+    tmem_ld32(tS + 64, v + 64);
+    tmem_ld32(tS + 96, v + 96);
+    tmem_wait_ld();
+    AF_STAMP_SM(3);
+    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+    for (int e = 0; e < BN; e += 2) {
+        float sv[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            sv[u] = __uint_as_float(v[e + u]);
+            if (ALIBI) sv[u] = fmaf(kb, static_cast<float>(e + u), sv[u]);
+            if (MASKED) sv[u] = (static_cast<uint32_t>(e + u - mlo) < mn) ? sv[u] : -INFINITY;
+            if (ALIBI || MASKED) v[e + u] = __float_as_uint(sv[u]);
+        }
+        mx4[(e >> 1) & 3] = fmax3(mx4[(e >> 1) & 3], sv[0], sv[1]);   // two scores per instruction
+    }
+    // scale > 0, so the max commutes with it
+    const float mx = fmaf(fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]), scale_log2, bias0);
+    AF_STAMP_SM(4);
+    // lazy rescale: keep the old reference max unless it grew by more than the threshold
+    const bool upd = mx > m_run + kRescaleThreshold;
+    float alpha = 1.f;
+    if (upd) {
+        alpha = ex2(m_run - mx);  // m_run = -inf -> 0
+        m_run = mx;
+    }
+    const float sub = bias0 - ((m_run == -INFINITY) ? 0.f : m_run);
+    const float2 sc2 = make_float2(scale_log2, scale_log2), sub2 = make_float2(sub, sub);
+    float2 ps2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+    constexpr int CPP = 4 / kPParts;   // 32-column chunks per part
+#pragma unroll
+    for (int pt = 0; pt < kPParts; ++pt) {
+#pragma unroll
+        for (int c = 0; c < CPP; ++c) {
+            uint32_t pk[16];
+            const int col0 = (pt * CPP + c) * 32;
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+                // packed fp32: one instruction scales and shifts two scores, one adds two probabilities
+                const float2 t = __ffma2_rn(make_float2(__uint_as_float(v[col0 + e]), __uint_as_float(v[col0 + e + 1])), sc2, sub2);
+                const float2 pe = make_float2(ex2(t.x), ex2(t.y));
+                ps2[(e >> 1) & 1] = __fadd2_rn(ps2[(e >> 1) & 1], pe);
+                pk[e >> 1] = pack_bf16x2(pe.x, pe.y);
+            }
+            // a part's bf16 pairs sit at the start of the part's own score columns
+            tmem_st16(tS + pt * (BN / kPParts) + c * 16, pk);
+        }
+        if (pt == 0 && n > 0 && __any_sync(0xffffffffu, upd)) {
+            // the accumulator must be rescaled before the first part of P V is added to it
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tO + c * 32, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                tmem_st32(tO + c * 32, o);
+            }
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_ready[pt]);
+        if (pt == 0) AF_STAMP_SM(5);
+    }
+    l_run = l_run * alpha + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
+    AF_STAMP_SM(6);
+    return true;
 }
 
 template <int D, int NQ, bool ROPE, int KS, int VS>
@@ -183,7 +302,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int i = 0; i < L::N_BARS; ++i) {
             uint32_t cnt = 1;
             if ((i >= L::B_QROT && i < L::B_QROT + NQ) || (i >= L::B_KROT && i < L::B_KROT + KS) ||
-                (i >= L::B_PREADY && i < L::B_PREADY + NQ))
+                (i >= L::B_PREADY && i < L::B_PREADY + 4 * NQ))
                 cnt = 4;  // one elected arrive per warp of the producing warpgroup
             mbar_init(&bars[i], cnt);
         }
@@ -247,21 +366,37 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             auto issue_S = [&](int q, int ks) {
                 const uint32_t q_lo = desc_lo(smem_u32(sQ + q * TILE), 16), k_lo = desc_lo(smem_u32(sK + ks * TILE), 16);
                 const uint32_t d = tmem_base + q * BN;
+                if (kSplitS) {
+                    // two N = 64 halves: key rows [64 h, 64 h + 64) of the tile (8 KB further in each box)
+                    constexpr uint32_t IDESC_SH = idesc_bf16_f32(BM, 64, 0, 0);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
-                    if (kk == 0) mma_ss_lo<false>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
-                    else mma_ss_lo<true>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
+                    for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+                        for (int kk = 0; kk < D / 16; ++kk) {
+                            const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
+                            if (kk == 0) mma_ss_lo<false>(d + hf * 64, q_lo + off, k_lo + off + hf * 512, dhi, IDESC_SH);
+                            else mma_ss_lo<true>(d + hf * 64, q_lo + off, k_lo + off + hf * 512, dhi, IDESC_SH);
+                        }
+                        mma_commit(&bars[L::B_SFULL + 2 * q + hf]);
+                    }
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
+                        if (kk == 0) mma_ss_lo<false>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
+                        else mma_ss_lo<true>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
+                    }
+                    mma_commit(&bars[L::B_SFULL + 2 * q]);
                 }
-                mma_commit(&bars[L::B_SFULL + q]);
             };
-            auto issue_O = [&](int q, int vs, bool acc) {
-                // V is [BN key rows][D]: MN-major B operand; 16 key rows per step = 2 KB
+            // part pt of O += P V: its 8 / kPParts K-steps; that part of P starts at its own score columns
+            auto issue_O_part = [&](int q, int vs, bool acc, int pt) {
+                constexpr int KPP = 8 / kPParts;
                 const uint32_t v_lo = desc_lo(smem_u32(sV + vs * TILE), BOX_BYTES);
-                const uint32_t d = tmem_base + NQ * BN + q * D, a = tmem_base + q * BN;
+                const uint32_t d = tmem_base + NQ * BN + q * D, a = tmem_base + q * BN + pt * (BN / kPParts);
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk)
-                    mma_ts_lo(d, a + kk * 8, v_lo + kk * 128, dhi, IDESC_O, (acc || kk > 0) ? 1u : 0u);
+                for (int k = 0; k < KPP; ++k)
+                    mma_ts_lo(d, a + k * 8, v_lo + (pt * KPP + k) * 128, dhi, IDESC_O, (acc || pt > 0 || k > 0) ? 1u : 0u);
             };
 
             // prologue: S of the first key tile, each query tile as soon as it is ready (the softmax
@@ -288,11 +423,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
                     if (ok && j >= jlo[q] && j <= jhi[q]) {
-                        ok = mbar_wait(&bars[L::B_PREADY + q], cnt[q] & 1, abort_flag, 6);
-                        AF_STAMP(0, it, 2 + 3 * q);
+#pragma unroll
+                        for (int pt = 0; pt < kPParts; ++pt) {
+                            if (ok) ok = mbar_wait(&bars[L::B_PREADY + 4 * q + pt], cnt[q] & 1, abort_flag, 6);
+                            if (pt == 0) AF_STAMP(0, it, 2 + 3 * q);
+                            if (ok) {
+                                tc_fence_after_sync();
+                                issue_O_part(q, vs, cnt[q] > 0, pt);
+                            }
+                        }
                         if (ok) {
-                            tc_fence_after_sync();
-                            issue_O(q, vs, cnt[q] > 0);
                             AF_STAMP(0, it, 3 + 3 * q);
                             ++cnt[q];
                             if (j == jhi[q]) mma_commit(&bars[L::B_ODONE + q]);
@@ -393,25 +533,20 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int j = jlo[q]; ok && j <= jhi[q]; ++j, ++n) {
             const int j0 = j * BN;
             AF_STAMP(2 + q, n, 0);
-            ok = mbar_wait_warp(&bars[L::B_SFULL + q], n & 1, abort_flag, 10);
-            AF_STAMP(2 + q, n, 1);
-            if (!ok) break;
-            tc_fence_after_sync();
             const bool need_mask = tile_needs_mask(ms, i0[q], j0);
             const float bias0 = slope2 * static_cast<float>(j0 - i);
             int mlo = 0;
             uint32_t mn = BN;
             if (need_mask) kept_keys_of_query(ms, i, j0, mlo, mn);
+            uint64_t* sf = &bars[L::B_SFULL + 2 * q];
+            uint64_t* pr = &bars[L::B_PREADY + 4 * q];
             if (alibi) {
-                if (need_mask) softmax_tile<D, true, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
-                else softmax_tile<D, false, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
+                if (need_mask) ok = softmax_tile_halves<D, true, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
+                else ok = softmax_tile_halves<D, false, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
             } else {
-                if (need_mask) softmax_tile<D, true, false>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
-                else softmax_tile<D, false, false>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
+                if (need_mask) ok = softmax_tile_halves<D, true, false>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
+                else ok = softmax_tile_halves<D, false, false>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
             }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars[L::B_PREADY + q]);
             AF_STAMP(2 + q, n, 2);
         }
         // epilogue (Section 4.4: save L = m + ln l)
