@@ -29,10 +29,10 @@ struct Fwd2Smem {
     static constexpr int OFF_V = OFF_K + KS * KHALF;
     static constexpr int OFF_BAR = OFF_V + VS * VHALF;
     static constexpr int B_QFULL = 0, B_KFULL = B_QFULL + 2, B_VFULL = B_KFULL + KS, B_KEMPTY = B_VFULL + VS,
-                         B_VEMPTY = B_KEMPTY + KS, B_SFULL = B_VEMPTY + VS, B_ODONE = B_SFULL + 2,
+                         B_VEMPTY = B_KEMPTY + KS, B_SFULL = B_VEMPTY + VS, B_ODONE = B_SFULL + 4,   // SFULL: two slots per tile (first used)
                          // consumed by the leader's MMA thread, arrivals from both CTAs:
                          B_QREADY = B_ODONE + 2, B_KREADY = B_QREADY + 2, B_VREADY = B_KREADY + KS,
-                         B_PREADY = B_VREADY + VS, N_BARS = B_PREADY + 2;
+                         B_PREADY = B_VREADY + VS, N_BARS = B_PREADY + 8;   // PREADY: up to four P parts per tile
     static constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;
     static constexpr int BYTES = OFF_MISC + 16 + 1024;
 };
@@ -113,7 +113,7 @@ attn_fwd2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         for (int i = 0; i < L::N_BARS; ++i) {
             uint32_t cnt = 1;
             if ((i >= L::B_QREADY && i < L::B_QREADY + 2) || (i >= L::B_KREADY && i < L::B_KREADY + KS) ||
-                (i >= L::B_PREADY && i < L::B_PREADY + 2))
+                (i >= L::B_PREADY && i < L::B_PREADY + 8))
                 cnt = 8;   // four warps of a warpgroup in each of the two CTAs
             if (i >= L::B_VREADY && i < L::B_VREADY + VS) cnt = 2;   // one relay thread per CTA
             mbar_init(&bars[i], cnt);
@@ -176,14 +176,15 @@ attn_fwd2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     if (kk == 0) mma2_ss_lo<false>(d, q_lo + qoff, k_lo + koff, dhi, IDESC_S);
                     else mma2_ss_lo<true>(d, q_lo + qoff, k_lo + koff, dhi, IDESC_S);
                 }
-                mma2_commit_both(&bars[L::B_SFULL + q]);
+                mma2_commit_both(&bars[L::B_SFULL + 2 * q]);
             };
-            auto issue_O = [&](int q, int vs, bool acc) {
+            auto issue_O_part = [&](int q, int vs, bool acc, int pt) {
+                constexpr int KPP = 8 / kPParts;
                 const uint32_t v_lo = desc_lo(smem_u32(sV + vs * L::VHALF), BOX_BYTES);
-                const uint32_t d = tmem_base + NQ * BN + q * D, a = tmem_base + q * BN;
+                const uint32_t d = tmem_base + NQ * BN + q * D, a = tmem_base + q * BN + pt * (BN / kPParts);
 #pragma unroll
-                for (int kk = 0; kk < BN / 16; ++kk)
-                    mma2_ts_lo(d, a + kk * 8, v_lo + kk * 128, dhi, IDESC_O, (acc || kk > 0) ? 1u : 0u);
+                for (int k = 0; k < KPP; ++k)
+                    mma2_ts_lo(d, a + k * 8, v_lo + (pt * KPP + k) * 128, dhi, IDESC_O, (acc || pt > 0 || k > 0) ? 1u : 0u);
             };
             ok = mbar_wait_cluster(&bars[L::B_KREADY + 0], 0, abort_flag, 44);
 #pragma unroll
@@ -200,12 +201,15 @@ attn_fwd2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 ok = mbar_wait_cluster(&bars[L::B_VREADY + vs], (it / VS) & 1, abort_flag, 45);
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
-                    if (ok) ok = mbar_wait_cluster(&bars[L::B_PREADY + q], it & 1, abort_flag, 46);
-                    if (ok) {
-                        tc_fence_after_sync();
-                        issue_O(q, vs, it > 0);
-                        if (!next) mma2_commit_both(&bars[L::B_ODONE + q]);
+#pragma unroll
+                    for (int pt = 0; pt < kPParts; ++pt) {
+                        if (ok) ok = mbar_wait_cluster(&bars[L::B_PREADY + 4 * q + pt], it & 1, abort_flag, 46);
+                        if (ok) {
+                            tc_fence_after_sync();
+                            issue_O_part(q, vs, it > 0, pt);
+                        }
                     }
+                    if (ok && !next) mma2_commit_both(&bars[L::B_ODONE + q]);
                     if (ok && next) {
                         if (!kwaited) {
                             ok = mbar_wait_cluster(&bars[L::B_KREADY + ks1], ((it + 1) / KS) & 1, abort_flag, 47);
@@ -301,24 +305,21 @@ attn_fwd2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         for (int it = 0; ok && it < n_it; ++it) {
             const int j0 = (jlo + it) * BN;
-            ok = mbar_wait_warp(&bars[L::B_SFULL + q], it & 1, abort_flag, 51);
-            if (!ok) break;
-            tc_fence_after_sync();
             const bool need_mask = tile_needs_mask(ms, i0, j0);
             const float bias0 = slope2 * static_cast<float>(j0 - i);
             int mlo = 0;
             uint32_t mn = BN;
             if (need_mask) kept_keys_of_query(ms, i, j0, mlo, mn);
+            uint64_t* sf = &bars[L::B_SFULL + 2 * q];
+            uint64_t* pr = &bars[L::B_PREADY + 4 * q];
+            const int n = it;
             if (alibi) {
-                if (need_mask) softmax_tile<D, true, true>(tS, tO, it, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
-                else softmax_tile<D, false, true>(tS, tO, it, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
+                if (need_mask) ok = softmax_tile_halves<D, true, true, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
+                else ok = softmax_tile_halves<D, false, true, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
             } else {
-                if (need_mask) softmax_tile<D, true, false>(tS, tO, it, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
-                else softmax_tile<D, false, false>(tS, tO, it, p.scale_log2, kb, bias0, mlo, mn, m_run, l_run);
+                if (need_mask) ok = softmax_tile_halves<D, true, false, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
+                else ok = softmax_tile_halves<D, false, false, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
             }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(&bars[L::B_PREADY + q], 0);
         }
         // epilogue (Section 4.4: save L = m + ln l)
         if (ok) ok = mbar_wait_warp(&bars[L::B_ODONE + q], 0, abort_flag, 52);

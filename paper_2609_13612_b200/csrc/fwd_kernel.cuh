@@ -160,7 +160,8 @@ constexpr int kPParts = AF_P_PARTS;          // P is handed to the MMA issuer in
 //    first four K-steps of O += P V run while the second half of the exponentials is computed.
 // P halves sit at the start of their own 64 score columns (bf16 pairs: 32 columns each).
 // Returns false if a bounded wait gave up.
-template <int D, bool MASKED, bool ALIBI>
+// PAIR: the barriers p_ready live in the leader CTA of a CTA pair (arrive through the cluster).
+template <int D, bool MASKED, bool ALIBI, bool PAIR = false>
 __device__ __forceinline__ bool softmax_tile_halves(uint32_t tS, uint32_t tO, int n, float scale_log2, float kb,
                                                     float bias0, int mlo, uint32_t mn, uint64_t* s_full, uint64_t* p_ready,
                                                     uint32_t parity, volatile uint32_t* abort_flag, int lane, float& m_run,
@@ -240,7 +241,10 @@ __device__ __forceinline__ bool softmax_tile_halves(uint32_t tS, uint32_t tO, in
         tmem_wait_st();
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&p_ready[pt]);
+        if (lane == 0) {
+            if (PAIR) mbar_arrive_cluster(&p_ready[pt], 0);
+            else mbar_arrive(&p_ready[pt]);
+        }
         if (pt == 0) AF_STAMP_SM(5);
     }
     l_run = l_run * alpha + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
