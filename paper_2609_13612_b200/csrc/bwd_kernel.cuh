@@ -252,6 +252,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             uint32_t cnt = 1;
             if ((i >= L::B_AROT && i < L::B_AROT + NST) || i == L::B_PDS || i == L::B_PDS + 1) cnt = 4;  // per-warp arrives
             if (i == L::B_XROT) cnt = 8;  // both gradient warpgroups
+            if (i == L::B_TFULL || i == L::B_TFULL + 1 || i == L::B_DONE || (i >= L::B_EMPTY && i < L::B_EMPTY + NST))
+                cnt = 2;  // one arrival per MMA issuer
             mbar_init(&bars[i], cnt);
         }
         *abort_flag = 0;
@@ -289,50 +291,55 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == 2) {
+        // ------------------------------------------------------------ MMA issuers
+        // Two issuing threads on different SM sub-partitions, split by product so that every accumulator has
+        // exactly one issuer (the order of its additions stays fixed: deterministic results):
+        //   issuer 0: T1 = X A^T and acc1 (DKV: dV += P^T dO;  DQ: dQ' += dS K')
+        //   issuer 1: T2 = Y Bc^T and, in the DKV role, acc2 (dK' += dS^T Q')
+        // A single thread issuing all 48 MMAs of a tile pair was the bottleneck of this kernel.
         if (lane == 0) {
             constexpr int B_XREADY = ROT_X ? L::B_XROT : L::B_XFULL;
             constexpr int B_AREADY = ROT_A ? L::B_AROT : L::B_AFULL;
-            bool ok = mbar_wait(&bars[B_XREADY], 0, abort_flag, 22);
-            if (ok && DKV && ROT_X && p.store_x) {
-                // publish the rotated K' tile (rows past S are clipped by the tensor map)
+            const int who = warp - 1;
+            bool ok = true;
+            if (who == 0) {
+                ok = mbar_wait(&bars[B_XREADY], 0, abort_flag, 22);
+                if (ok && DKV && ROT_X && p.store_x) {
+                    // publish the rotated K' tile (rows past S are clipped by the tensor map)
 #pragma unroll
-                for (int bx = 0; bx < NBOX; ++bx) tma_store_4d(&tm_s, sX + bx * BOX_BYTES, bx * BOX_COLS, x0, xh, b);
-                tma_store_commit();
+                    for (int bx = 0; bx < NBOX; ++bx) tma_store_4d(&tm_s, sX + bx * BOX_BYTES, bx * BOX_COLS, x0, xh, b);
+                    tma_store_commit();
+                }
+            } else {
+                ok = mbar_wait(&bars[L::B_YFULL], 0, abort_flag, 23);
             }
-            if (ok) ok = mbar_wait(&bars[L::B_YFULL], 0, abort_flag, 23);
             const uint32_t xa = smem_u32(sX), ya = smem_u32(sY);
             constexpr uint32_t IDESC_TH = idesc_bf16_f32(128, 64, 0, 0);   // half tile: 64 streamed rows
-            // T1/T2 half hf of streamed tile n: rows [64 hf, 64 hf + 64) of A and Bc are the N index
             const uint32_t dhi = desc_hi(1024);
-            const uint32_t x_lo = desc_lo(xa, 16), y_lo = desc_lo(ya, 16);
+            const uint32_t s_lo = desc_lo(who == 0 ? xa : ya, 16);          // this issuer's stationary operand
+            const uint32_t t_dst = tmem_base + (who == 0 ? T1 : T2);
+            // T1 or T2, half hf of streamed tile n: rows [64 hf, 64 hf + 64) of A (or Bc) are the N index
             auto issue_T = [&](int n, int hf) {
                 const int st = n % NST;
-                const uint32_t a_lo = desc_lo(smem_u32(sA + st * TILE) + hf * 64 * 128, 16);
-                const uint32_t b_lo = desc_lo(smem_u32(sB + st * TILE) + hf * 64 * 128, 16);
-                const uint32_t d1 = tmem_base + T1 + hf * 64, d2 = tmem_base + T2 + hf * 64;
+                const uint32_t r_lo = desc_lo(smem_u32((who == 0 ? sA : sB) + st * TILE) + hf * 64 * 128, 16);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
-                    if (kk == 0) mma_ss_lo<false>(d1, x_lo + off, a_lo + off, dhi, IDESC_TH);
-                    else mma_ss_lo<true>(d1, x_lo + off, a_lo + off, dhi, IDESC_TH);
+                    if (kk == 0) mma_ss_lo<false>(t_dst + hf * 64, s_lo + off, r_lo + off, dhi, IDESC_TH);
+                    else mma_ss_lo<true>(t_dst + hf * 64, s_lo + off, r_lo + off, dhi, IDESC_TH);
                 }
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
-                    if (kk == 0) mma_ss_lo<false>(d2, y_lo + off, b_lo + off, dhi, IDESC_TH);
-                    else mma_ss_lo<true>(d2, y_lo + off, b_lo + off, dhi, IDESC_TH);
-                }
-                mma_commit(&bars[L::B_TFULL + hf]);
+                mma_commit(&bars[L::B_TFULL + hf]);   // complete when both issuers' halves are
             };
             auto wait_stream = [&](int n) {
                 const int st = n % NST;
-                bool r = mbar_wait(&bars[B_AREADY + st], (n / NST) & 1, abort_flag, 24);
-                if (r) r = mbar_wait(&bars[L::B_BFULL + st], (n / NST) & 1, abort_flag, 25);
+                bool r = mbar_wait(&bars[(who == 0 ? B_AREADY : L::B_BFULL) + st], (n / NST) & 1, abort_flag, 24);
+                // the accumulator MMAs of issuer 1 (DKV) read A as well, those of issuer 0 (DKV) read Bc
+                if (r && DKV) r = mbar_wait(&bars[(who == 0 ? L::B_BFULL : B_AREADY) + st], (n / NST) & 1, abort_flag, 25);
                 tc_fence_after_sync();
                 return r;
             };
+            const bool has_acc = who == 0 || DKV;
             if (ok && n_it > 0) ok = wait_stream(0);
             if (ok && n_it > 0) {
                 issue_T(0, 0);
@@ -340,32 +347,30 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             }
             for (int n = 0; ok && n < n_it; ++n) {
                 const int st = n % NST;
-                // MN-major B operands of the accumulator MMAs: 16 streamed rows (2 KB) per K step
-                const uint32_t am_lo = desc_lo(smem_u32(sA + st * TILE), BOX_BYTES), bm_lo = desc_lo(smem_u32(sB + st * TILE), BOX_BYTES);
+                // MN-major B operand of this issuer's accumulator MMAs: 16 streamed rows (2 KB) per K step
+                const uint32_t m_lo = desc_lo(smem_u32(((who == 0) == DKV ? sB : sA) + st * TILE), BOX_BYTES);
+                const uint32_t acc_dst = tmem_base + (who == 0 ? ACC1 : ACC2);
                 const bool next = n + 1 < n_it;
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
-                    // accumulate this half: 4 K = 16 steps over its 64 streamed rows; the bf16 operands sit at
-                    // the start of the half's own columns
+                    // this half: 4 K = 16 steps over its 64 streamed rows; the bf16 operands sit at the start of
+                    // the half's own columns of T1 (issuer 0) or T2 (issuer 1)
                     ok = mbar_wait(&bars[L::B_PDS + hf], n & 1, abort_flag, 26);
                     if (!ok) break;
                     tc_fence_after_sync();
+                    if (has_acc) {
 #pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4) {
-                        const int kk = hf * 4 + k4;
-                        const uint32_t a_off = hf * 64 + k4 * 8;
-                        const uint32_t acc_on = (n > 0 || kk > 0) ? 1u : 0u;
-                        if (DKV) {
-                            // acc1 (dV) += P^T dO, acc2 (dK') += dS^T Q': dO and Q' are MN-major B operands
-                            mma_ts_lo(tmem_base + ACC1, tmem_base + T1 + a_off, bm_lo + kk * 128, dhi, IDESC_ACC, acc_on);
-                            mma_ts_lo(tmem_base + ACC2, tmem_base + T2 + a_off, am_lo + kk * 128, dhi, IDESC_ACC, acc_on);
-                        } else {
-                            // acc1 (dQ') += dS K'
-                            mma_ts_lo(tmem_base + ACC1, tmem_base + T1 + a_off, am_lo + kk * 128, dhi, IDESC_ACC, acc_on);
+                        for (int k4 = 0; k4 < 4; ++k4) {
+                            const int kk = hf * 4 + k4;
+                            mma_ts_lo(acc_dst, t_dst + hf * 64 + k4 * 8, m_lo + kk * 128, dhi, IDESC_ACC, (n > 0 || kk > 0) ? 1u : 0u);
                         }
                     }
-                    if (hf == 1) mma_commit(&bars[L::B_EMPTY + st]);   // the stage is free once both halves are consumed
-                    // the same half of the next streamed tile may overwrite T1/T2 right behind (in-order pipe)
+                    if (hf == 1) {
+                        // the stage is free once both issuers have consumed both halves
+                        if (has_acc) mma_commit(&bars[L::B_EMPTY + st]);
+                        else mbar_arrive(&bars[L::B_EMPTY + st]);   // DQ, issuer 1: its T2 MMAs of this stage were complete at TFULL
+                    }
+                    // the same half of the next streamed tile may overwrite T1/T2 right behind (in-order per issuer)
                     if (next) {
                         if (hf == 0) ok = wait_stream(n + 1);
                         if (!ok) break;
@@ -373,9 +378,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                     }
                 }
                 if (!ok) break;
-                if (!next) mma_commit(&bars[L::B_DONE]);
+                if (!next) {
+                    if (has_acc) mma_commit(&bars[L::B_DONE]);
+                    else mbar_arrive(&bars[L::B_DONE]);
+                }
             }
-            if (DKV && ROT_X && p.store_x) tma_store_wait_all();   // the tile must stay in place until it has been read
+            if (who == 0 && DKV && ROT_X && p.store_x) tma_store_wait_all();   // the tile must stay in place until it has been read
         }
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------ rotation warpgroup: X once, every A tile
