@@ -320,8 +320,25 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             const uint32_t s_lo = desc_lo(who == 0 ? xa : ya, 16);          // this issuer's stationary operand
             const uint32_t t_dst = tmem_base + (who == 0 ? T1 : T2);
             // T1 or T2, half hf of streamed tile n: rows [64 hf, 64 hf + 64) of A (or Bc) are the N index
+#ifndef AF_BWD_TFULL
+#define AF_BWD_TFULL 0
+#endif
+            constexpr bool kTFull = AF_BWD_TFULL != 0;   // T1/T2 as one N = 128 MMA group per tile instead of two N = 64 halves
             auto issue_T = [&](int n, int hf) {
                 const int st = n % NST;
+                if (kTFull) {
+                    if (hf == 0) return;   // issued once per tile, at the second half's turn
+                    const uint32_t r_lo = desc_lo(smem_u32((who == 0 ? sA : sB) + st * TILE), 16);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
+                        if (kk == 0) mma_ss_lo<false>(t_dst, s_lo + off, r_lo + off, dhi, IDESC_T);
+                        else mma_ss_lo<true>(t_dst, s_lo + off, r_lo + off, dhi, IDESC_T);
+                    }
+                    mma_commit(&bars[L::B_TFULL + 0]);
+                    mma_commit(&bars[L::B_TFULL + 1]);
+                    return;
+                }
                 const uint32_t r_lo = desc_lo(smem_u32((who == 0 ? sA : sB) + st * TILE) + hf * 64 * 128, 16);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
