@@ -322,10 +322,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    // Register budget: the softmax warpgroups hold a full row of 128 scores; the others need little.
+    // Register budget: the softmax warpgroups hold a full row of 128 scores; the others need little, but the
+    // MMA issuer must not spill (it is the most latency-sensitive thread of the CTA: at 64 registers it spilled
+    // and the kernel was 4 % slower), and the rotation warpgroup fits in 80.  80 + 80 + 2 x 176 = 512.
     constexpr int kSoftmaxRegs = NQ == 2 ? 176 : 232;
+    constexpr int kIssuerRegs = 80, kRotRegs = 80;
 
-    if (warp < 4) setmaxnreg_dec<64>();
+    if (warp < 4) setmaxnreg_dec<kIssuerRegs>();
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -460,7 +463,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------ rotation warpgroup (Section 4.1)
-        setmaxnreg_dec<96>();
+        setmaxnreg_dec<kRotRegs>();
         if (ROPE) {
             const int t = threadIdx.x - 128;
             auto run = [&](auto cp_tag) {
