@@ -8,8 +8,8 @@
 #include <string.h>
 
 #include "../../include/attnfuse.h"
-#include "bwd_kernel.cuh"
 #include "fwd_kernel.cuh"
+#include "bwd_kernel.cuh"
 #include "fwd2_kernel.cuh"
 #include "rope_kernels.cuh"
 

@@ -115,40 +115,60 @@ __device__ __forceinline__ void store_acc_rotated(uint32_t t_acc, float* stg, in
                                       __uint_as_float(v[e + 2]) * mul, __uint_as_float(v[e + 3]) * mul);
     }
     wg_sync();
-    constexpr int RPP = 256 / D;  // rows per pass (2 for D = 128, 4 for D = 64)
-    const int d = gtid % D, rsub = gtid / D;
+    // Second phase: thread (rsub, d4) writes the four columns 4 d4 .. 4 d4 + 3 of rows rsub, rsub + RPP, ...
+    // with 16-byte shared loads and coalesced 16-byte (fp32) or 8-byte (bf16) global stores.  The four
+    // frequencies' cos/sin come from the table once (first row, and the next one to get the step angle as
+    // a difference of angles) and then walk by the angle-addition recurrence: no table read in the loop.
+    constexpr int TPR = D / 4;        // threads per row
+    constexpr int RPP = 256 / TPR;    // rows per pass (8 for D = 128, 16 for D = 64)
+    const int d = (gtid % TPR) * 4, rsub = gtid / TPR;
     const int half = R >> 1;
-    const int fi = d < half ? d : d - half;
-    // This thread writes column d of rows rsub, rsub + RPP, ...: one frequency, positions RPP apart.  Its
-    // cos/sin come from the table once (first row, and the next one to get the step angle as a
-    // difference of angles) and then walk by the angle-addition recurrence: no table read in the loop.
-    float c = 1.f, sn = 0.f, cst = 1.f, sst = 0.f;
-    if (d < R) {
-        const int r0 = min(row0 + rsub, S - 1), r1 = min(row0 + rsub + RPP, S - 1);
-        const float2 t0 = __ldg(table + static_cast<size_t>(r0) * half + fi);
-        const float2 t1 = __ldg(table + static_cast<size_t>(r1) * half + fi);
-        c = t0.x;
-        sn = t0.y;
-        cst = fmaf(t1.x, t0.x, t1.y * t0.y);    // cos(a1 - a0)
-        sst = fmaf(t1.y, t0.x, -t1.x * t0.y);   // sin(a1 - a0)
-    }
+    const bool rot = d < R;           // R is a multiple of 8: the four columns are on one side of R and of R / 2
     const bool upper = d >= half;
-    const int partner = d < half ? d + half : d - half;
-#pragma unroll 4
+    const int partner = upper ? d - half : d + half;
+    float c[4] = {1.f, 1.f, 1.f, 1.f}, sn[4] = {0.f, 0.f, 0.f, 0.f}, cst[4] = {1.f, 1.f, 1.f, 1.f}, sst[4] = {0.f, 0.f, 0.f, 0.f};
+    if (rot) {
+        const int fi = upper ? d - half : d;
+        const int r0 = min(row0 + rsub, S - 1), r1 = min(row0 + rsub + RPP, S - 1);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float2 t0 = __ldg(table + static_cast<size_t>(r0) * half + fi + u);
+            const float2 t1 = __ldg(table + static_cast<size_t>(r1) * half + fi + u);
+            c[u] = t0.x;
+            sn[u] = upper ? -t0.y : t0.y;                 // transpose rotation: y c + other s below R/2, y c - other s above
+            cst[u] = fmaf(t1.x, t0.x, t1.y * t0.y);       // cos(a1 - a0)
+            sst[u] = fmaf(t1.y, t0.x, -t1.x * t0.y);      // sin(a1 - a0)
+            if (upper) sst[u] = -sst[u];                  // the sign rides along with sn
+        }
+    }
+#pragma unroll 2
     for (int r = rsub; r < 128; r += RPP) {
         if (row0 + r < S) {
-            float y = stg[r * STRIDE + d];
-            if (d < R) {
-                const float other = stg[r * STRIDE + partner];
-                y = upper ? fmaf(y, c, -other * sn) : fmaf(y, c, other * sn);   // transpose rotation
+            float4 y = *reinterpret_cast<const float4*>(stg + r * STRIDE + d);
+            if (rot) {
+                const float4 o = *reinterpret_cast<const float4*>(stg + r * STRIDE + partner);
+                y.x = fmaf(y.x, c[0], o.x * sn[0]);
+                y.y = fmaf(y.y, c[1], o.y * sn[1]);
+                y.z = fmaf(y.z, c[2], o.z * sn[2]);
+                y.w = fmaf(y.w, c[3], o.w * sn[3]);
             }
-            const size_t o = (out_row0 + r) * D + d;
-            if (out_f32) static_cast<float*>(out)[o] = y;
-            else static_cast<__nv_bfloat16*>(out)[o] = __float2bfloat16_rn(y);
+            const size_t oi = (out_row0 + r) * D + d;
+            if (out_f32) {
+                *reinterpret_cast<float4*>(static_cast<float*>(out) + oi) = y;
+            } else {
+                *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(out) + oi) =
+                    make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+            }
         }
-        const float nc = fmaf(c, cst, -sn * sst), ns = fmaf(sn, cst, c * sst);
-        c = nc;
-        sn = ns;
+        if (rot) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                // (c, sn) -> next row; with sn and sst negated together the recurrence keeps its form
+                const float nc = fmaf(c[u], cst[u], -sn[u] * sst[u]), ns = fmaf(sn[u], cst[u], c[u] * sst[u]);
+                c[u] = nc;
+                sn[u] = ns;
+            }
+        }
     }
     wg_sync();
 }
@@ -210,6 +230,17 @@ __device__ __forceinline__ void grad_pass32(uint32_t t1, uint32_t t2, int col0, 
 // both (K' once, every Q' tile) and, when the caller's workspace has room (p.store_x), writes its rotated
 // K' tile to that workspace through tm_s; the dQ role then streams those rows and rotates only its own
 // Q' tile, instead of rotating every K tile again for every query tile.
+// timeline stamps for tuning (compiled out unless AF_TRACE): CTA (0, 0), lane 0 of each warp
+#ifdef AF_TRACE
+#define AF_BSTAMP(role, it, ph)                                                                          \
+    do {                                                                                                 \
+        if (g_trace && blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && (it) < 64)       \
+            g_trace[((role) * 64 + (it)) * 8 + (ph)] = clock64();                                        \
+    } while (0)
+#else
+#define AF_BSTAMP(role, it, ph) do { } while (0)
+#endif
+
 template <int D, bool DKV, bool ROT_X, bool ROT_A>
 __global__ void __launch_bounds__(512, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_y,
@@ -267,6 +298,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    AF_BSTAMP(5, 0, 0);
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -357,7 +389,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 return r;
             };
             const bool has_acc = who == 0 || DKV;
+            AF_BSTAMP(who, 63, 0);   // stationary operand ready
             if (ok && n_it > 0) ok = wait_stream(0);
+            AF_BSTAMP(who, 63, 1);   // first streamed tile ready
             if (ok && n_it > 0) {
                 issue_T(0, 0);
                 issue_T(0, 1);
@@ -372,7 +406,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 for (int hf = 0; hf < 2; ++hf) {
                     // this half: 4 K = 16 steps over its 64 streamed rows; the bf16 operands sit at the start of
                     // the half's own columns of T1 (issuer 0) or T2 (issuer 1)
+                    AF_BSTAMP(who, n, 3 * hf);
                     ok = mbar_wait(&bars[L::B_PDS + hf], n & 1, abort_flag, 26);
+                    AF_BSTAMP(who, n, 3 * hf + 1);
                     if (!ok) break;
                     tc_fence_after_sync();
                     if (has_acc) {
@@ -393,6 +429,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                         if (!ok) break;
                         issue_T(n + 1, hf);
                     }
+                    AF_BSTAMP(who, n, 3 * hf + 2);
                 }
                 if (!ok) break;
                 if (!next) {
@@ -419,12 +456,15 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                     const int sg = n % NST, a0 = stream_row0(n);
                     const int run_pos = DKV ? n % per_head : n;
                     if (CP > 0 && (run_pos % kRotResync) == 0) rotate_prefetch(st, p.table, a0, p.S, p.R, t);
+                    AF_BSTAMP(4, n, 0);
                     if (!mbar_wait_warp(&bars[L::B_AFULL + sg], (n / NST) & 1, abort_flag, 28)) return;
+                    AF_BSTAMP(4, n, 1);
                     if (CP > 0) rotate_tile_fast(sA + sg * TILE, st, step, t);
                     else rotate_tile_smem(sA + sg * TILE, a0, p.S, p.R, p.table, t, 128);
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars[L::B_AROT + sg]);
+                    AF_BSTAMP(4, n, 2);
                 }
             };
             if (p.R == 128) run(std::integral_constant<int, 8>{});
@@ -501,7 +541,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             const float sb = DKV ? -my_slope2 : my_slope2;
             const float bias_base = sb * static_cast<float>(a0 - xrow);
             // this warpgroup's half of T1/T2; the barrier also publishes the statistics within the warpgroup
+            AF_BSTAMP(2 + hf, n, 0);
             ok = bar_all(mbar_wait(&bars[L::B_TFULL + hf], n & 1, abort_flag, 29), 1 + hf, 128);
+            AF_BSTAMP(2 + hf, n, 1);
             if (!ok) break;
             tc_fence_after_sync();
 #pragma unroll
@@ -517,13 +559,17 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                     else grad_pass32<DKV, false, false>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, my_l2, my_delta, mlo, mn);
                 }
             }
+            AF_BSTAMP(2 + hf, n, 2);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[L::B_PDS + hf]);
+            AF_BSTAMP(2 + hf, n, 3);
         }
         // epilogue: stage through shared memory (the stream stages are idle now), rotate back, store
+        AF_BSTAMP(2 + hf, 63, 0);
         if (ok && n_it > 0) ok = wg_all(mbar_wait(&bars[L::B_DONE], 0, abort_flag, 30));
+        AF_BSTAMP(2 + hf, 63, 1);   // accumulators complete
         if (ok && n_it > 0) {
             tc_fence_after_sync();
             float* stg = reinterpret_cast<float*>(sA);
@@ -539,6 +585,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
 
     tc_fence_before_sync();
     __syncthreads();
+    AF_BSTAMP(5, 0, 1);
     if (warp == 1) {
         __syncwarp();
         tmem_dealloc(tmem_base, TMEM_COLS);
