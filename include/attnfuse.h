@@ -104,15 +104,19 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
                             void* cuda_stream);
 
 /* ---- fused backward (Section 4.4) -------------------------------------------------------------------
- * Three kernels: row-reduced gradients delta = rowsum(dO * O); dK/dV accumulation per key tile;
- * dQ accumulation per query tile.  Probabilities are recomputed from lse; the rotation is recomputed
- * on chip and gradients w.r.t. rotated rows are rotated back in the epilogues.
+ * Row-reduced gradients delta = rowsum(dO * O); dK/dV accumulation per key tile; dQ accumulation per
+ * query tile.  Probabilities are recomputed from lse; the rotation is recomputed and gradients w.r.t.
+ * rotated rows are rotated back in the epilogues.
  * o, d_o: [B,Hq,S,D] bf16 contiguous; lse from the forward.
  * dq [B,Hq,S,D] (dq_dtype), dk, dv [B,Hkv,S,D] (dkv_dtype), contiguous; dk/dv sum over the group.
  * workspace: attnfuse_bwd_workspace_bytes(shape) bytes hold delta (4 bytes per query row, rounded up to
- * 256) followed by a cache of the rotated K (B*Hkv*S*D bf16) that the dK/dV kernel fills and the dQ
- * kernel reads, so K is rotated once per key tile instead of once per (query tile, key tile).  A smaller
- * workspace is accepted down to the delta part alone; the dQ kernel then rotates K on chip itself. */
+ * 256), a cache of the rotated K (B*Hkv*S*D bf16) and a cache of the rotated Q (B*Hq*S*D bf16), in this
+ * order.  With all three, K is rotated once by a RoPE pass, each Q tile once by the dQ kernel that owns it
+ * (which also writes it to the cache), and the dK/dV kernel runs last without rotating anything in its
+ * loop.  A smaller workspace is accepted: with delta + K cache the dK/dV kernel runs first, rotates K once
+ * per key tile and every Q tile it streams, and the dQ kernel streams the cached K; with delta alone both
+ * kernels rotate everything they touch on chip.  Results of the three set-ups agree up to the bf16
+ * rounding of a few rotated elements. */
 size_t    attnfuse_bwd_workspace_bytes(const af_shape* shape);
 af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, const void* v,
                        const void* o, const float* lse, const void* d_o,

@@ -172,12 +172,29 @@ af_status launch_bwd_variant(const CUtensorMap& tx, const CUtensorMap& ty, const
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
-// delta, then the dK/dV kernel, then the dQ kernel.  tkp: tensor map over the rotated-K cache in the
-// workspace, or nullptr when the workspace has no room for it (then the dQ kernel rotates K itself).
+// RoPE pass x [B, H, S, D] (strided) -> x_out (contiguous); R > 0.
+af_status launch_rope(const void* x_in, const af_strides& st, void* x_out, int B, int H, int S, int D, int R,
+                      const void* rope_table, int inverse, cudaStream_t stream) {
+    constexpr int HPT = 4;
+    const long long NH = static_cast<long long>(B) * H;
+    const int per_row = (R >> 4) + ((D - R) >> 3);
+    const long long items = static_cast<long long>(S) * per_row;
+    dim3 grid(static_cast<unsigned>((items + 255) / 256), static_cast<unsigned>((NH + HPT - 1) / HPT), 1);
+    if (grid.y > 65535) return AF_ERR_SHAPE;
+    rope_apply_kernel<HPT><<<grid, 256, 0, stream>>>(static_cast<const uint4*>(x_in), static_cast<uint4*>(x_out),
+                                                     static_cast<const float2*>(rope_table), static_cast<int>(NH), H, S,
+                                                     D, R, inverse ? -1.f : 1.f, st.b, st.h, st.s);
+    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+// delta, then the two gradient kernels.  tkp / tqp: tensor maps over the rotated-K and rotated-Q caches in
+// the workspace, or nullptr when the workspace has no room for them (see bwd_kernel.cuh for the three set-ups).
+// k / stkv / kcache: the caller's K, its strides and the K' cache, for the RoPE pass of the two-cache set-up.
 template <int D>
 af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                     const CUtensorMap& tdo, const CUtensorMap* tkp, const void* o, const void* d_o, BwdParams p,
-                     void* dq, int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, cudaStream_t stream) {
+                     const CUtensorMap& tdo, const CUtensorMap* tkp, const CUtensorMap* tqp, const void* k,
+                     const af_strides& stkv, void* kcache, const void* o, const void* d_o, BwdParams p, void* dq,
+                     int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, cudaStream_t stream) {
     const long long rows = static_cast<long long>(sh->B) * sh->Hq * sh->S;
     const long long threads = rows * (D / 8);
     bwd_delta_kernel<D><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
@@ -187,15 +204,22 @@ af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMa
     const unsigned tiles = static_cast<unsigned>((sh->S + 127) / 128);
     af_status st;
     const int only = env_int("AF_BWD_ONLY", 0);   // tuning aid: 1 = dK/dV kernel only, 2 = dQ kernel only
+    dim3 gkv(sh->B * sh->Hkv, tiles, 1), gq(sh->B * sh->Hq, tiles, 1);
+    if (p.R > 0 && tkp && tqp && only == 0) {
+        // both caches: K' by the RoPE pass, Q' by the dQ kernel, no on-chip rotation in the dK/dV loop
+        if ((st = launch_rope(k, stkv, kcache, sh->B, sh->Hkv, sh->S, D, p.R, p.table, 0, stream)) != AF_OK) return st;
+        p.out1 = dq; p.out2 = nullptr; p.out_f32 = dq_f32; p.store_x = 1;
+        if ((st = launch_bwd_variant<D, false, true, false>(tq, tdo, *tkp, tv, *tqp, p, gq, stream)) != AF_OK) return st;
+        p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32; p.store_x = 0;
+        return launch_bwd_variant<D, true, false, false>(*tkp, tv, *tqp, tdo, tk, p, gkv, stream);
+    }
     const bool cache = p.R > 0 && tkp != nullptr && only != 2;
     p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32; p.store_x = cache ? 1 : 0;
-    dim3 gkv(sh->B * sh->Hkv, tiles, 1);
     st = only == 2 ? AF_OK
          : p.R > 0 ? launch_bwd_variant<D, true, true, true>(tk, tv, tq, tdo, cache ? *tkp : tk, p, gkv, stream)
                    : launch_bwd_variant<D, true, false, false>(tk, tv, tq, tdo, tk, p, gkv, stream);
     if (st != AF_OK || only == 1) return st;
     p.out1 = dq; p.out2 = nullptr; p.out_f32 = dq_f32; p.store_x = 0;
-    dim3 gq(sh->B * sh->Hq, tiles, 1);
     if (p.R == 0) return launch_bwd_variant<D, false, false, false>(tq, tdo, tk, tv, tk, p, gq, stream);
     return cache ? launch_bwd_variant<D, false, true, false>(tq, tdo, *tkp, tv, tk, p, gq, stream)
                  : launch_bwd_variant<D, false, true, true>(tq, tdo, tk, tv, tk, p, gq, stream);
@@ -206,6 +230,9 @@ size_t bwd_delta_bytes(const af_shape* sh) {
 }
 size_t bwd_kcache_bytes(const af_shape* sh) {
     return static_cast<size_t>(sh->B) * sh->Hkv * sh->S * sh->D * 2;
+}
+size_t bwd_qcache_bytes(const af_shape* sh) {
+    return static_cast<size_t>(sh->B) * sh->Hq * sh->S * sh->D * 2;
 }
 
 }  // namespace
@@ -279,15 +306,9 @@ af_status attnfuse_rope(const af_shape* shape, int n_heads, const void* x_in, vo
             return AF_ERR_CUDA;
         return AF_OK;
     }
-    constexpr int HPT = 4;
-    const int per_row = (R >> 4) + ((D - R) >> 3);
-    const long long items = static_cast<long long>(shape->S) * per_row;
-    dim3 grid(static_cast<unsigned>((items + 255) / 256), static_cast<unsigned>((NH + HPT - 1) / HPT), 1);
-    if (grid.y > 65535) return AF_ERR_SHAPE;
-    rope_apply_kernel<HPT><<<grid, 256, 0, stream>>>(static_cast<const uint4*>(x_in), static_cast<uint4*>(x_out),
-                                                     static_cast<const float2*>(rope_table), static_cast<int>(NH),
-                                                     shape->S, D, R, inverse ? -1.f : 1.f);
-    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+    af_strides st;
+    st.b = static_cast<int64_t>(n_heads) * shape->S * D; st.h = static_cast<int64_t>(shape->S) * D; st.s = D;
+    return launch_rope(x_in, st, x_out, shape->B, n_heads, shape->S, D, R, rope_table, inverse, stream);
 }
 
 af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
@@ -372,7 +393,7 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
 
 size_t attnfuse_bwd_workspace_bytes(const af_shape* shape) {
     if (!shape) return 0;
-    return bwd_delta_bytes(shape) + bwd_kcache_bytes(shape);   // delta + rotated-K cache
+    return bwd_delta_bytes(shape) + bwd_kcache_bytes(shape) + bwd_qcache_bytes(shape);   // delta + rotated-K and -Q caches
 }
 
 af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,
@@ -413,20 +434,26 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
     p.delta = nullptr; p.out1 = nullptr; p.out2 = nullptr; p.out_f32 = 0; p.store_x = 0;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     float* delta = static_cast<float*>(workspace);
-    // rotated-K cache: used when there is a rotation and the workspace has room behind delta
-    CUtensorMap tkp;
-    const bool have_cache = p.R > 0 && workspace_bytes >= bwd_delta_bytes(shape) + bwd_kcache_bytes(shape);
-    if (have_cache) {
+    // rotated-K and rotated-Q caches: used when there is a rotation and the workspace has room behind delta
+    CUtensorMap tkp, tqp;
+    const size_t off_k = bwd_delta_bytes(shape), off_q = off_k + bwd_kcache_bytes(shape);
+    const bool have_k = p.R > 0 && workspace_bytes >= off_q;
+    const bool have_q = have_k && workspace_bytes >= off_q + bwd_qcache_bytes(shape);
+    void* kc = static_cast<uint8_t*>(workspace) + off_k;
+    if (have_k) {
         af_strides stk;
         resolve_strides(nullptr, shape->Hkv, shape->S, shape->D, &stk);
-        void* kc = static_cast<uint8_t*>(workspace) + bwd_delta_bytes(shape);
         if ((st = make_tmap(&tkp, kc, shape->B, shape->Hkv, shape->S, shape->D, stk, 128)) != AF_OK) return st;
     }
+    if (have_q) {
+        void* qc = static_cast<uint8_t*>(workspace) + off_q;
+        if ((st = make_tmap(&tqp, qc, shape->B, shape->Hq, shape->S, shape->D, stc, 128)) != AF_OK) return st;
+    }
     return shape->D == 128
-               ? launch_bwd<128>(shape, tq, tk, tv, tdo, have_cache ? &tkp : nullptr, o, d_o, p, dq, dq_dtype == AF_F32, dk,
-                                 dv, dkv_dtype == AF_F32, delta, stream)
-               : launch_bwd<64>(shape, tq, tk, tv, tdo, have_cache ? &tkp : nullptr, o, d_o, p, dq, dq_dtype == AF_F32, dk,
-                                dv, dkv_dtype == AF_F32, delta, stream);
+               ? launch_bwd<128>(shape, tq, tk, tv, tdo, have_k ? &tkp : nullptr, have_q ? &tqp : nullptr, k, stkv, kc, o,
+                                 d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, stream)
+               : launch_bwd<64>(shape, tq, tk, tv, tdo, have_k ? &tkp : nullptr, have_q ? &tqp : nullptr, k, stkv, kc, o,
+                                d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, stream);
 }
 
 }  // extern "C"

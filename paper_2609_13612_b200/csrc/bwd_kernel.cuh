@@ -226,10 +226,14 @@ __device__ __forceinline__ void grad_pass32(uint32_t t1, uint32_t t2, int col0, 
     }
 }
 
-// ROT_X / ROT_A: rotate the stationary tile X / every streamed tile A on chip.  The dK/dV role rotates
-// both (K' once, every Q' tile) and, when the caller's workspace has room (p.store_x), writes its rotated
-// K' tile to that workspace through tm_s; the dQ role then streams those rows and rotates only its own
-// Q' tile, instead of rotating every K tile again for every query tile.
+// ROT_X / ROT_A: rotate the stationary tile X / every streamed tile A on chip.  With p.store_x the rotated
+// stationary tile is also written to a cache in the caller's workspace through tm_s, so that the other
+// role can stream rotated rows instead of rotating every streamed tile again for every stationary tile.
+// Three set-ups, by the room the workspace has:
+//  - both caches: a RoPE pass writes K' first; the dQ role (ROT_X, stores Q') streams K'; the dK/dV role then
+//    runs without any on-chip rotation on (K', V) and streamed (Q', dO) - only its epilogue rotates dK' back;
+//  - K' cache only: the dK/dV role runs first (ROT_X, ROT_A, stores K'), the dQ role (ROT_X) streams K';
+//  - no cache: both roles rotate everything they touch.
 // timeline stamps for tuning (compiled out unless AF_TRACE): CTA (0, 0), lane 0 of each warp
 #ifdef AF_TRACE
 #define AF_BSTAMP(role, it, ph)                                                                          \
@@ -337,8 +341,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             bool ok = true;
             if (who == 0) {
                 ok = mbar_wait(&bars[B_XREADY], 0, abort_flag, 22);
-                if (ok && DKV && ROT_X && p.store_x) {
-                    // publish the rotated K' tile (rows past S are clipped by the tensor map)
+                if (ok && ROT_X && p.store_x) {
+                    // publish the rotated stationary tile (rows past S are clipped by the tensor map)
 #pragma unroll
                     for (int bx = 0; bx < NBOX; ++bx) tma_store_4d(&tm_s, sX + bx * BOX_BYTES, bx * BOX_COLS, x0, xh, b);
                     tma_store_commit();
@@ -437,7 +441,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                     else mbar_arrive(&bars[L::B_DONE]);
                 }
             }
-            if (who == 0 && DKV && ROT_X && p.store_x) tma_store_wait_all();   // the tile must stay in place until it has been read
+            if (who == 0 && ROT_X && p.store_x) tma_store_wait_all();   // the tile must stay in place until it has been read
         }
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------ rotation warpgroup: X once, every A tile

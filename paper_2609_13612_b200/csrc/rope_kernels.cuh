@@ -20,14 +20,14 @@ __global__ void rope_table_kernel(float2* __restrict__ table, int S, int R, doub
     table[idx] = make_float2(static_cast<float>(cs), static_cast<float>(sn));
 }
 
-// x [NH, S, D] -> y, rows rotated by their position.  One thread owns the 16-byte chunk pair
+// x [B, H, S, D] (element strides xb, xh, xs; D contiguous) -> y [B*H, S, D] contiguous, rows rotated by their position; NH = B * H.  One thread owns the 16-byte chunk pair
 // (columns 8cp.., R/2+8cp..) of sequence row s for HPT consecutive heads, so the table entry is
 // read once and reused; consecutive threads touch consecutive 16-byte chunks (coalesced).
 // Chunks past R are copied when y != x.  sgn = -1 applies the transpose rotation.
 template <int HPT>
 __global__ void __launch_bounds__(256)
-rope_apply_kernel(const uint4* x, uint4* y, const float2* __restrict__ table, int NH, int S,
-                  int D, int R, float sgn) {
+rope_apply_kernel(const uint4* x, uint4* y, const float2* __restrict__ table, int NH, int H, int S,
+                  int D, int R, float sgn, long long xb, long long xh, long long xs) {
     const int CP = R >> 4;                 // rotated chunk pairs per row
     const int PT = (D - R) >> 3;           // pass-through chunks per row
     const int per_row = CP + PT;
@@ -36,6 +36,10 @@ rope_apply_kernel(const uint4* x, uint4* y, const float2* __restrict__ table, in
     const int s = static_cast<int>(idx / per_row), c = static_cast<int>(idx - static_cast<long long>(s) * per_row);
     const int h0 = blockIdx.y * HPT;
     const int row_chunks = D >> 3;
+    // 16-byte chunk index of row s of flattened head h in the (possibly strided) input
+    auto in_base = [&](int h) {
+        return static_cast<size_t>(((h / H) * xb + (h % H) * xh + static_cast<long long>(s) * xs) >> 3);
+    };
     if (c < CP) {
         const float4* tb = reinterpret_cast<const float4*>(table + static_cast<size_t>(s) * (R >> 1) + c * 8);
         float4 t0 = __ldg(tb), t1 = __ldg(tb + 1), t2 = __ldg(tb + 2), t3 = __ldg(tb + 3);
@@ -45,7 +49,7 @@ rope_apply_kernel(const uint4* x, uint4* y, const float2* __restrict__ table, in
 #pragma unroll
         for (int u = 0; u < HPT; ++u) {
             if (h0 + u < NH) {
-                const size_t base = (static_cast<size_t>(h0 + u) * S + s) * row_chunks;
+                const size_t base = in_base(h0 + u);
                 lo[u] = __ldcs(x + base + c);
                 hi[u] = __ldcs(x + base + c + CP);
             }
@@ -68,7 +72,7 @@ rope_apply_kernel(const uint4* x, uint4* y, const float2* __restrict__ table, in
         for (int u = 0; u < HPT; ++u) {
             if (h0 + u < NH) {
                 const size_t base = (static_cast<size_t>(h0 + u) * S + s) * row_chunks;
-                y[base + cc] = __ldcs(x + base + cc);
+                y[base + cc] = __ldcs(x + in_base(h0 + u) + cc);
             }
         }
     }

@@ -114,24 +114,33 @@ def test_config5_training_shape_sampled_units():
         pu.assert_close("c5 dV", pu.to_np(dv[b:b + 1, hk:hk + 1]), wv)
 
 
-def test_backward_without_room_for_the_rotated_k_cache_gives_the_same_result():
-    """With a workspace that holds only delta the dQ kernel rotates K itself; both ways match the oracle."""
-    w = W("small_ws", 2, 4, 2, 515, 128, theta=5e5, backward=True, seed_id=224)
+def test_backward_workspace_tiers_give_the_same_result():
+    """Three set-ups by workspace size: delta + K' cache + Q' cache (nothing rotated in the dK/dV loop),
+    delta + K' cache (the dQ kernel streams cached K'), delta alone (both kernels rotate on chip).
+    All match the oracle and agree with one another up to a few bf16 roundings of rotated rows."""
+    w = W("ws_tiers", 2, 4, 2, 515, 128, theta=5e5, backward=True, seed_id=224)
     t = synth.draw_all(w)
     dev = {k: pu.to_dev(v) for k, v in t.items()}
     o, lse = pu.gpu_fwd(w, dev)
     rope, mask = pu.specs(w)
     table = af.rope_table(rope, w.S)
+    n_delta = (w.B * w.Hq * w.S * 4 + 255) // 256 * 256
+    n_k = w.B * w.Hkv * w.S * w.D * 2
     full = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale)
-    small_ws = torch.empty((w.B * w.Hq * w.S * 4 + 255) // 256 * 256, dtype=torch.uint8, device="cuda")
+    mid_ws = torch.empty(n_delta + n_k, dtype=torch.uint8, device="cuda")
+    mid = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale, workspace=mid_ws)
+    small_ws = torch.empty(n_delta, dtype=torch.uint8, device="cuda")
     small = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale, workspace=small_ws)
     torch.cuda.synchronize()
     assert af.device_status()[0] == 0
-    # dK and dV come from the same kernel either way; dQ sees K rotated with cos/sin walked over
-    # different runs of rows, so a few bf16 roundings of rotated K may differ by one ulp
-    assert torch.equal(full[1], small[1]) and torch.equal(full[2], small[2])
-    assert (full[0].float() - small[0].float()).abs().max().item() <= 1e-2
+    # with or without the K' cache dK and dV come from the same kernel on the same rotated rows
+    assert torch.equal(mid[1], small[1]) and torch.equal(mid[2], small[2])
+    # elsewhere cos/sin are walked over different runs of rows (or read from the table), so a few bf16
+    # roundings of rotated rows may differ by one ulp
+    for a, b in ((full, mid), (mid, small)):
+        for x, y in zip(a, b):
+            assert (x.float() - y.float()).abs().max().item() <= 1e-2
     want = oracle.run_workload(w, t, backward=True)
-    for res in (full, small):
+    for res in (full, mid, small):
         for name, got, ref in zip(("dQ", "dK", "dV"), res, want):
             pu.assert_close("%s %s" % (w.name, name), pu.to_np(got), ref)
