@@ -101,20 +101,7 @@ __device__ __forceinline__ void store_acc_rotated(uint32_t t_acc, float* stg, in
                                                   const float2* table, int row0, int S, void* out, size_t out_row0,
                                                   int out_f32) {
     constexpr int STRIDE = BwdSmem<D>::STG_STRIDE;
-    const int lane_row = gtid & 127, chalf = gtid >> 7;
-#pragma unroll 1
-    for (int c = 0; c < D / 64; ++c) {
-        const int col = chalf * (D / 2) + c * 32;
-        uint32_t v[32];
-        tmem_ld32(t_acc + col, v);
-        tmem_wait_ld();
-        float4* dst = reinterpret_cast<float4*>(stg + lane_row * STRIDE + col);
-#pragma unroll
-        for (int e = 0; e < 32; e += 4)
-            dst[e >> 2] = make_float4(__uint_as_float(v[e]) * mul, __uint_as_float(v[e + 1]) * mul,
-                                      __uint_as_float(v[e + 2]) * mul, __uint_as_float(v[e + 3]) * mul);
-    }
-    wg_sync();
+    // (set-up of the second phase first: its table reads are in flight while the first phase runs)
     // Second phase: thread (rsub, d4) writes the four columns 4 d4 .. 4 d4 + 3 of rows rsub, rsub + RPP, ...
     // with 16-byte shared loads and coalesced 16-byte (fp32) or 8-byte (bf16) global stores.  The four
     // frequencies' cos/sin come from the table once (first row, and the next one to get the step angle as
@@ -141,6 +128,20 @@ __device__ __forceinline__ void store_acc_rotated(uint32_t t_acc, float* stg, in
             if (upper) sst[u] = -sst[u];                  // the sign rides along with sn
         }
     }
+    const int lane_row = gtid & 127, chalf = gtid >> 7;
+#pragma unroll 1
+    for (int cc = 0; cc < D / 64; ++cc) {
+        const int col = chalf * (D / 2) + cc * 32;
+        uint32_t v[32];
+        tmem_ld32(t_acc + col, v);
+        tmem_wait_ld();
+        float4* dst = reinterpret_cast<float4*>(stg + lane_row * STRIDE + col);
+#pragma unroll
+        for (int e = 0; e < 32; e += 4)
+            dst[e >> 2] = make_float4(__uint_as_float(v[e]) * mul, __uint_as_float(v[e + 1]) * mul,
+                                      __uint_as_float(v[e + 2]) * mul, __uint_as_float(v[e + 3]) * mul);
+    }
+    wg_sync();
 #pragma unroll 2
     for (int r = rsub; r < 128; r += RPP) {
         if (row0 + r < S) {
