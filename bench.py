@@ -376,6 +376,34 @@ def main():
                        "bwd_pct_of_measured_peak": 100 * w5.bwd_flops() / (t_b / k_ex) / 1e9 / peaks["bf16_tflops"]}
         del s5
         torch.cuda.empty_cache()
+
+        def bwd_ms(wl):
+            r, m, tb = specs(wl)
+            ss = make_sets(wl, min(2, n_sets_for(wl)))
+            o_, l_ = af.fwd(ss[0]["q"], ss[0]["k"], ss[0]["v"], r, tb, m, wl.scale)
+            wsb = torch.empty(af.lib().attnfuse_bwd_workspace_bytes(
+                __import__("ctypes").byref(binding._Shape(wl.B, wl.Hq, wl.Hkv, wl.S, wl.D))), dtype=torch.uint8, device=dev)
+            t, _, _ = timed(lambda i: af.bwd(ss[i % len(ss)]["q"], ss[i % len(ss)]["k"], ss[i % len(ss)]["v"], o_, l_,
+                                             ss[i % len(ss)]["do"], r, tb, m, wl.scale, workspace=wsb), k_ex, w_ex)
+            return t / k_ex
+
+        # the single-GPU geometry of the paper's tables (Section 5: B = 4, 12 heads, D = 64, N = 4096), RoPE + causal
+        wg = synth.Workload("gpt2_small_geometry_d64", 4, 12, 12, 4096, 64, theta=1.0e4, backward=True, seed_id=51)
+        ms_f, ss = fwd_ms(wg, True)
+        ms_s, _ = fwd_ms(wg, False, ss)
+        del ss
+        torch.cuda.empty_cache()
+        ms_b = bwd_ms(wg)
+        ex[wg.name] = {"fused_fwd_ms": ms_f, "fused_fwd_tflops": wg.fwd_flops() / ms_f / 1e9,
+                       "separate_rope_fwd_ms": ms_s, "fused_over_separate_speedup": ms_s / ms_f,
+                       "bwd_ms": ms_b, "bwd_tflops": wg.bwd_flops() / ms_b / 1e9}
+        # the composed variant (window + ALiBi) through the backward, on config 3's shape
+        c3 = synth.CONFIGS[2]
+        wc = synth.Workload("c3_composed_backward", c3.B, c3.Hq, c3.Hkv, c3.S, c3.D, theta=c3.theta, window=c3.window,
+                            alibi=True, backward=True, seed_id=52)
+        ms_b = bwd_ms(wc)
+        ex[wc.name] = {"bwd_ms": ms_b, "bwd_tflops": wc.bwd_flops() / ms_b / 1e9}
+        torch.cuda.empty_cache()
         # Rotation Calculus sweep (Section 5.3): fused vs separate RoPE at constant B*S = 32768 tokens
         sweep = []
         for S in (512, 1024, 2048, 4096, 8192, 16384, 32768):

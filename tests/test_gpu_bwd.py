@@ -144,3 +144,62 @@ def test_backward_workspace_tiers_give_the_same_result():
     for res in (full, mid, small):
         for name, got, ref in zip(("dQ", "dK", "dV"), res, want):
             pu.assert_close("%s %s" % (w.name, name), pu.to_np(got), ref)
+
+
+def _check_units(w, units, t, o, lse, grads, tag):
+    """Oracle forward + backward on whole (batch, kv head) units of a larger workload."""
+    dq, dk, dv = grads
+    g = w.group
+    slopes = w.alibi_slopes()
+    for b, hk in units:
+        hs = slice(hk * g, (hk + 1) * g)
+        kw = dict(theta=w.theta, rotary_dim=w.R, pos_offset=w.pos_offset, causal=w.causal, window=w.window,
+                  slopes=None if slopes is None else slopes[hs], scale=w.scale)
+        q, k, v, do = t["q"][b:b + 1, hs], t["k"][b:b + 1, hk:hk + 1], t["v"][b:b + 1, hk:hk + 1], t["do"][b:b + 1, hs]
+        want_o, want_l = oracle.fwd(q, k, v, **kw)
+        pu.assert_close(tag + " O", pu.to_np(o[b:b + 1, hs]), want_o)
+        assert np.abs(pu.to_np(lse[b:b + 1, hs]) - want_l).max() <= pu.LSE_TOL
+        wq, wk, wv = oracle.bwd(q, k, v, do, **kw)
+        pu.assert_close(tag + " dQ", pu.to_np(dq[b:b + 1, hs]), wq)
+        pu.assert_close(tag + " dK", pu.to_np(dk[b:b + 1, hk:hk + 1]), wk)
+        pu.assert_close(tag + " dV", pu.to_np(dv[b:b + 1, hk:hk + 1]), wv)
+
+
+def test_gpt2_small_geometry_d64_forward_and_backward_sampled_units():
+    """The geometry of Section 5's single-GPU tables (B = 4, 12 heads, D = 64), RoPE + causal, at N = 4096."""
+    w = W("gpt2_small_d64", 4, 12, 12, 4096, 64, theta=1e4, backward=True, seed_id=230)
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    o, lse = pu.gpu_fwd(w, dev)
+    grads = pu.gpu_bwd(w, dev, o, lse)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    _check_units(w, ((0, 0), (3, 11)), t, o, lse, grads, "gpt2-small")
+
+
+def test_composed_window_alibi_backward_sampled_units():
+    """Config 3's composed variant (RoPE + causal + window 1024 + ALiBi) through the backward at S = 8192:
+    steep and shallow slopes, both kept-interval edges of the window in many tiles.  With the steepest slope a
+    row attends to about three keys, nothing averages out and |dQ| reaches 8: the gradient is taken in fp32,
+    since bf16 output rounding alone (half an ulp is 0.016 in [4, 8)) would use up the 2e-2 bound."""
+    c3 = synth.CONFIGS[2]
+    w = W("c3_bwd", 1, c3.Hq, c3.Hkv, c3.S, c3.D, theta=c3.theta, window=c3.window, alibi=True, backward=True, seed_id=231)
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    o, lse = pu.gpu_fwd(w, dev)
+    grads = pu.gpu_bwd(w, dev, o, lse, dq_dtype=torch.float32)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    _check_units(w, ((0, 0), (0, w.Hkv - 1)), t, o, lse, grads, "c3 backward")
+
+
+def test_partial_rotary_at_scale_sampled_units():
+    """Rotary dimension 64 of D = 128 (the rest of each row passes through) with GQA at S = 2048."""
+    w = W("partial_rotary_2k", 2, 8, 2, 2048, 128, theta=5e5, rotary_dim=64, backward=True, seed_id=232)
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    o, lse = pu.gpu_fwd(w, dev)
+    grads = pu.gpu_bwd(w, dev, o, lse)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    _check_units(w, ((1, 1),), t, o, lse, grads, "partial rotary")
