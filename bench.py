@@ -159,7 +159,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--extras", type=int, default=1, help="also time configs 3-5, the separate-RoPE arm and the sweep")
     ap.add_argument("--cpu-baseline", type=int, default=1)
-    ap.add_argument("--profile", default="", choices=["", "fwd", "bwd", "rope"],
+    ap.add_argument("--profile", default="", choices=["", "fwd", "bwd", "rope", "decode"],
                     help="run only a few launches of one path (for ncu captures) and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -239,6 +239,17 @@ def main():
             total_ms = float(tt.item())
         return total_ms, per, wall_ms
 
+    if args.profile == "decode":
+        # Flash Decoding on the Llama-3-70B geometry of the paper's decode table (64 q / 8 kv heads, 32768 keys)
+        gq = torch.Generator(device=dev).manual_seed(7)
+        qd = torch.randn(1, 64, 128, device=dev, generator=gq).to(torch.bfloat16)
+        kc = [torch.randn(1, 8, 32768, 128, device=dev, generator=gq).to(torch.bfloat16) for _ in range(3)]
+        vc = [torch.randn(1, 8, 32768, 128, device=dev, generator=gq).to(torch.bfloat16) for _ in range(3)]
+        for i in range(6):
+            af.decode(qd, kc[i % 3], vc[i % 3], af.MaskSpec(True, -1, None), 128 ** -0.5)
+        torch.cuda.synchronize()
+        print(json.dumps({"profile": "decode", "workload": "llama3_70b_decode_32768", "device_status": af.device_status()[0]}))
+        return
     if args.profile:
         # a handful of launches of one path on its configuration, nothing else: the target of ncu captures
         wl = {"fwd": synth.CONFIGS[1], "bwd": synth.CONFIGS[4], "rope": synth.CONFIGS[3]}[args.profile]
@@ -404,6 +415,42 @@ def main():
         ms_b = bwd_ms(wc)
         ex[wc.name] = {"bwd_ms": ms_b, "bwd_tflops": wc.bwd_flops() / ms_b / 1e9}
         torch.cuda.empty_cache()
+        # Flash Decoding (Section 4.5, the paper's decode table): query length 1, D = 128, B = 1.  HBM-bound: the
+        # algorithmic bytes are the K and V caches, read once.  Caches rotate over sets larger than L2 in total.
+        # Timed twice: as a replayed CUDA graph (device time per call) and through the C-ABI call from the host.
+        dec = []
+        for name, Hq_, Hkv_, N_, paper_ms in (("llama3_8b", 32, 8, 4096, 0.034), ("llama3_70b", 64, 8, 32768, 0.184),
+                                              ("mistral_7b", 32, 8, 16384, 0.072)):
+            nbytes = 2 * Hkv_ * N_ * 128 * 2
+            nsets = max(2, int(300e6 // nbytes) + 1)
+            gq = torch.Generator(device=dev).manual_seed(7)
+            qd = torch.randn(1, Hq_, 128, device=dev, generator=gq).to(torch.bfloat16)
+            kcs = [torch.randn(1, Hkv_, N_, 128, device=dev, generator=gq).to(torch.bfloat16) for _ in range(nsets)]
+            vcs = [torch.randn(1, Hkv_, N_, 128, device=dev, generator=gq).to(torch.bfloat16) for _ in range(nsets)]
+            md = af.MaskSpec(True, -1, None)
+            od = torch.empty(1, Hq_, 128, device=dev, dtype=torch.bfloat16)
+            ld = torch.empty(1, Hq_, device=dev, dtype=torch.float32)
+            shp = binding._Shape(1, Hq_, Hkv_, N_, 128)
+            nsp = af.lib().attnfuse_decode_splits(__import__("ctypes").byref(shp))
+            wsd = torch.empty(af.lib().attnfuse_decode_workspace_bytes(__import__("ctypes").byref(shp), nsp),
+                              dtype=torch.uint8, device=dev)
+            call = lambda i: af.decode(qd, kcs[i % nsets], vcs[i % nsets], md, 128 ** -0.5, n_splits=nsp, out=od, lse=ld,
+                                       workspace=wsd)
+            t_host, _, _ = timed(call, 2 * k_ex, w_ex)
+            side = torch.cuda.Stream(device=dev)
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(gr, stream=side):
+                    for i in range(nsets):
+                        call(i)
+            t_gr, _, _ = timed(lambda i: gr.replay(), k_ex, w_ex)
+            us = t_gr / k_ex / nsets * 1e3
+            dec.append({"geometry": name, "Hq": Hq_, "Hkv": Hkv_, "cache": N_, "n_splits": nsp, "kv_bytes": nbytes,
+                        "graph_replay_us": us, "GB/s": nbytes / us / 1e3, "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"],
+                        "c_abi_call_from_host_us": t_host / (2 * k_ex) * 1e3, "paper_ms_other_hardware": paper_ms})
+            del kcs, vcs
+            torch.cuda.empty_cache()
+        ex["flash_decoding"] = dec
         # Rotation Calculus sweep (Section 5.3): fused vs separate RoPE at constant B*S = 32768 tokens
         sweep = []
         for S in (512, 1024, 2048, 4096, 8192, 16384, 32768):

@@ -103,6 +103,25 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
                             void* o_host, float* lse_host, void* staging, size_t staging_bytes,
                             void* cuda_stream);
 
+/* ---- Flash Decoding (Section 4.5; Table "Flash Decoding") ---------------------------------------------
+ * One query position per head (the last one, N - 1) against a KV cache of N = shape->S keys:
+ *   o[b,h,:] = softmax_j( c * <q[b,h], k[b,h/g,j]> + m_h (j - (N - 1)) ) v[b,h/g,j],  j kept iff j >= N - 1 - W.
+ * Phase 1 splits the cache over n_splits CTAs per (batch, kv head); each computes a partial (max, sum,
+ * accumulator) for the g query heads of its kv head (packed as rows of one MMA tile, K and V read once);
+ * phase 2 merges the partials with a log-sum-exp.  No rotation is applied: q and the cached keys are used
+ * as they are (a cache holds rotated keys; rotate q with attnfuse_rope).  mask->causal is ignored (every
+ * cached key precedes the query); window and ALiBi slopes apply as in attnfuse_fwd.
+ * q, o: [B,Hq,D] bf16 contiguous (device); k, v: [B,Hkv,N,D] bf16 with strides skv (NULL = contiguous; the
+ * rows need 16-byte alignment and strides that are multiples of 8 elements); lse (nullable): [B,Hq] fp32.
+ * gqa_group <= 16; D in {64, 128}.  n_splits <= 0: attnfuse_decode_splits(shape) (about two CTAs per SM).
+ * workspace: attnfuse_decode_workspace_bytes(shape, n_splits) device bytes for the partials. */
+int       attnfuse_decode_splits(const af_shape* shape);
+size_t    attnfuse_decode_workspace_bytes(const af_shape* shape, int n_splits);
+af_status attnfuse_decode(const af_shape* shape, const void* q, const void* k, const void* v,
+                          const af_strides* skv, const af_mask* mask, int gqa_group, float softmax_scale,
+                          void* o, float* lse, int n_splits,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* ---- fused backward (Section 4.4) -------------------------------------------------------------------
  * Row-reduced gradients delta = rowsum(dO * O); dK/dV accumulation per key tile; dQ accumulation per
  * query tile.  Probabilities are recomputed from lse; the rotation is recomputed and gradients w.r.t.

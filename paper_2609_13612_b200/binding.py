@@ -86,6 +86,12 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_bwd.restype = i
         L.attnfuse_bwd.argtypes = [P(_Shape), vp, vp, vp, vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp,
                                    P(_Mask), i, f, vp, i, vp, vp, i, vp, sz, vp]
+        L.attnfuse_decode_splits.restype = i
+        L.attnfuse_decode_splits.argtypes = [P(_Shape)]
+        L.attnfuse_decode_workspace_bytes.restype = sz
+        L.attnfuse_decode_workspace_bytes.argtypes = [P(_Shape), i]
+        L.attnfuse_decode.restype = i
+        L.attnfuse_decode.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Mask), i, f, vp, vp, i, vp, sz, vp]
         L.attnfuse_bwd_static.restype = i
         L.attnfuse_bwd_static.argtypes = [P(_Shape), vp, vp, vp, vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp,
                                           P(_Mask), i, f, vp, i, vp, vp, i, vp]
@@ -238,6 +244,35 @@ def bwd(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softma
 
 
 BWD_STATIC_MAX_ROWS = 1 << 20
+
+
+def decode(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, mask: MaskSpec, softmax_scale: float,
+           n_splits: int = 0, out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+           workspace: Optional[torch.Tensor] = None, want_lse: bool = True):
+    """Flash Decoding: q [B,Hq,D] (one position per head, the last one) against the cache k/v [B,Hkv,N,D].
+    Returns (o [B,Hq,D] bf16, lse [B,Hq])."""
+    _need_cuda(q, k, v, out, lse, workspace)
+    assert q.dtype == k.dtype == v.dtype == torch.bfloat16 and q.is_contiguous()
+    B, Hq, D = q.shape
+    Hkv, N = k.shape[1], k.shape[2]
+    assert k.shape == v.shape == (B, Hkv, N, D) and k.stride() == v.stride()
+    if out is None:
+        out = torch.empty((B, Hq, D), dtype=torch.bfloat16, device=q.device)
+    if lse is None and want_lse:
+        lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device)
+    sh = _Shape(B, Hq, Hkv, N, D)
+    if n_splits <= 0:
+        n_splits = lib().attnfuse_decode_splits(ctypes.byref(sh))
+    n_ws = lib().attnfuse_decode_workspace_bytes(ctypes.byref(sh), n_splits)
+    if workspace is None:
+        workspace = torch.empty(n_ws, dtype=torch.uint8, device=q.device)
+    skv = _strides(k)
+    m = _mask_struct(mask)
+    _check(lib().attnfuse_decode(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), ctypes.byref(skv),
+                                 ctypes.byref(m), Hq // Hkv, float(softmax_scale), out.data_ptr(),
+                                 lse.data_ptr() if lse is not None else None, int(n_splits), workspace.data_ptr(),
+                                 workspace.numel() * workspace.element_size(), _stream()))
+    return out, lse
 
 
 def bwd_static(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softmax_scale: float,

@@ -10,6 +10,7 @@
 #include "../../include/attnfuse.h"
 #include "fwd_kernel.cuh"
 #include "bwd_kernel.cuh"
+#include "decode_kernels.cuh"
 #include "fwd2_kernel.cuh"
 #include "rope_kernels.cuh"
 
@@ -389,6 +390,79 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
     if (lse_host && cudaMemcpyAsync(lse_host, dl, ln, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
         return AF_ERR_CUDA;
     return AF_OK;
+}
+
+int attnfuse_decode_splits(const af_shape* shape) {
+    if (!shape || shape->B < 1 || shape->Hkv < 1 || shape->S < 1) return 0;
+    // one CTA per SM fits (its stages take most of the shared memory): as many splits as give at most one
+    // CTA per SM (148 SMs) in a single wave, at least 128 keys (one tile per warp) per split
+    const int ctas_per_split = shape->B * shape->Hkv;
+    const int want = 148 / ctas_per_split;
+    const int most = (shape->S + 127) / 128;
+    return want < 1 ? 1 : (want > most ? most : want);
+}
+
+size_t attnfuse_decode_workspace_bytes(const af_shape* shape, int n_splits) {
+    if (!shape) return 0;
+    if (n_splits <= 0) n_splits = attnfuse_decode_splits(shape);
+    return static_cast<size_t>(shape->B) * shape->Hq * n_splits * (shape->D + 2) * sizeof(float);
+}
+
+af_status attnfuse_decode(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* skv,
+                          const af_mask* mask, int gqa_group, float softmax_scale, void* o, float* lse, int n_splits,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!shape || !mask || !q || !k || !v || !o || !workspace) return AF_ERR_NULL;
+    if (shape->B < 1 || shape->Hq < 1 || shape->Hkv < 1 || shape->S < 1) return AF_ERR_SHAPE;
+    if (shape->D != 64 && shape->D != 128) return AF_ERR_SHAPE;
+    if (gqa_group < 1 || gqa_group > 16 || shape->Hkv * gqa_group != shape->Hq) return AF_ERR_SHAPE;
+    if (static_cast<long long>(shape->B) * shape->Hkv > 65535) return AF_ERR_SHAPE;
+    if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return AF_ERR_SPEC;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(workspace)) return AF_ERR_ALIGN;
+    if (n_splits <= 0) n_splits = attnfuse_decode_splits(shape);
+    if (n_splits > (shape->S + 127) / 128) n_splits = (shape->S + 127) / 128;
+    if (n_splits > kCombineMaxSplits) n_splits = kCombineMaxSplits;
+    if (workspace_bytes < attnfuse_decode_workspace_bytes(shape, n_splits)) return AF_ERR_WORKSPACE;
+    af_status st;
+    af_strides stkv;
+    if ((st = resolve_strides(skv, shape->Hkv, shape->S, shape->D, &stkv)) != AF_OK) return st;
+    if ((st = check_arch()) != AF_OK) return st;
+    CUtensorMap tk, tv;
+    if ((st = make_tmap(&tk, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, kDecTile)) != AF_OK) return st;
+    if ((st = make_tmap(&tv, v, shape->B, shape->Hkv, shape->S, shape->D, stkv, kDecTile)) != AF_OK) return st;
+    DecodeParams p;
+    p.B = shape->B; p.Hq = shape->Hq; p.Hkv = shape->Hkv; p.N = shape->S; p.group = gqa_group;
+    p.window = mask->window < 0 ? -1 : mask->window;
+    p.scale_log2 = softmax_scale * 1.4426950408889634f;
+    p.slopes = mask->alibi_slopes;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.n_splits = n_splits;
+    p.part_o = static_cast<float*>(workspace);
+    p.part_ml = p.part_o + static_cast<size_t>(shape->B) * shape->Hq * n_splits * shape->D;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    dim3 grid(n_splits, shape->B * shape->Hkv, 1);
+    if (shape->D == 128) {
+        static bool configured = false;
+        if (!configured) {
+            if (cudaFuncSetAttribute(decode_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     DecodeSmem<128>::BYTES) != cudaSuccess)
+                return AF_ERR_CUDA;
+            configured = true;
+        }
+        decode_split_kernel<128><<<grid, kDecWarps * 32, DecodeSmem<128>::BYTES, stream>>>(tk, tv, p);
+    } else {
+        static bool configured = false;
+        if (!configured) {
+            if (cudaFuncSetAttribute(decode_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     DecodeSmem<64>::BYTES) != cudaSuccess)
+                return AF_ERR_CUDA;
+            configured = true;
+        }
+        decode_split_kernel<64><<<grid, kDecWarps * 32, DecodeSmem<64>::BYTES, stream>>>(tk, tv, p);
+    }
+    if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
+    decode_combine_kernel<<<shape->B * shape->Hq, kCombineThreads, 0, stream>>>(p.part_o, p.part_ml, n_splits, shape->D,
+                                                                         static_cast<__nv_bfloat16*>(o), lse);
+    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
 size_t attnfuse_bwd_workspace_bytes(const af_shape* shape) {
