@@ -31,6 +31,11 @@ def _load():
         lib.af_oracle_fwd.restype = None
         lib.af_oracle_bwd.argtypes = [dp, dp, dp, dp, i, i, i, i, i, d, i, i, i, i, dp, d, dp, dp, dp]
         lib.af_oracle_bwd.restype = None
+        bp = ctypes.POINTER(ctypes.c_ubyte)
+        lib.af_oracle_fwd_blocks.argtypes = [dp, dp, dp, i, i, i, i, i, d, i, i, i, i, dp, d, bp, i, ip, i, dp, dp]
+        lib.af_oracle_fwd_blocks.restype = None
+        lib.af_oracle_bwd_blocks.argtypes = [dp, dp, dp, dp, i, i, i, i, i, d, i, i, i, i, dp, d, bp, i, dp, dp, dp]
+        lib.af_oracle_bwd_blocks.restype = None
         _lib = lib
     return _lib
 
@@ -63,11 +68,22 @@ def _check(q, k, v):
     return B, Hq, Hkv, S, D
 
 
+def _blocks(blocks, block_size, S):
+    """Active-block matrix [nb, nb] (Section 4.6) as contiguous bytes, or None."""
+    if blocks is None:
+        return None, None
+    nb = (S + block_size - 1) // block_size
+    a = np.ascontiguousarray(np.asarray(blocks) != 0, dtype=np.uint8)
+    assert a.shape == (nb, nb) and block_size > 0
+    return a, a.ctypes.data_as(ctypes.POINTER(ctypes.c_ubyte))
+
+
 def fwd(q, k, v, *, theta: float = 10000.0, rotary_dim: int = 0, pos_offset: int = 0,
         causal: bool = True, window: int = -1, slopes=None, scale: Optional[float] = None,
-        rows: Optional[Sequence[int]] = None):
+        rows: Optional[Sequence[int]] = None, blocks=None, block_size: int = 128):
     """O and L = m + ln(l) of the composed variant.  `rows`: optional subset of query
-    rows (same for every head); then O is [B,Hq,len(rows),D]."""
+    rows (same for every head); then O is [B,Hq,len(rows),D].  `blocks`: optional [nb, nb] matrix of
+    active blocks (Section 4.6): pairs in inactive blocks are dropped on top of the element mask."""
     q, k, v = _f64(q), _f64(k), _f64(v)
     B, Hq, Hkv, S, D = _check(q, k, v)
     scale = float(scale) if scale is not None else 1.0 / np.sqrt(D)
@@ -82,14 +98,16 @@ def fwd(q, k, v, *, theta: float = 10000.0, rotary_dim: int = 0, pos_offset: int
         nr, rp = len(ra), ra.ctypes.data_as(ctypes.POINTER(ctypes.c_int))
     o = np.empty((B, Hq, nr, D), dtype=np.float64)
     lse = np.empty((B, Hq, nr), dtype=np.float64)
-    _load().af_oracle_fwd(_p(q), _p(k), _p(v), B, Hq, Hkv, S, D, float(theta), int(rotary_dim),
-                          int(pos_offset), int(bool(causal)), int(window), _p(sl), scale,
-                          rp, nr, _p(o), _p(lse))
+    ba, bptr = _blocks(blocks, block_size, S)
+    _load().af_oracle_fwd_blocks(_p(q), _p(k), _p(v), B, Hq, Hkv, S, D, float(theta), int(rotary_dim),
+                                 int(pos_offset), int(bool(causal)), int(window), _p(sl), scale,
+                                 bptr, int(block_size), rp, nr, _p(o), _p(lse))
     return o, lse
 
 
 def bwd(q, k, v, d_o, *, theta: float = 10000.0, rotary_dim: int = 0, pos_offset: int = 0,
-        causal: bool = True, window: int = -1, slopes=None, scale: Optional[float] = None):
+        causal: bool = True, window: int = -1, slopes=None, scale: Optional[float] = None,
+        blocks=None, block_size: int = 128):
     """dQ, dK, dV for upstream dO (Section 4.4 algebra, rotation transposed back)."""
     q, k, v, d_o = _f64(q), _f64(k), _f64(v), _f64(d_o)
     B, Hq, Hkv, S, D = _check(q, k, v)
@@ -99,9 +117,10 @@ def bwd(q, k, v, d_o, *, theta: float = 10000.0, rotary_dim: int = 0, pos_offset
     dq = np.empty_like(q)
     dk = np.empty_like(k)
     dv = np.empty_like(v)
-    _load().af_oracle_bwd(_p(q), _p(k), _p(v), _p(d_o), B, Hq, Hkv, S, D, float(theta), int(rotary_dim),
-                          int(pos_offset), int(bool(causal)), int(window), _p(sl), scale,
-                          _p(dq), _p(dk), _p(dv))
+    ba, bptr = _blocks(blocks, block_size, S)
+    _load().af_oracle_bwd_blocks(_p(q), _p(k), _p(v), _p(d_o), B, Hq, Hkv, S, D, float(theta), int(rotary_dim),
+                                 int(pos_offset), int(bool(causal)), int(window), _p(sl), scale,
+                                 bptr, int(block_size), _p(dq), _p(dk), _p(dv))
     return dq, dk, dv
 
 

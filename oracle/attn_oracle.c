@@ -16,6 +16,10 @@
  *  - Sliding window with causal: keep 0 <= i-j <= W (W+1 keys); without causal |i-j| <= W.
  *  - ALiBi: slope_h * (j - i) added after the softmax scale is applied.
  *  - Saved statistic (Section 4.4): L_i = m_i + ln(l_i), natural log.
+ *  - Block-sparse attention (Section 4.6): the active-block lists only restrict the kept set: a pair
+ *    (i, j) is kept iff the element mask keeps it AND block (i / bs, j / bs) is active.  Here the lists
+ *    arrive as a dense nb x nb byte matrix (nb = ceil(S / bs)); a row with no kept pair gives O = 0,
+ *    L = -inf and zero gradients.
  *  - Backward (Section 4.4, FlashAttention-2 algebra) with the chain rule through the
  *    rotation: gradients w.r.t. rotated rows are rotated back by the transpose.
  */
@@ -50,8 +54,12 @@ void af_oracle_rope(const double* x, double* y, int B, int H, int S, int D,
     }
 }
 
-static int kept(int i, int j, int causal, int window)
+/* Section 4.6: active-block matrix (NULL = every block active). */
+typedef struct { const unsigned char* active; int bs, nb; } block_mask;
+
+static int kept(int i, int j, int causal, int window, const block_mask* bm)
 {
+    if (bm && bm->active && !bm->active[(long)(i / bm->bs) * bm->nb + j / bm->bs]) return 0;
     if (causal && j > i) return 0;
     if (window >= 0) {
         int d = i - j;
@@ -66,12 +74,15 @@ static int kept(int i, int j, int causal, int window)
  * Otherwise only the n_rows listed query rows (same list for every head):
  * o is [B,Hq,n_rows,D], lse [B,Hq,n_rows].  slopes: Hq doubles or NULL.
  */
-void af_oracle_fwd(const double* q, const double* k, const double* v,
-                   int B, int Hq, int Hkv, int S, int D,
-                   double theta, int R, int p0, int causal, int window,
-                   const double* slopes, double scale,
-                   const int* rows, int n_rows, double* o, double* lse)
+void af_oracle_fwd_blocks(const double* q, const double* k, const double* v,
+                          int B, int Hq, int Hkv, int S, int D,
+                          double theta, int R, int p0, int causal, int window,
+                          const double* slopes, double scale,
+                          const unsigned char* blocks, int block_size,
+                          const int* rows, int n_rows, double* o, double* lse)
 {
+    block_mask bmv = { blocks, block_size, block_size > 0 ? (S + block_size - 1) / block_size : 0 };
+    const block_mask* bm = blocks ? &bmv : NULL;
     int g = Hq / Hkv;
     int nr = rows ? n_rows : S;
 #pragma omp parallel for schedule(dynamic, 1)
@@ -89,7 +100,7 @@ void af_oracle_fwd(const double* q, const double* k, const double* v,
             rope_row(qh + (long)i * D, qr, D, R, theta, (long)p0 + i, 1);
             double m = -INFINITY;
             for (int j = 0; j < S; ++j) {
-                if (!kept(i, j, causal, window)) { sc[j] = -INFINITY; continue; }
+                if (!kept(i, j, causal, window, bm)) { sc[j] = -INFINITY; continue; }
                 double dot = 0.0;
                 for (int d = 0; d < D; ++d) dot += qr[d] * kr[(long)j * D + d];
                 double s = scale * dot;
@@ -114,16 +125,29 @@ void af_oracle_fwd(const double* q, const double* k, const double* v,
     }
 }
 
+void af_oracle_fwd(const double* q, const double* k, const double* v,
+                   int B, int Hq, int Hkv, int S, int D,
+                   double theta, int R, int p0, int causal, int window,
+                   const double* slopes, double scale,
+                   const int* rows, int n_rows, double* o, double* lse)
+{
+    af_oracle_fwd_blocks(q, k, v, B, Hq, Hkv, S, D, theta, R, p0, causal, window, slopes, scale, NULL, 0,
+                         rows, n_rows, o, lse);
+}
+
 /*
  * Backward, given upstream dO [B,Hq,S,D].  Recomputes P from the definition.
  * dq [B,Hq,S,D], dk, dv [B,Hkv,S,D]; dk and dv of a kv head sum over its g query heads.
  */
-void af_oracle_bwd(const double* q, const double* k, const double* v, const double* d_o,
-                   int B, int Hq, int Hkv, int S, int D,
-                   double theta, int R, int p0, int causal, int window,
-                   const double* slopes, double scale,
-                   double* dq, double* dk, double* dv)
+void af_oracle_bwd_blocks(const double* q, const double* k, const double* v, const double* d_o,
+                          int B, int Hq, int Hkv, int S, int D,
+                          double theta, int R, int p0, int causal, int window,
+                          const double* slopes, double scale,
+                          const unsigned char* blocks, int block_size,
+                          double* dq, double* dk, double* dv)
 {
+    block_mask bmv = { blocks, block_size, block_size > 0 ? (S + block_size - 1) / block_size : 0 };
+    const block_mask* bm = blocks ? &bmv : NULL;
     int g = Hq / Hkv;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int bk = 0; bk < B * Hkv; ++bk) {
@@ -149,7 +173,7 @@ void af_oracle_bwd(const double* q, const double* k, const double* v, const doub
                 const double* doi = doh + (long)i * D;
                 double m = -INFINITY;
                 for (int j = 0; j < S; ++j) {
-                    if (!kept(i, j, causal, window)) { pr[j] = -INFINITY; continue; }
+                    if (!kept(i, j, causal, window, bm)) { pr[j] = -INFINITY; continue; }
                     double dot = 0.0;
                     for (int d = 0; d < D; ++d) dot += qr[d] * kr[(long)j * D + d];
                     double s = scale * dot;
@@ -191,4 +215,14 @@ void af_oracle_bwd(const double* q, const double* k, const double* v, const doub
         for (int j = 0; j < S; ++j) rope_row(dkr + (long)j * D, dkh + (long)j * D, D, R, theta, (long)p0 + j, -1);
         free(kr); free(dkr); free(qr); free(dqr); free(orow); free(pr);
     }
+}
+
+void af_oracle_bwd(const double* q, const double* k, const double* v, const double* d_o,
+                   int B, int Hq, int Hkv, int S, int D,
+                   double theta, int R, int p0, int causal, int window,
+                   const double* slopes, double scale,
+                   double* dq, double* dk, double* dv)
+{
+    af_oracle_bwd_blocks(q, k, v, d_o, B, Hq, Hkv, S, D, theta, R, p0, causal, window, slopes, scale, NULL, 0,
+                         dq, dk, dv);
 }

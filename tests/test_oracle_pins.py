@@ -311,3 +311,55 @@ def test_backward_structural_properties():
     perm = [2, 1, 0, 3]
     _, dk3, _ = oracle.bwd(q[:, perm], k, v, do[:, perm], **kw)
     assert not np.allclose(dk3, dk, atol=1e-6)
+
+
+# ---------------------------------------------------------------- block-sparse attention (Section 4.6)
+
+def test_blocks_all_active_is_the_dense_result():
+    q, k, v, do = rnd((1, 4, 24, 8), 60), rnd((1, 2, 24, 8), 61), rnd((1, 2, 24, 8), 62), rnd((1, 4, 24, 8), 63)
+    kw = dict(theta=100.0, rotary_dim=8, pos_offset=3, causal=True, window=9, scale=0.3)
+    ones = np.ones((6, 6))
+    a, b = oracle.fwd(q, k, v, **kw), oracle.fwd(q, k, v, blocks=ones, block_size=4, **kw)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    ga, gb = oracle.bwd(q, k, v, do, **kw), oracle.bwd(q, k, v, do, blocks=ones, block_size=4, **kw)
+    assert all(np.array_equal(x, y) for x, y in zip(ga, gb))
+
+
+def test_block_diagonal_mask_is_independent_attention_per_block():
+    """With only the diagonal blocks active (no causal rule) every block attends to itself: the same as
+    running each block alone, at its own position offset (a ragged last block included)."""
+    S, bs, D = 22, 8, 8
+    q, k, v, do = rnd((1, 2, S, D), 64), rnd((1, 2, S, D), 65), rnd((1, 2, S, D), 66), rnd((1, 2, S, D), 67)
+    nb = 3
+    kw = dict(theta=50.0, rotary_dim=4, causal=False, scale=0.4)
+    o, l = oracle.fwd(q, k, v, pos_offset=5, blocks=np.eye(nb), block_size=bs, **kw)
+    dq, dk, dv = oracle.bwd(q, k, v, do, pos_offset=5, blocks=np.eye(nb), block_size=bs, **kw)
+    for b0 in range(0, S, bs):
+        sl = slice(b0, min(S, b0 + bs))
+        ob, lb = oracle.fwd(q[:, :, sl], k[:, :, sl], v[:, :, sl], pos_offset=5 + b0, **kw)
+        assert np.allclose(o[:, :, sl], ob, atol=1e-13) and np.allclose(l[:, :, sl], lb, atol=1e-13)
+        gq, gk, gv = oracle.bwd(q[:, :, sl], k[:, :, sl], v[:, :, sl], do[:, :, sl], pos_offset=5 + b0, **kw)
+        assert np.allclose(dq[:, :, sl], gq, atol=1e-13) and np.allclose(dk[:, :, sl], gk, atol=1e-13)
+        assert np.allclose(dv[:, :, sl], gv, atol=1e-13)
+
+
+def test_blocks_brute_force_and_autograd_tiny():
+    """Random block pattern on top of the causal rule against an explicit masked softmax in torch
+    (forward) and its autograd (backward); one query block has no active block at all."""
+    S, bs, D, Hq, Hkv = 12, 3, 4, 4, 2
+    q, k, v, do = rnd((2, Hq, S, D), 70), rnd((2, Hkv, S, D), 71), rnd((2, Hkv, S, D), 72), rnd((2, Hq, S, D), 73)
+    blocks = np.array([[1, 0, 0, 0], [0, 0, 0, 0], [1, 0, 1, 0], [0, 1, 1, 1]])
+    keep = np.kron(blocks, np.ones((bs, bs))).astype(bool) & (np.arange(S)[None, :] <= np.arange(S)[:, None])
+    tq, tk, tv = (torch.from_numpy(x).requires_grad_(True) for x in (q, k, v))
+    s = 0.5 * tq @ tk.repeat_interleave(2, dim=1).transpose(-1, -2)
+    s = s.masked_fill(~torch.from_numpy(keep), float("-inf"))
+    p = torch.nan_to_num(torch.softmax(s, -1), nan=0.0)      # rows without a kept pair: all zero
+    out = p @ tv.repeat_interleave(2, dim=1)
+    out.backward(torch.from_numpy(do))
+    o, l = oracle.fwd(q, k, v, rotary_dim=0, causal=True, scale=0.5, blocks=blocks, block_size=bs)
+    assert np.allclose(o, out.detach().numpy(), atol=1e-12)
+    assert np.all(o[:, :, 3:6] == 0.0) and np.all(np.isneginf(l[:, :, 3:6]))
+    dq, dk, dv = oracle.bwd(q, k, v, do, rotary_dim=0, causal=True, scale=0.5, blocks=blocks, block_size=bs)
+    assert np.allclose(dq, tq.grad.numpy(), atol=1e-11) and np.allclose(dk, tk.grad.numpy(), atol=1e-11)
+    assert np.allclose(dv, tv.grad.numpy(), atol=1e-11)
+    assert np.all(dq[:, :, 3:6] == 0.0)
