@@ -92,6 +92,30 @@ af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, cons
                        int gqa_group, float softmax_scale,
                        void* o, af_dtype o_dtype, float* lse, void* cuda_stream);
 
+/* ---- block-sparse attention (Section 4.6) ------------------------------------------------------------
+ * The caller evaluates its block predicate once and passes the active 128 x 128 blocks as index lists
+ * (device memory, int32): by query row block (CSR: row_ptr [nb + 1], col_idx [row_ptr[nb]], nb = ceil(S/128))
+ * and, for the backward, by key block (CSC: col_ptr [nb + 1], row_idx [col_ptr[nb]]).  Kernels visit only
+ * the listed blocks, so the work is proportional to the active fraction.  A pair (i, j) is kept iff its
+ * block is listed AND the element mask of af_mask keeps it (so listing a diagonal block under a causal
+ * mask gives the usual triangle); a query row without a kept pair gets O = 0, L = -inf, zero gradients.
+ * The lists are not validated on the device: indices must lie in [0, nb) and the CSC lists must describe
+ * the same set of blocks as the CSR lists. */
+typedef struct {
+    int block;            /* block edge; must be 128 */
+    const int* row_ptr;   /* CSR by query row block (device) */
+    const int* col_idx;
+    const int* col_ptr;   /* CSC by key block (device); needed by attnfuse_bwd_blocks only */
+    const int* row_idx;
+} af_blocks;
+
+/* attnfuse_fwd over the listed blocks. */
+af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* k, const void* v,
+                              const af_strides* sq, const af_strides* skv,
+                              const af_rope* rope, const void* rope_table, const af_mask* mask,
+                              int gqa_group, float softmax_scale, const af_blocks* blocks,
+                              void* o, af_dtype o_dtype, float* lse, void* cuda_stream);
+
 /* Same computation with HOST buffers: q, k, v, o (bf16) and lse (nullable) are host pointers
  * (pinned memory recommended).  `staging` is a DEVICE buffer of at least attnfuse_fwd_host_staging_bytes()
  * bytes; the call enqueues host-to-device copies, the kernel and device-to-host copies on the stream.

@@ -29,6 +29,11 @@ class _Strides(ctypes.Structure):
     _fields_ = [("b", ctypes.c_int64), ("h", ctypes.c_int64), ("s", ctypes.c_int64)]
 
 
+class _Blocks(ctypes.Structure):
+    _fields_ = [("block", ctypes.c_int), ("row_ptr", ctypes.c_void_p), ("col_idx", ctypes.c_void_p),
+                ("col_ptr", ctypes.c_void_p), ("row_idx", ctypes.c_void_p)]
+
+
 class _Rope(ctypes.Structure):
     _fields_ = [("theta", ctypes.c_float), ("rotary_dim", ctypes.c_int), ("pos_offset", ctypes.c_int)]
 
@@ -86,6 +91,9 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_bwd.restype = i
         L.attnfuse_bwd.argtypes = [P(_Shape), vp, vp, vp, vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp,
                                    P(_Mask), i, f, vp, i, vp, vp, i, vp, sz, vp]
+        L.attnfuse_fwd_blocks.restype = i
+        L.attnfuse_fwd_blocks.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp, P(_Mask), i, f,
+                                          P(_Blocks), vp, i, vp, vp]
         L.attnfuse_decode_splits.restype = i
         L.attnfuse_decode_splits.argtypes = [P(_Shape)]
         L.attnfuse_decode_workspace_bytes.restype = sz
@@ -188,6 +196,57 @@ def fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, 
                               ctypes.byref(m), Hq // Hkv, float(softmax_scale), out.data_ptr(),
                               AF_F32 if out.dtype == torch.float32 else AF_BF16,
                               lse.data_ptr() if lse is not None else None, _stream()))
+    return out, lse
+
+
+class BlockMask:
+    """Active 128 x 128 blocks of a block-sparse mask (Section 4.6) as device index lists: CSR by query row
+    block and CSC by key block.  Built once from a boolean [nb, nb] matrix (nb = ceil(S / 128))."""
+
+    def __init__(self, active, device="cuda"):
+        a = torch.as_tensor(active).to(torch.bool).cpu()
+        assert a.dim() == 2 and a.shape[0] == a.shape[1]
+        self.nb = a.shape[0]
+        self.active = a
+        counts = a.sum(1).to(torch.int32)
+        self.row_ptr = torch.cat([torch.zeros(1, dtype=torch.int32), counts.cumsum(0).to(torch.int32)]).to(device)
+        self.col_idx = a.nonzero()[:, 1].to(torch.int32).contiguous().to(device)
+        at = a.t().contiguous()
+        counts_t = at.sum(1).to(torch.int32)
+        self.col_ptr = torch.cat([torch.zeros(1, dtype=torch.int32), counts_t.cumsum(0).to(torch.int32)]).to(device)
+        self.row_idx = at.nonzero()[:, 1].to(torch.int32).contiguous().to(device)
+        if self.col_idx.numel() == 0:   # keep the pointers valid
+            self.col_idx = torch.zeros(1, dtype=torch.int32, device=device)
+            self.row_idx = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def struct(self):
+        return _Blocks(128, self.row_ptr.data_ptr(), self.col_idx.data_ptr(), self.col_ptr.data_ptr(),
+                       self.row_idx.data_ptr())
+
+
+def fwd_blocks(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor],
+               mask: MaskSpec, softmax_scale: float, blocks: BlockMask, out: Optional[torch.Tensor] = None,
+               lse: Optional[torch.Tensor] = None, out_dtype: torch.dtype = torch.bfloat16):
+    """Block-sparse forward: `fwd` restricted to the active blocks of `blocks`.  Returns (o, lse)."""
+    _need_cuda(q, k, v, table, out, lse)
+    assert q.dtype == k.dtype == v.dtype == torch.bfloat16
+    B, Hq, S, D = q.shape
+    Hkv = k.shape[1]
+    assert k.shape == v.shape == (B, Hkv, S, D) and k.stride() == v.stride()
+    assert blocks.nb == (S + 127) // 128
+    if out is None:
+        out = torch.empty((B, Hq, S, D), dtype=out_dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((B, Hq, S), dtype=torch.float32, device=q.device)
+    sh = _Shape(B, Hq, Hkv, S, D)
+    sq, skv = _strides(q), _strides(k)
+    r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
+    m = _mask_struct(mask)
+    bl = blocks.struct()
+    _check(lib().attnfuse_fwd_blocks(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), ctypes.byref(sq),
+                                     ctypes.byref(skv), ctypes.byref(r), table.data_ptr() if table is not None else None,
+                                     ctypes.byref(m), Hq // Hkv, float(softmax_scale), ctypes.byref(bl), out.data_ptr(),
+                                     AF_F32 if out.dtype == torch.float32 else AF_BF16, lse.data_ptr(), _stream()))
     return out, lse
 
 

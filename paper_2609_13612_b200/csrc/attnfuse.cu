@@ -146,6 +146,35 @@ af_status launch_fwd2_variant(const CUtensorMap& tq, const CUtensorMap& tk2, con
     return cudaLaunchKernelEx(&cfg, kern, tq, tk2, tv, p) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
+// Block-sparse variant (Section 4.6): the grid is (heads or head pairs, 128-row blocks); every CTA walks the
+// list of active key blocks of its row block.  An even GQA group pairs two heads per CTA, otherwise one head.
+template <int D, int NQ, bool ROPE>
+af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, FwdParams p,
+                                    cudaStream_t stream) {
+    using L = FwdSmem<D, NQ, 2, 2>;
+    auto kern = attn_fwd_kernel<D, NQ, ROPE, 2, 2, true>;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
+            return AF_ERR_CUDA;
+        configured = true;
+    }
+    p.pair_heads = NQ == 2 ? 1 : 0;
+    p.n_row_blocks = (p.S + BM - 1) / BM;
+    dim3 grid(NQ == 2 ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
+    kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, p);
+    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+template <int D>
+af_status launch_fwd_blocks(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
+                            cudaStream_t stream) {
+    if ((p.group % 2) == 0)
+        return p.R > 0 ? launch_fwd_blocks_variant<D, 2, true>(tq, tk, tv, p, stream)
+                       : launch_fwd_blocks_variant<D, 2, false>(tq, tk, tv, p, stream);
+    return p.R > 0 ? launch_fwd_blocks_variant<D, 1, true>(tq, tk, tv, p, stream)
+                   : launch_fwd_blocks_variant<D, 1, false>(tq, tk, tv, p, stream);
+}
+
 template <int D>
 af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                      cudaStream_t stream) {
@@ -312,9 +341,14 @@ af_status attnfuse_rope(const af_shape* shape, int n_heads, const void* x_in, vo
     return launch_rope(x_in, st, x_out, shape->B, n_heads, shape->S, D, R, rope_table, inverse, stream);
 }
 
-af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
-                       const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
-                       int gqa_group, float softmax_scale, void* o, af_dtype o_dtype, float* lse, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+// Forward, dense (bs_row_ptr == nullptr) or over CSR lists of active 128 x 128 blocks.
+af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
+                   const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
+                   int gqa_group, float softmax_scale, const int* bs_row_ptr, const int* bs_col_idx, void* o,
+                   af_dtype o_dtype, float* lse, void* cuda_stream) {
     af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
     if (st != AF_OK) return st;
     if (!q || !k || !v || !o) return AF_ERR_NULL;
@@ -342,11 +376,15 @@ af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, cons
     p.o = o; p.o_f32 = (o_dtype == AF_F32); p.lse = lse;
     p.n_row_blocks = 0;
     p.pair_heads = 0;
+    p.bs_row_ptr = bs_row_ptr;
+    p.bs_col_idx = bs_col_idx;
 #ifdef AF_TRACE
     p.trace = reinterpret_cast<long long*>(getenv("AF_TRACE_PTR") ? strtoull(getenv("AF_TRACE_PTR"), nullptr, 0) : 0ull);
     cudaMemcpyToSymbol(af::g_trace, &p.trace, sizeof(p.trace));
 #endif
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (bs_row_ptr)
+        return shape->D == 128 ? launch_fwd_blocks<128>(tq, tk, tv, p, stream) : launch_fwd_blocks<64>(tq, tk, tv, p, stream);
     const int R = rope->rotary_dim;
     const bool pair_ok = shape->D == 128 && (gqa_group % 4) == 0 && (R == 0 || R == 16 || R == 32 || R == 64 || R == 128);
     if (pair_ok && env_int("AF_FWD_2CTA", 0)) {
@@ -355,6 +393,26 @@ af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, cons
         return R > 0 ? launch_fwd2_variant<true>(tq, tk2, tv, p, stream) : launch_fwd2_variant<false>(tq, tk2, tv, p, stream);
     }
     return shape->D == 128 ? launch_fwd<128>(tq, tk, tv, p, stream) : launch_fwd<64>(tq, tk, tv, p, stream);
+}
+}  // namespace
+
+extern "C" {
+
+af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
+                       const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
+                       int gqa_group, float softmax_scale, void* o, af_dtype o_dtype, float* lse, void* cuda_stream) {
+    return fwd_impl(shape, q, k, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, nullptr, nullptr, o,
+                    o_dtype, lse, cuda_stream);
+}
+
+af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
+                              const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
+                              int gqa_group, float softmax_scale, const af_blocks* blocks, void* o, af_dtype o_dtype,
+                              float* lse, void* cuda_stream) {
+    if (!blocks || !blocks->row_ptr || !blocks->col_idx) return AF_ERR_NULL;
+    if (blocks->block != 128) return AF_ERR_SPEC;
+    return fwd_impl(shape, q, k, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, blocks->row_ptr,
+                    blocks->col_idx, o, o_dtype, lse, cuda_stream);
 }
 
 size_t attnfuse_fwd_host_staging_bytes(const af_shape* shape) {

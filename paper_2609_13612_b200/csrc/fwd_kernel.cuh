@@ -23,6 +23,11 @@ struct FwdParams {
     float* lse;         // nullable
     int n_row_blocks;   // ceil(S / (128 * NQ)), or ceil(S / 128) with pair_heads
     int pair_heads;     // NQ = 2 only: the two query tiles are the same 128 rows of two heads of one kv group
+    // Block-sparse attention (Section 4.6), BS kernels only: CSR lists of the active 128 x 128 blocks, row_ptr
+    // [ceil(S/128) + 1] and col_idx [row_ptr[last]] (device).  The key loop walks a row block's list instead of
+    // a contiguous tile range; the element mask (causal, window) still applies inside the listed tiles.
+    const int* bs_row_ptr;
+    const int* bs_col_idx;
 #ifdef AF_TRACE
     long long* trace;
 #endif
@@ -252,7 +257,7 @@ __device__ __forceinline__ bool softmax_tile_halves(uint32_t tS, uint32_t tO, in
     return true;
 }
 
-template <int D, int NQ, bool ROPE, int KS, int VS>
+template <int D, int NQ, bool ROPE, int KS, int VS, bool BS = false>
 __global__ void __launch_bounds__(128 * (2 + NQ), 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const FwdParams p) {
@@ -299,6 +304,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             jhi[q] = 0;  // empty
         }
     }
+    // Block-sparse: the loops below run over positions in the row block's list (jlo = 0, jhi = length - 1, the
+    // same for both query tiles, which share the row block); tile_at() gives the key tile of a position.
+    int bs_base = 0;
+    if constexpr (BS) {
+        bs_base = __ldg(p.bs_row_ptr + rb);
+        const int len = (rb * BM < p.S) ? __ldg(p.bs_row_ptr + rb + 1) - bs_base : 0;
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            jlo[q] = 0;
+            jhi[q] = len - 1;
+        }
+        jlo_c = 0;
+        jhi_c = len - 1;
+    }
+    auto tile_at = [&](int pos) { return BS ? __ldg(p.bs_col_idx + bs_base + pos) : pos; };
     const int n_it = jhi_c - jlo_c + 1;
     AF_STAMP(0, 63, 0);  // kernel entry
 
@@ -344,7 +364,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     tma_load_4d(sQ + q * TILE + bx * BOX_BYTES, &tm_q, &bars[L::B_QFULL + q], bx * BOX_COLS, i0[q], hq[q], b);
             }
             for (int it = 0; it < n_it; ++it) {
-                const int j0 = (jlo_c + it) * BN;
+                const int j0 = tile_at(jlo_c + it) * BN;
                 const int ks = it % KS, vs = it % VS;
                 if (!mbar_wait(&bars[L::B_KEMPTY + ks], ((it / KS) & 1) ^ 1, abort_flag, 1)) break;
                 mbar_arrive_expect_tx(&bars[L::B_KFULL + ks], TILE);
@@ -408,6 +428,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
             // prologue: S of the first key tile, each query tile as soon as it is ready (the softmax
             // warpgroups rotate their Q tiles while the rotation warpgroup rotates K tile 0)
+            if (BS && n_it <= 0) ok = false;   // a row block without active blocks: nothing to issue
             if (ok) ok = mbar_wait(&bars[B_KREADY + 0], 0, abort_flag, 4);
             AF_STAMP(0, 63, 3);  // first K ready
 #pragma unroll
@@ -476,13 +497,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // K tiles are consecutive: the recurrence carries the cos/sin state from tile to tile
                 for (int it = 0; ok && it < n_it; ++it) {
                     const int ks = it % KS;
-                    if (CP > 0 && (it % kRotResync) == 0) rotate_prefetch(st, p.table, (jlo_c + it) * BN, p.S, p.R, t);
+                    // (listed tiles need not be consecutive: the cos/sin state is read for every tile)
+                    if (CP > 0 && (BS || (it % kRotResync) == 0)) rotate_prefetch(st, p.table, tile_at(jlo_c + it) * BN, p.S, p.R, t);
                     AF_STAMP(1, it, 0);
                     ok = mbar_wait_warp(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
                     AF_STAMP(1, it, 1);
                     if (!ok) break;
                     if (CP > 0) rotate_tile_fast(sK + ks * TILE, st, step, t);
-                    else rotate_tile_smem(sK + ks * TILE, (jlo_c + it) * BN, p.S, p.R, p.table, t, 128);
+                    else rotate_tile_smem(sK + ks * TILE, tile_at(jlo_c + it) * BN, p.S, p.R, p.table, t, 128);
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars[L::B_KROT + ks]);
@@ -538,7 +560,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             else rot_q(std::integral_constant<int, 0>{});
         }
         for (int j = jlo[q]; ok && j <= jhi[q]; ++j, ++n) {
-            const int j0 = j * BN;
+            const int j0 = tile_at(j) * BN;
             AF_STAMP(2 + q, n, 0);
             const bool need_mask = tile_needs_mask(ms, i0[q], j0);
             const float bias0 = slope2 * static_cast<float>(j0 - i);
@@ -590,6 +612,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (p.lse && i < p.S)
                 p.lse[static_cast<size_t>(bh) * p.S + i] =
                     l_run > 0.f ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+        }
+        if (BS && ok && jhi[q] < jlo[q] && i < p.S) {
+            // no active block in this row block: the output row is zero and L = -inf
+            const size_t orow = (static_cast<size_t>(bh) * p.S + i) * D;
+            if (p.o_f32) {
+                float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + orow);
+                for (int e = 0; e < D / 4; ++e) dst[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else {
+                uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.o) + orow);
+                for (int e = 0; e < D / 8; ++e) dst[e] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            if (p.lse) p.lse[static_cast<size_t>(bh) * p.S + i] = -INFINITY;
         }
     }
 
