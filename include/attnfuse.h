@@ -169,6 +169,16 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
                        void* dq, af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* attnfuse_bwd over the listed blocks (Section 4.6); needs both the CSR and the CSC lists of `blocks`.
+ * lse must come from attnfuse_fwd_blocks with the same lists; rows whose L is -inf get zero gradients. */
+af_status attnfuse_bwd_blocks(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,
+                              const float* lse, const void* d_o,
+                              const af_strides* sq, const af_strides* skv,
+                              const af_rope* rope, const void* rope_table, const af_mask* mask,
+                              int gqa_group, float softmax_scale, const af_blocks* blocks,
+                              void* dq, af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* ---- backward without a caller workspace (the paper has no counterpart) ---------------------------
  * Some callers are not allowed to obtain device memory at the point where they need the backward:
  * a plug-in that runs inside another framework's enqueue hook, a serving loop whose memory pool was

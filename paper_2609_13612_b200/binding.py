@@ -94,6 +94,9 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_fwd_blocks.restype = i
         L.attnfuse_fwd_blocks.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp, P(_Mask), i, f,
                                           P(_Blocks), vp, i, vp, vp]
+        L.attnfuse_bwd_blocks.restype = i
+        L.attnfuse_bwd_blocks.argtypes = [P(_Shape), vp, vp, vp, vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp,
+                                          P(_Mask), i, f, P(_Blocks), vp, i, vp, vp, i, vp, sz, vp]
         L.attnfuse_decode_splits.restype = i
         L.attnfuse_decode_splits.argtypes = [P(_Shape)]
         L.attnfuse_decode_workspace_bytes.restype = sz
@@ -276,8 +279,9 @@ def fwd_host_staging_bytes(B: int, Hq: int, Hkv: int, S: int, D: int) -> int:
 
 
 def bwd(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softmax_scale: float,
-        dq_dtype: torch.dtype = torch.bfloat16, dkv_dtype: torch.dtype = torch.float32, workspace=None):
-    """Fused backward.  Returns (dq, dk, dv)."""
+        dq_dtype: torch.dtype = torch.bfloat16, dkv_dtype: torch.dtype = torch.float32, workspace=None,
+        blocks: Optional[BlockMask] = None):
+    """Fused backward (over the active blocks of `blocks`, if given).  Returns (dq, dk, dv)."""
     _need_cuda(q, k, v, o, lse, d_o, table, workspace)
     B, Hq, S, D = q.shape
     Hkv = k.shape[1]
@@ -294,6 +298,16 @@ def bwd(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softma
     r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
     m = _mask_struct(mask)
     code = lambda dt: AF_F32 if dt == torch.float32 else AF_BF16
+    if blocks is not None:
+        assert blocks.nb == (S + 127) // 128
+        bl = blocks.struct()
+        _check(lib().attnfuse_bwd_blocks(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                         lse.data_ptr(), d_o.data_ptr(), ctypes.byref(sq), ctypes.byref(skv),
+                                         ctypes.byref(r), table.data_ptr() if table is not None else None,
+                                         ctypes.byref(m), Hq // Hkv, float(softmax_scale), ctypes.byref(bl),
+                                         dq.data_ptr(), code(dq_dtype), dk.data_ptr(), dv.data_ptr(), code(dkv_dtype),
+                                         workspace.data_ptr(), workspace.numel(), _stream()))
+        return dq, dk, dv
     _check(lib().attnfuse_bwd(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
                               lse.data_ptr(), d_o.data_ptr(), ctypes.byref(sq), ctypes.byref(skv), ctypes.byref(r),
                               table.data_ptr() if table is not None else None, ctypes.byref(m), Hq // Hkv,

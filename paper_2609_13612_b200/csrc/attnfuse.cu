@@ -187,11 +187,11 @@ af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
                    : launch_fwd_variant<D, 2, false, 2, 2>(tq, tk, tv, p, stream);
 }
 
-template <int D, bool DKV, bool ROT_X, bool ROT_A>
-af_status launch_bwd_variant(const CUtensorMap& tx, const CUtensorMap& ty, const CUtensorMap& ta, const CUtensorMap& tb,
-                             const CUtensorMap& ts, const BwdParams& p, dim3 grid, cudaStream_t stream) {
+template <int D, bool DKV, bool ROT_X, bool ROT_A, bool BS>
+af_status launch_bwd_variant_bs(const CUtensorMap& tx, const CUtensorMap& ty, const CUtensorMap& ta, const CUtensorMap& tb,
+                                const CUtensorMap& ts, const BwdParams& p, dim3 grid, cudaStream_t stream) {
     using L = BwdSmem<D>;
-    auto kern = attn_bwd_kernel<D, DKV, ROT_X, ROT_A>;
+    auto kern = attn_bwd_kernel<D, DKV, ROT_X, ROT_A, BS>;
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
@@ -200,6 +200,13 @@ af_status launch_bwd_variant(const CUtensorMap& tx, const CUtensorMap& ty, const
     }
     kern<<<grid, 512, L::BYTES, stream>>>(tx, ty, ta, tb, ts, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+// dense or, when the parameters carry block lists, block-sparse instantiation
+template <int D, bool DKV, bool ROT_X, bool ROT_A>
+af_status launch_bwd_variant(const CUtensorMap& tx, const CUtensorMap& ty, const CUtensorMap& ta, const CUtensorMap& tb,
+                             const CUtensorMap& ts, const BwdParams& p, dim3 grid, cudaStream_t stream) {
+    return p.bs_ptr ? launch_bwd_variant_bs<D, DKV, ROT_X, ROT_A, true>(tx, ty, ta, tb, ts, p, grid, stream)
+                    : launch_bwd_variant_bs<D, DKV, ROT_X, ROT_A, false>(tx, ty, ta, tb, ts, p, grid, stream);
 }
 
 // RoPE pass x [B, H, S, D] (strided) -> x_out (contiguous); R > 0.
@@ -224,7 +231,13 @@ template <int D>
 af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                      const CUtensorMap& tdo, const CUtensorMap* tkp, const CUtensorMap* tqp, const void* k,
                      const af_strides& stkv, void* kcache, const void* o, const void* d_o, BwdParams p, void* dq,
-                     int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, cudaStream_t stream) {
+                     int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, const af_blocks* blocks,
+                     cudaStream_t stream) {
+    // block lists by stationary block: by key block for the dK/dV role, by query block for the dQ role
+    auto role_lists = [&](bool dkv_role) {
+        p.bs_ptr = blocks ? (dkv_role ? blocks->col_ptr : blocks->row_ptr) : nullptr;
+        p.bs_idx = blocks ? (dkv_role ? blocks->row_idx : blocks->col_idx) : nullptr;
+    };
     const long long rows = static_cast<long long>(sh->B) * sh->Hq * sh->S;
     const long long threads = rows * (D / 8);
     bwd_delta_kernel<D><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
@@ -239,17 +252,21 @@ af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMa
         // both caches: K' by the RoPE pass, Q' by the dQ kernel, no on-chip rotation in the dK/dV loop
         if ((st = launch_rope(k, stkv, kcache, sh->B, sh->Hkv, sh->S, D, p.R, p.table, 0, stream)) != AF_OK) return st;
         p.out1 = dq; p.out2 = nullptr; p.out_f32 = dq_f32; p.store_x = 1;
+        role_lists(false);
         if ((st = launch_bwd_variant<D, false, true, false>(tq, tdo, *tkp, tv, *tqp, p, gq, stream)) != AF_OK) return st;
         p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32; p.store_x = 0;
+        role_lists(true);
         return launch_bwd_variant<D, true, false, false>(*tkp, tv, *tqp, tdo, tk, p, gkv, stream);
     }
     const bool cache = p.R > 0 && tkp != nullptr && only != 2;
     p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32; p.store_x = cache ? 1 : 0;
+    role_lists(true);
     st = only == 2 ? AF_OK
          : p.R > 0 ? launch_bwd_variant<D, true, true, true>(tk, tv, tq, tdo, cache ? *tkp : tk, p, gkv, stream)
                    : launch_bwd_variant<D, true, false, false>(tk, tv, tq, tdo, tk, p, gkv, stream);
     if (st != AF_OK || only == 1) return st;
     p.out1 = dq; p.out2 = nullptr; p.out_f32 = dq_f32; p.store_x = 0;
+    role_lists(false);
     if (p.R == 0) return launch_bwd_variant<D, false, false, false>(tq, tdo, tk, tv, tk, p, gq, stream);
     return cache ? launch_bwd_variant<D, false, true, false>(tq, tdo, *tkp, tv, tk, p, gq, stream)
                  : launch_bwd_variant<D, false, true, true>(tq, tdo, tk, tv, tk, p, gq, stream);
@@ -528,11 +545,15 @@ size_t attnfuse_bwd_workspace_bytes(const af_shape* shape) {
     return bwd_delta_bytes(shape) + bwd_kcache_bytes(shape) + bwd_qcache_bytes(shape);   // delta + rotated-K and -Q caches
 }
 
-af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,
-                       const float* lse, const void* d_o, const af_strides* sq, const af_strides* skv,
-                       const af_rope* rope, const void* rope_table, const af_mask* mask, int gqa_group,
-                       float softmax_scale, void* dq, af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
-                       void* workspace, size_t workspace_bytes, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+// Backward, dense (blocks == nullptr) or over the index lists of active 128 x 128 blocks.
+af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,
+                   const float* lse, const void* d_o, const af_strides* sq, const af_strides* skv,
+                   const af_rope* rope, const void* rope_table, const af_mask* mask, int gqa_group,
+                   float softmax_scale, const af_blocks* blocks, void* dq, af_dtype dq_dtype, void* dk, void* dv,
+                   af_dtype dkv_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
     if (st != AF_OK) return st;
     if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv) return AF_ERR_NULL;
@@ -564,6 +585,7 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
     p.table = static_cast<const float2*>(rope_table);
     p.lse = lse;
     p.delta = nullptr; p.out1 = nullptr; p.out2 = nullptr; p.out_f32 = 0; p.store_x = 0;
+    p.bs_ptr = nullptr; p.bs_idx = nullptr;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     float* delta = static_cast<float*>(workspace);
     // rotated-K and rotated-Q caches: used when there is a rotation and the workspace has room behind delta
@@ -583,9 +605,33 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
     }
     return shape->D == 128
                ? launch_bwd<128>(shape, tq, tk, tv, tdo, have_k ? &tkp : nullptr, have_q ? &tqp : nullptr, k, stkv, kc, o,
-                                 d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, stream)
+                                 d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream)
                : launch_bwd<64>(shape, tq, tk, tv, tdo, have_k ? &tkp : nullptr, have_q ? &tqp : nullptr, k, stkv, kc, o,
-                                d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, stream);
+                                d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream);
+}
+}  // namespace
+
+extern "C" {
+
+af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,
+                       const float* lse, const void* d_o, const af_strides* sq, const af_strides* skv,
+                       const af_rope* rope, const void* rope_table, const af_mask* mask, int gqa_group,
+                       float softmax_scale, void* dq, af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return bwd_impl(shape, q, k, v, o, lse, d_o, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, nullptr, dq,
+                    dq_dtype, dk, dv, dkv_dtype, workspace, workspace_bytes, cuda_stream);
+}
+
+af_status attnfuse_bwd_blocks(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,
+                              const float* lse, const void* d_o, const af_strides* sq, const af_strides* skv,
+                              const af_rope* rope, const void* rope_table, const af_mask* mask, int gqa_group,
+                              float softmax_scale, const af_blocks* blocks, void* dq, af_dtype dq_dtype, void* dk,
+                              void* dv, af_dtype dkv_dtype, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream) {
+    if (!blocks || !blocks->row_ptr || !blocks->col_idx || !blocks->col_ptr || !blocks->row_idx) return AF_ERR_NULL;
+    if (blocks->block != 128) return AF_ERR_SPEC;
+    return bwd_impl(shape, q, k, v, o, lse, d_o, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, blocks, dq,
+                    dq_dtype, dk, dv, dkv_dtype, workspace, workspace_bytes, cuda_stream);
 }
 
 }  // extern "C"

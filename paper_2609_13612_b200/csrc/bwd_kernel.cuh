@@ -36,7 +36,12 @@ struct BwdParams {
     void* out1;           // DKV: dV   DQ: dQ
     void* out2;           // DKV: dK   DQ: unused
     int out_f32;
-    int store_x;          // DKV role: write the rotated X tile through tm_s
+    int store_x;          // write the rotated X tile through tm_s
+    // Block-sparse attention (Section 4.6), BS kernels only: index lists of the active 128 x 128 blocks by
+    // stationary block - for the dK/dV role by key block (the query blocks that see it), for the dQ role by
+    // query block (its key blocks): ptr [ceil(S/128) + 1], idx [ptr[last]] (device).
+    const int* bs_ptr;
+    const int* bs_idx;
 };
 
 // delta[row] = <dO[row], O[row]>; one 16-byte chunk per thread, D/8 threads per row.
@@ -246,7 +251,7 @@ __device__ __forceinline__ void grad_pass32(uint32_t t1, uint32_t t2, int col0, 
 #define AF_BSTAMP(role, it, ph) do { } while (0)
 #endif
 
-template <int D, bool DKV, bool ROT_X, bool ROT_A>
+template <int D, bool DKV, bool ROT_X, bool ROT_A, bool BS = false>
 __global__ void __launch_bounds__(512, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_y,
                 const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
@@ -277,11 +282,20 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
     int lo, hi;  // streamed tile range
     if (DKV) qtile_range(ms, x0, lo, hi);
     else tile_range(ms, x0, lo, hi);
+    int bs_base = 0;
+    if constexpr (BS) {   // block-sparse: positions in the stationary block's list instead of a tile range
+        bs_base = __ldg(p.bs_ptr + x0 / 128);
+        lo = 0;
+        hi = __ldg(p.bs_ptr + x0 / 128 + 1) - bs_base - 1;
+    }
     const int per_head = hi - lo + 1;
     const int n_it = DKV ? per_head * p.group : per_head;
     // iteration n -> (streamed head, streamed row0)
     auto stream_head = [&](int n) { return DKV ? xh * p.group + n / per_head : xh / p.group; };
-    auto stream_row0 = [&](int n) { return (lo + (DKV ? n % per_head : n)) * 128; };
+    auto stream_row0 = [&](int n) {
+        const int pos = lo + (DKV ? n % per_head : n);
+        return (BS ? __ldg(p.bs_idx + bs_base + pos) : pos) * 128;
+    };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::N_BARS; ++i) {
@@ -460,7 +474,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 for (int n = 0; n < n_it; ++n) {
                     const int sg = n % NST, a0 = stream_row0(n);
                     const int run_pos = DKV ? n % per_head : n;
-                    if (CP > 0 && (run_pos % kRotResync) == 0) rotate_prefetch(st, p.table, a0, p.S, p.R, t);
+                    // (listed tiles need not be consecutive: then the cos/sin state is read for every tile)
+                    if (CP > 0 && (BS || (run_pos % kRotResync) == 0)) rotate_prefetch(st, p.table, a0, p.S, p.R, t);
                     AF_BSTAMP(4, n, 0);
                     if (!mbar_wait_warp(&bars[L::B_AFULL + sg], (n / NST) & 1, abort_flag, 28)) return;
                     AF_BSTAMP(4, n, 1);
@@ -575,6 +590,19 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
         AF_BSTAMP(2 + hf, 63, 0);
         if (ok && n_it > 0) ok = wg_all(mbar_wait(&bars[L::B_DONE], 0, abort_flag, 30));
         AF_BSTAMP(2 + hf, 63, 1);   // accumulators complete
+        if (BS && ok && n_it <= 0) {
+            // no active block for this stationary block: its gradient rows are zero
+            const size_t row0 = (static_cast<size_t>(b) * xh_count + xh) * p.S + x0;
+            const int rows = min(128, p.S - x0);
+            for (int idx = gtid; idx < rows * (D / 4); idx += 256) {
+                const size_t off = (row0 + idx / (D / 4)) * D + (idx % (D / 4)) * 4;
+                for (int w2 = 0; w2 < (DKV ? 2 : 1); ++w2) {
+                    void* out = w2 == 0 ? p.out1 : p.out2;
+                    if (p.out_f32) *reinterpret_cast<float4*>(static_cast<float*>(out) + off) = make_float4(0.f, 0.f, 0.f, 0.f);
+                    else *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(out) + off) = make_uint2(0u, 0u);
+                }
+            }
+        }
         if (ok && n_it > 0) {
             tc_fence_after_sync();
             float* stg = reinterpret_cast<float*>(sA);

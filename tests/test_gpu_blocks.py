@@ -86,3 +86,55 @@ def test_block_sparse_all_active_equals_the_dense_kernel():
     # the same arithmetic except that cos/sin are read from the table for every tile instead of walked on
     assert (o1.float() - o2.float()).abs().max().item() <= 8e-3
     assert (l1 - l2).abs().max().item() <= 1e-3
+
+
+def run_bwd(w, active, workspace_tier=2, dq_dtype=torch.bfloat16):
+    t, dev, o, lse, bm = run_fwd(w, active)
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S) if w.R > 0 else None
+    n_delta = (w.B * w.Hq * w.S * 4 + 255) // 256 * 256
+    n_ws = n_delta + (w.B * w.Hkv * w.S * w.D * 2 if workspace_tier >= 1 else 0) + \
+        (w.B * w.Hq * w.S * w.D * 2 if workspace_tier >= 2 else 0)
+    ws = torch.empty(n_ws, dtype=torch.uint8, device="cuda")
+    dq, dk, dv = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale, workspace=ws,
+                        blocks=bm, dq_dtype=dq_dtype)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    want = oracle.bwd(t["q"], t["k"], t["v"], t["do"], theta=w.theta, rotary_dim=w.R, pos_offset=w.pos_offset,
+                      causal=w.causal, window=w.window, slopes=w.alibi_slopes(), scale=w.scale, blocks=active,
+                      block_size=128)
+    for name, got, ref in zip(("dQ", "dK", "dV"), (dq, dk, dv), want):
+        pu.assert_close("%s %s" % (w.name, name), pu.to_np(got), ref)
+
+
+BWD_CASES = [
+    (W("bsb_dense_pattern", 1, 4, 2, 512, 128, theta=1e4, backward=True, seed_id=421), lambda nb: np.tril(np.ones((nb, nb), bool)), 2),
+    (W("bsb_bigbird_noncausal", 2, 4, 2, 1024, 128, theta=5e5, causal=False, backward=True, seed_id=422), lambda nb: bigbird_blocks(nb, seed=11), 2),
+    (W("bsb_bigbird_causal_gqa4", 1, 8, 2, 1100, 128, theta=5e5, backward=True, seed_id=423), lambda nb: bigbird_blocks(nb, seed=12, causal=True), 2),
+    (W("bsb_bigbird_k_cache_only", 1, 4, 2, 900, 128, theta=1e4, causal=False, backward=True, seed_id=424), lambda nb: bigbird_blocks(nb, seed=13), 1),
+    (W("bsb_bigbird_no_cache", 1, 4, 2, 900, 128, theta=1e4, causal=False, backward=True, seed_id=425), lambda nb: bigbird_blocks(nb, seed=14), 0),
+    (W("bsb_d64_norope", 1, 4, 4, 700, 64, rotary_dim=0, causal=False, backward=True, seed_id=426), lambda nb: bigbird_blocks(nb, seed=15), 2),
+    (W("bsb_window_alibi", 1, 4, 2, 900, 128, theta=1e4, window=300, alibi=True, backward=True, seed_id=427), lambda nb: np.tril(np.ones((nb, nb), bool)), 2),
+]
+
+
+@pytest.mark.parametrize("w,pattern,tier", BWD_CASES, ids=lambda x: x.name if hasattr(x, "name") else "")
+def test_block_sparse_backward(w, pattern, tier):
+    run_bwd(w, pattern((w.S + 127) // 128), workspace_tier=tier)
+
+
+def test_block_sparse_backward_empty_lists_give_zero_gradient_rows():
+    w = W("bsb_empty", 1, 4, 2, 512, 128, theta=1e4, causal=False, backward=True, seed_id=430)
+    a = np.zeros((4, 4), dtype=bool)
+    a[0, 1] = a[2, 0] = a[2, 3] = True      # query blocks 1, 3 and key block 2 are never touched
+    run_bwd(w, a)
+
+
+def test_bigbird_n4096_forward_and_backward():
+    """The paper's block-sparse workload: a BigBird mask over 32 x 32 blocks at N = 4096 (about 8 % of the
+    blocks active), RoPE on, full size in the launch configuration the bench times."""
+    w = W("bigbird_4096", 1, 8, 2, 4096, 128, theta=5e5, causal=False, backward=True, seed_id=431)
+    a = bigbird_blocks(32, window=1, n_global=0, n_random=0, seed=21)
+    a[0, :] = True
+    a[:, 0] = True      # one global block row and column; band of three: (3 * 32 - 2 + 62) / 1024 = 15 %
+    run_bwd(w, a)
