@@ -107,6 +107,9 @@ typedef struct {
     const int* col_idx;
     const int* col_ptr;   /* CSC by key block (device); needed by attnfuse_bwd_blocks only */
     const int* row_idx;
+    const int* row_order; /* optional (NULL = 0, 1, 2, ...): the query row blocks in the order in which CTAs should be
+                             launched, normally by decreasing list length so that the longest lists start first */
+    const int* col_order; /* the same for key blocks (dK/dV kernel of the backward) */
 } af_blocks;
 
 /* attnfuse_fwd over the listed blocks. */

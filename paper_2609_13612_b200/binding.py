@@ -31,7 +31,8 @@ class _Strides(ctypes.Structure):
 
 class _Blocks(ctypes.Structure):
     _fields_ = [("block", ctypes.c_int), ("row_ptr", ctypes.c_void_p), ("col_idx", ctypes.c_void_p),
-                ("col_ptr", ctypes.c_void_p), ("row_idx", ctypes.c_void_p)]
+                ("col_ptr", ctypes.c_void_p), ("row_idx", ctypes.c_void_p), ("row_order", ctypes.c_void_p),
+                ("col_order", ctypes.c_void_p)]
 
 
 class _Rope(ctypes.Structure):
@@ -218,13 +219,16 @@ class BlockMask:
         counts_t = at.sum(1).to(torch.int32)
         self.col_ptr = torch.cat([torch.zeros(1, dtype=torch.int32), counts_t.cumsum(0).to(torch.int32)]).to(device)
         self.row_idx = at.nonzero()[:, 1].to(torch.int32).contiguous().to(device)
+        # launch orders: longest lists first
+        self.row_order = torch.argsort(counts, descending=True, stable=True).to(torch.int32).to(device)
+        self.col_order = torch.argsort(counts_t, descending=True, stable=True).to(torch.int32).to(device)
         if self.col_idx.numel() == 0:   # keep the pointers valid
             self.col_idx = torch.zeros(1, dtype=torch.int32, device=device)
             self.row_idx = torch.zeros(1, dtype=torch.int32, device=device)
 
     def struct(self):
         return _Blocks(128, self.row_ptr.data_ptr(), self.col_idx.data_ptr(), self.col_ptr.data_ptr(),
-                       self.row_idx.data_ptr())
+                       self.row_idx.data_ptr(), self.row_order.data_ptr(), self.col_order.data_ptr())
 
 
 def fwd_blocks(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor],

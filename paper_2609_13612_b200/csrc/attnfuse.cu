@@ -237,6 +237,7 @@ af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMa
     auto role_lists = [&](bool dkv_role) {
         p.bs_ptr = blocks ? (dkv_role ? blocks->col_ptr : blocks->row_ptr) : nullptr;
         p.bs_idx = blocks ? (dkv_role ? blocks->row_idx : blocks->col_idx) : nullptr;
+        p.bs_order = blocks ? (dkv_role ? blocks->col_order : blocks->row_order) : nullptr;
     };
     const long long rows = static_cast<long long>(sh->B) * sh->Hq * sh->S;
     const long long threads = rows * (D / 8);
@@ -364,8 +365,8 @@ namespace {
 // Forward, dense (bs_row_ptr == nullptr) or over CSR lists of active 128 x 128 blocks.
 af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
                    const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
-                   int gqa_group, float softmax_scale, const int* bs_row_ptr, const int* bs_col_idx, void* o,
-                   af_dtype o_dtype, float* lse, void* cuda_stream) {
+                   int gqa_group, float softmax_scale, const int* bs_row_ptr, const int* bs_col_idx,
+                   const int* bs_order, void* o, af_dtype o_dtype, float* lse, void* cuda_stream) {
     af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
     if (st != AF_OK) return st;
     if (!q || !k || !v || !o) return AF_ERR_NULL;
@@ -395,6 +396,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     p.pair_heads = 0;
     p.bs_row_ptr = bs_row_ptr;
     p.bs_col_idx = bs_col_idx;
+    p.bs_order = bs_order;
 #ifdef AF_TRACE
     p.trace = reinterpret_cast<long long*>(getenv("AF_TRACE_PTR") ? strtoull(getenv("AF_TRACE_PTR"), nullptr, 0) : 0ull);
     cudaMemcpyToSymbol(af::g_trace, &p.trace, sizeof(p.trace));
@@ -418,8 +420,8 @@ extern "C" {
 af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
                        const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
                        int gqa_group, float softmax_scale, void* o, af_dtype o_dtype, float* lse, void* cuda_stream) {
-    return fwd_impl(shape, q, k, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, nullptr, nullptr, o,
-                    o_dtype, lse, cuda_stream);
+    return fwd_impl(shape, q, k, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, nullptr, nullptr, nullptr,
+                    o, o_dtype, lse, cuda_stream);
 }
 
 af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
@@ -429,7 +431,7 @@ af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* 
     if (!blocks || !blocks->row_ptr || !blocks->col_idx) return AF_ERR_NULL;
     if (blocks->block != 128) return AF_ERR_SPEC;
     return fwd_impl(shape, q, k, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, blocks->row_ptr,
-                    blocks->col_idx, o, o_dtype, lse, cuda_stream);
+                    blocks->col_idx, blocks->row_order, o, o_dtype, lse, cuda_stream);
 }
 
 size_t attnfuse_fwd_host_staging_bytes(const af_shape* shape) {
@@ -585,7 +587,7 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     p.table = static_cast<const float2*>(rope_table);
     p.lse = lse;
     p.delta = nullptr; p.out1 = nullptr; p.out2 = nullptr; p.out_f32 = 0; p.store_x = 0;
-    p.bs_ptr = nullptr; p.bs_idx = nullptr;
+    p.bs_ptr = nullptr; p.bs_idx = nullptr; p.bs_order = nullptr;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     float* delta = static_cast<float*>(workspace);
     // rotated-K and rotated-Q caches: used when there is a rotation and the workspace has room behind delta

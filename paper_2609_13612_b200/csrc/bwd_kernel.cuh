@@ -42,6 +42,7 @@ struct BwdParams {
     // query block (its key blocks): ptr [ceil(S/128) + 1], idx [ptr[last]] (device).
     const int* bs_ptr;
     const int* bs_idx;
+    const int* bs_order;   // optional launch order of the stationary blocks (longest lists first), or nullptr
 };
 
 // delta[row] = <dO[row], O[row]>; one 16-byte chunk per thread, D/8 threads per row.
@@ -278,7 +279,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
     const int xh_count = DKV ? p.Hkv : p.Hq;
     const int b = blockIdx.x / xh_count, xh = blockIdx.x - b * xh_count;
     // heaviest tiles first: under a causal mask early key tiles and late query tiles see the most work
-    const int x0 = (DKV ? static_cast<int>(blockIdx.y) : static_cast<int>(gridDim.y - 1 - blockIdx.y)) * 128;
+    const int x0 = ((BS && p.bs_order) ? __ldg(p.bs_order + blockIdx.y)
+                                       : (DKV ? static_cast<int>(blockIdx.y) : static_cast<int>(gridDim.y - 1 - blockIdx.y))) * 128;
     int lo, hi;  // streamed tile range
     if (DKV) qtile_range(ms, x0, lo, hi);
     else tile_range(ms, x0, lo, hi);

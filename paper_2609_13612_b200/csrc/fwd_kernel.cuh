@@ -28,6 +28,7 @@ struct FwdParams {
     // a contiguous tile range; the element mask (causal, window) still applies inside the listed tiles.
     const int* bs_row_ptr;
     const int* bs_col_idx;
+    const int* bs_order;   // optional launch order of the row blocks (longest lists first), or nullptr
 #ifdef AF_TRACE
     long long* trace;
 #endif
@@ -287,7 +288,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
     for (int q = 0; q < NQ; ++q) hq[q] = p.pair_heads ? 2 * u + q : u;
     const int hk = hq[0] / p.group;
-    const int rb = p.n_row_blocks - 1 - static_cast<int>(blockIdx.y);  // heaviest (last) row blocks first
+    // heaviest row blocks first: the last ones under a causal mask; with block lists the caller's order
+    const int rb = (BS && p.bs_order) ? __ldg(p.bs_order + blockIdx.y) : p.n_row_blocks - 1 - static_cast<int>(blockIdx.y);
     const MaskSpec ms{p.S, p.causal, p.window};
 
     int i0[NQ], jlo[NQ], jhi[NQ];
