@@ -96,8 +96,8 @@ int env_int(const char* name, int dflt) {
 }
 
 template <int D, int NQ, bool ROPE, int KS, int VS>
-af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, FwdParams p,
-                             cudaStream_t stream) {
+af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                             FwdParams p, cudaStream_t stream) {
     using L = FwdSmem<D, NQ, KS, VS>;
     auto kern = attn_fwd_kernel<D, NQ, ROPE, KS, VS>;
     static bool configured = false;
@@ -111,7 +111,7 @@ af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const
     const int rows_per_cta = p.pair_heads ? BM : BM * NQ;
     p.n_row_blocks = (p.S + rows_per_cta - 1) / rows_per_cta;
     dim3 grid(p.pair_heads ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
-    kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, p);
+    kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, to, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
@@ -149,8 +149,8 @@ af_status launch_fwd2_variant(const CUtensorMap& tq, const CUtensorMap& tk2, con
 // Block-sparse variant (Section 4.6): the grid is (heads or head pairs, 128-row blocks); every CTA walks the
 // list of active key blocks of its row block.  An even GQA group pairs two heads per CTA, otherwise one head.
 template <int D, int NQ, bool ROPE>
-af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, FwdParams p,
-                                    cudaStream_t stream) {
+af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                                    const CUtensorMap& to, FwdParams p, cudaStream_t stream) {
     using L = FwdSmem<D, NQ, 2, 2>;
     auto kern = attn_fwd_kernel<D, NQ, ROPE, 2, 2, true>;
     static bool configured = false;
@@ -162,29 +162,29 @@ af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk
     p.pair_heads = NQ == 2 ? 1 : 0;
     p.n_row_blocks = (p.S + BM - 1) / BM;
     dim3 grid(NQ == 2 ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
-    kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, p);
+    kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, to, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 template <int D>
-af_status launch_fwd_blocks(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
-                            cudaStream_t stream) {
+af_status launch_fwd_blocks(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                            const FwdParams& p, cudaStream_t stream) {
     if ((p.group % 2) == 0)
-        return p.R > 0 ? launch_fwd_blocks_variant<D, 2, true>(tq, tk, tv, p, stream)
-                       : launch_fwd_blocks_variant<D, 2, false>(tq, tk, tv, p, stream);
-    return p.R > 0 ? launch_fwd_blocks_variant<D, 1, true>(tq, tk, tv, p, stream)
-                   : launch_fwd_blocks_variant<D, 1, false>(tq, tk, tv, p, stream);
+        return p.R > 0 ? launch_fwd_blocks_variant<D, 2, true>(tq, tk, tv, to, p, stream)
+                       : launch_fwd_blocks_variant<D, 2, false>(tq, tk, tv, to, p, stream);
+    return p.R > 0 ? launch_fwd_blocks_variant<D, 1, true>(tq, tk, tv, to, p, stream)
+                   : launch_fwd_blocks_variant<D, 1, false>(tq, tk, tv, to, p, stream);
 }
 
 template <int D>
-af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
+af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const FwdParams& p,
                      cudaStream_t stream) {
     const int nq = env_int("AF_FWD_NQ", 2);
     if (nq == 1) {
-        return p.R > 0 ? launch_fwd_variant<D, 1, true, 2, 2>(tq, tk, tv, p, stream)
-                       : launch_fwd_variant<D, 1, false, 2, 2>(tq, tk, tv, p, stream);
+        return p.R > 0 ? launch_fwd_variant<D, 1, true, 2, 2>(tq, tk, tv, to, p, stream)
+                       : launch_fwd_variant<D, 1, false, 2, 2>(tq, tk, tv, to, p, stream);
     }
-    return p.R > 0 ? launch_fwd_variant<D, 2, true, 2, 2>(tq, tk, tv, p, stream)
-                   : launch_fwd_variant<D, 2, false, 2, 2>(tq, tk, tv, p, stream);
+    return p.R > 0 ? launch_fwd_variant<D, 2, true, 2, 2>(tq, tk, tv, to, p, stream)
+                   : launch_fwd_variant<D, 2, false, 2, 2>(tq, tk, tv, to, p, stream);
 }
 
 template <int D, bool DKV, bool ROT_X, bool ROT_A, bool BS>
@@ -378,10 +378,17 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     if ((st = resolve_strides(skv, shape->Hkv, shape->S, shape->D, &stkv)) != AF_OK) return st;
     if ((st = check_arch()) != AF_OK) return st;
 
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     if ((st = make_tmap(&tq, q, shape->B, shape->Hq, shape->S, shape->D, stq, BM)) != AF_OK) return st;
     if ((st = make_tmap(&tk, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, BN)) != AF_OK) return st;
     if ((st = make_tmap(&tv, v, shape->B, shape->Hkv, shape->S, shape->D, stkv, BN)) != AF_OK) return st;
+    // bf16 output goes out through TMA (contiguous [B,Hq,S,D]); with fp32 output the map is not used
+    to = tq;
+    if (o_dtype == AF_BF16) {
+        af_strides sto;
+        resolve_strides(nullptr, shape->Hq, shape->S, shape->D, &sto);
+        if ((st = make_tmap(&to, o, shape->B, shape->Hq, shape->S, shape->D, sto, BM)) != AF_OK) return st;
+    }
 
     FwdParams p;
     p.B = shape->B; p.Hq = shape->Hq; p.Hkv = shape->Hkv; p.S = shape->S; p.group = gqa_group;
@@ -403,7 +410,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
 #endif
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (bs_row_ptr)
-        return shape->D == 128 ? launch_fwd_blocks<128>(tq, tk, tv, p, stream) : launch_fwd_blocks<64>(tq, tk, tv, p, stream);
+        return shape->D == 128 ? launch_fwd_blocks<128>(tq, tk, tv, to, p, stream) : launch_fwd_blocks<64>(tq, tk, tv, to, p, stream);
     const int R = rope->rotary_dim;
     const bool pair_ok = shape->D == 128 && (gqa_group % 4) == 0 && (R == 0 || R == 16 || R == 32 || R == 64 || R == 128);
     if (pair_ok && env_int("AF_FWD_2CTA", 0)) {
@@ -411,7 +418,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
         if ((st = make_tmap(&tk2, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, 64)) != AF_OK) return st;
         return R > 0 ? launch_fwd2_variant<true>(tq, tk2, tv, p, stream) : launch_fwd2_variant<false>(tq, tk2, tv, p, stream);
     }
-    return shape->D == 128 ? launch_fwd<128>(tq, tk, tv, p, stream) : launch_fwd<64>(tq, tk, tv, p, stream);
+    return shape->D == 128 ? launch_fwd<128>(tq, tk, tv, to, p, stream) : launch_fwd<64>(tq, tk, tv, to, p, stream);
 }
 }  // namespace
 

@@ -261,7 +261,7 @@ __device__ __forceinline__ bool softmax_tile_halves(uint32_t tS, uint32_t tO, in
 template <int D, int NQ, bool ROPE, int KS, int VS, bool BS = false>
 __global__ void __launch_bounds__(128 * (2 + NQ), 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const FwdParams p) {
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const FwdParams p) {
     using L = FwdSmem<D, NQ, KS, VS>;
     constexpr int TILE = L::TILE;
     constexpr int NBOX = D / BOX_COLS;
@@ -587,8 +587,37 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tc_fence_after_sync();
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
             const size_t orow = (static_cast<size_t>(bh) * p.S + i) * D;
+            if (!p.o_f32) {
+                // bf16 output: stage the tile in shared memory - in this query tile's own Q buffer, which no MMA
+                // reads any more once O is complete, in the layout of the input tiles - and let TMA write it out.
+                // (Row-per-thread global stores touch 32 rows per instruction and kept the load/store unit busy
+                // for ~4 k cycles per CTA.)  Rows past S are clipped by the tensor map.
+                uint8_t* stg = sQ + q * TILE;
 #pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tO + c * 32, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8)
+                        *reinterpret_cast<uint4*>(stg + swz_chunk_offset(row, c * 4 + (e >> 3))) = make_uint4(
+                            pack_bf16x2(__uint_as_float(v[e]) * inv, __uint_as_float(v[e + 1]) * inv),
+                            pack_bf16x2(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv),
+                            pack_bf16x2(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv),
+                            pack_bf16x2(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv));
+                }
+                fence_proxy_async_smem();
+                asm volatile("bar.sync %0, 128;" ::"r"(4 + q) : "memory");   // this warpgroup only
+                if (row == 0) {
+#pragma unroll
+                    for (int bx = 0; bx < NBOX; ++bx)
+                        tma_store_4d(&tm_o, stg + bx * BOX_BYTES, bx * BOX_COLS, i0[q], hq[q], b);
+                    tma_store_commit();
+                    tma_store_wait_read();   // the buffer must stay in place until it has been read
+                }
+            }
+#pragma unroll 1
+            for (int c = 0; p.o_f32 && c < D / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld32(tO + c * 32, v);
                 tmem_wait_ld();
