@@ -38,7 +38,7 @@ UNIT = "TFLOP/s"
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes per launch of the forward kernel on this workload, from the ncu capture summarised in
 # profiles/attn_fwd_kernel_c2_llama3_8b.md (dram__bytes_read.sum + dram__bytes_write.sum).
-FWD_TRAFFIC_BYTES_PER_LAUNCH = 56.5e6
+FWD_TRAFFIC_BYTES_PER_LAUNCH = 55.3e6
 PAPER_CONTEXT = {
     "rtx3090_fused_vs_flex_prerotate_rope_causal": "2.10x (RTX 3090, fp16, B=4 H=12 D=64, N=4096)",
     "h100_llama3_8b_training_step_vs_sdpa": "within ~5% (H100 NVL, fp16, N=2048: 7.65 ms vs 7.27 ms)",
