@@ -69,85 +69,10 @@ struct FwdSmem {
 #define AF_STAMP_SM(ph) do { } while (0)
 #endif
 
-#ifndef AF_POLY_EVERY
-#define AF_POLY_EVERY 0
-#endif
 #ifdef AF_TRACE
 __device__ long long* g_trace = nullptr;
 #endif
-constexpr int kPolyEvery = AF_POLY_EVERY;   // share of exps computed by polynomial: 1 in kPolyEvery pairs (0: none)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the row max grows by more
-
-// One key tile of the online softmax for one query row (this thread's TMEM lane): reads the 128
-// raw scores, adds ALiBi and the mask in the raw domain, updates the running max and sum in the
-// log2 domain, writes P (bf16) over S and, when the reference max moved, rescales O.
-// MASKED / ALIBI select straight-line code: interior tiles carry no mask logic at all.
-//   score (log2 domain) t_e = c2 * (S_e + kb * e) + bias0,  kb = slope2 / c2, bias0 = slope2 * (j0 - i)
-template <int D, bool MASKED, bool ALIBI>
-__device__ __forceinline__ void softmax_tile(uint32_t tS, uint32_t tO, int n, float scale_log2, float kb,
-                                             float bias0, int mlo, uint32_t mn, float& m_run, float& l_run) {
-    uint32_t v[BN];
-    tmem_ld32(tS, v);
-    tmem_ld32(tS + 32, v + 32);
-    tmem_ld32(tS + 64, v + 64);
-    tmem_ld32(tS + 96, v + 96);
-    tmem_wait_ld();
-    AF_STAMP_SM(3);
-    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-    for (int e = 0; e < BN; e += 2) {
-        float sv[2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            sv[u] = __uint_as_float(v[e + u]);
-            if (ALIBI) sv[u] = fmaf(kb, static_cast<float>(e + u), sv[u]);
-            if (MASKED) sv[u] = (static_cast<uint32_t>(e + u - mlo) < mn) ? sv[u] : -INFINITY;
-            if (ALIBI || MASKED) v[e + u] = __float_as_uint(sv[u]);
-        }
-        mx4[(e >> 1) & 3] = fmax3(mx4[(e >> 1) & 3], sv[0], sv[1]);   // two scores per instruction
-    }
-    // scale > 0, so the max commutes with it
-    const float mx = fmaf(fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]), scale_log2, bias0);
-    AF_STAMP_SM(4);
-    // lazy rescale: keep the old reference max unless it grew by more than the threshold
-    const bool upd = mx > m_run + kRescaleThreshold;
-    float alpha = 1.f;
-    if (upd) {
-        alpha = ex2(m_run - mx);  // m_run = -inf -> 0
-        m_run = mx;
-    }
-    const float sub = bias0 - ((m_run == -INFINITY) ? 0.f : m_run);
-    const float2 sc2 = make_float2(scale_log2, scale_log2), sub2 = make_float2(sub, sub);
-    float2 ps2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-    uint32_t pk[BN / 2];
-#pragma unroll
-    for (int e = 0; e < BN; e += 2) {
-        // packed fp32: one instruction scales and shifts two scores, one adds two probabilities
-        const float2 t = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), sc2, sub2);
-        // every kPolyEvery-th pair takes the polynomial on the FMA pipe, the rest the special-function unit
-        const float2 pe = (kPolyEvery > 0 && ((e >> 1) % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) ? ex2_poly2(t)
-                                                                                               : make_float2(ex2(t.x), ex2(t.y));
-        ps2[(e >> 1) & 1] = __fadd2_rn(ps2[(e >> 1) & 1], pe);
-        pk[e >> 1] = pack_bf16x2(pe.x, pe.y);
-    }
-    tmem_st32(tS, pk);
-    tmem_st32(tS + 32, pk + 32);
-    AF_STAMP_SM(5);
-    l_run = l_run * alpha + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
-    if (n > 0 && __any_sync(0xffffffffu, upd)) {
-#pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            tmem_ld32(tO + c * 32, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(tO + c * 32, o);
-        }
-    }
-    tmem_wait_st();
-    AF_STAMP_SM(6);
-}
 
 #ifndef AF_SPLIT_S
 #define AF_SPLIT_S 0
@@ -158,7 +83,12 @@ constexpr bool kSplitS = AF_SPLIT_S != 0;   // S tile produced as two N = 64 hal
 #endif
 constexpr int kPParts = AF_P_PARTS;          // P is handed to the MMA issuer in this many column parts (2 or 4)
 
-// The same tile step with the work handed over in column halves, so that less of it sits on the
+// One key tile of the online softmax for one query row (this thread's TMEM lane): reads the 128
+// raw scores, adds ALiBi and the mask in the raw domain, updates the running max and sum in the
+// log2 domain, writes P (bf16) over S and, when the reference max moved, rescales O.
+// MASKED / ALIBI select straight-line code: interior tiles carry no mask logic at all.
+//   score (log2 domain) t_e = c2 * (S_e + kb * e) + bias0,  kb = slope2 / c2, bias0 = slope2 * (j0 - i)
+// The work is handed over in column halves, so that less of it sits on the
 // S-MMA -> softmax -> PV-MMA dependency chain of a query tile:
 //  - with kSplitS the scores arrive as two 64-column halves (two barriers): the TMEM load of the first
 //    half overlaps the MMAs of the second;

@@ -356,24 +356,6 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// 2^x for two values on the FMA pipe instead of the special-function unit (which two softmax warps of
-// a sub-partition share and which is as busy as the tensor pipe in attention): round to nearest integer
-// with the magic-number trick, degree-3 minimax polynomial for 2^f on [-0.5, 0.5] (max relative error
-// 7.5e-5, far below the bf16 rounding of P), integer part added into the exponent field.  Packed fp32.
-__device__ __forceinline__ float2 ex2_poly2(float2 x) {
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
-    const float2 r = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));          // 1.5 * 2^23: low bits = rint(x)
-    const float2 fl = __fadd2_rn(r, make_float2(-12582912.f, -12582912.f));
-    const float2 f = __ffma2_rn(fl, make_float2(-1.f, -1.f), x);
-    float2 p = __ffma2_rn(f, make_float2(0.0551716472f, 0.0551716472f), make_float2(0.242611121f, 0.242611121f));
-    p = __ffma2_rn(p, f, make_float2(0.693260989f, 0.693260989f));
-    p = __ffma2_rn(p, f, make_float2(0.999928074f, 0.999928074f));
-    p.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23));
-    p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23));
-    return p;
-}
-
 // max of three in one instruction (sm_100)
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float r;
