@@ -69,7 +69,10 @@ af_status attnfuse_device_status(unsigned int* detail);
 /* ---- cos/sin table (set-up step of Section 4.1; cached by the caller) --------------------------
  * table: S * rotary_dim/2 pairs of fp32 {cos, sin}(p * theta^(-2i/rotary_dim)), p = pos_offset + s,
  * row-major [S][rotary_dim/2]; angles are formed in fp64 before rounding.  One extra trailer row
- * holds the row-to-row step constants the fused kernels use.
+ * holds the row-to-row step constants the fused kernels use.  Behind these rows (at the next multiple
+ * of 256 bytes) the buffer carries a bf16 copy, S rows of [rotary_dim/2 cos | rotary_dim/2 sin], for
+ * the forward kernel's optional packed-bf16 key rotation (environment switch AF_FWD_KEYS_BF16=1:
+ * faster, about 1.4 times the rounding error on rotated keys; forward only, off by default).
  * attnfuse_rope_table_bytes returns the size the caller must provide (0 when rotary_dim = 0). */
 size_t    attnfuse_rope_table_bytes(int S, int rotary_dim);
 af_status attnfuse_rope_table(const af_rope* rope, int S, void* table, void* cuda_stream);

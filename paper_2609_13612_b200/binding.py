@@ -159,7 +159,8 @@ def rope_table(rope_spec: RopeSpec, S: int, device=None) -> Optional[torch.Tenso
     table = torch.empty(n // 4, dtype=torch.float32, device=device)
     r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
     _check(lib().attnfuse_rope_table(ctypes.byref(r), S, table.data_ptr(), _stream()))
-    return table.view(S + 1, rope_spec.rotary_dim // 2, 2)
+    # the fp32 rows; the buffer behind this view also carries the bf16 copy the forward kernel streams by TMA
+    return table[: (S + 1) * rope_spec.rotary_dim].view(S + 1, rope_spec.rotary_dim // 2, 2)
 
 
 def rope(x: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor], inverse: bool = False,

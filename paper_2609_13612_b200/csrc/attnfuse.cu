@@ -52,6 +52,41 @@ af_status make_tmap(CUtensorMap* tm, const void* ptr, int B, int H, int S, int D
     return r == CUDA_SUCCESS ? AF_OK : AF_ERR_CUDA;
 }
 
+// Byte offset of the bf16 copy of the cos/sin table inside the table buffer: after the fp32 rows (S positions
+// and the trailer), rounded up to 256 bytes.  Its rows are [R/2 cos | R/2 sin] in bf16, 2 R bytes each.
+size_t table_bf16_offset(int S, int R) {
+    const size_t f32 = static_cast<size_t>(S + 1) * (R / 2) * sizeof(float2);
+    return (f32 + 255) & ~static_cast<size_t>(255);
+}
+
+// Tensor map over that copy: [S rows][R columns] bf16, box of 128 rows x R columns, no swizzle, zero fill.
+af_status make_tmap_table(CUtensorMap* tm, const void* table, int S, int R) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return AF_ERR_CUDA;
+    cuuint64_t dims[2] = {static_cast<cuuint64_t>(R), static_cast<cuuint64_t>(S)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(R) * 2};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(R), 128};
+    cuuint32_t estr[2] = {1, 1};
+    void* base = const_cast<uint8_t*>(static_cast<const uint8_t*>(table) + table_bf16_offset(S, R));
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? AF_OK : AF_ERR_CUDA;
+}
+
+int env_int(const char* name, int dflt) {
+    const char* v = getenv(name);
+    return v ? atoi(v) : dflt;
+}
+
+// AF_FWD_KEYS_BF16=1 (forward only, rotary widths 16, 32, 64, 128): key tiles are rotated in packed bf16
+// arithmetic from the table's bf16 copy instead of fp32 arithmetic from the fp32 rows.  Faster (the rotation
+// competes with the softmax for issue slots), but a rotated key then carries about three bf16 roundings instead
+// of one; the backward pass always rotates in fp32, so a log-sum-exp produced in this mode is slightly
+// inconsistent with the scores the backward pass recomputes.  Off by default.
+bool keys_rotate_in_bf16(int R) {
+    return (R == 16 || R == 32 || R == 64 || R == 128) && env_int("AF_FWD_KEYS_BF16", 0);
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 af_status check_arch() {
@@ -90,16 +125,11 @@ af_status resolve_strides(const af_strides* in, int H, int S, int D, af_strides*
     return AF_OK;
 }
 
-int env_int(const char* name, int dflt) {
-    const char* v = getenv(name);
-    return v ? atoi(v) : dflt;
-}
-
-template <int D, int NQ, bool ROPE, int KS, int VS>
-af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+template <int D, int NQ, bool ROPE, int KS, int VS, bool TAB = false>
+af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const CUtensorMap& tt,
                              FwdParams p, cudaStream_t stream) {
-    using L = FwdSmem<D, NQ, KS, VS>;
-    auto kern = attn_fwd_kernel<D, NQ, ROPE, KS, VS>;
+    using L = FwdSmem<D, NQ, KS, VS, ROPE && TAB>;
+    auto kern = attn_fwd_kernel<D, NQ, ROPE, KS, VS, false, TAB>;
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
@@ -111,7 +141,7 @@ af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const
     const int rows_per_cta = p.pair_heads ? BM : BM * NQ;
     p.n_row_blocks = (p.S + rows_per_cta - 1) / rows_per_cta;
     dim3 grid(p.pair_heads ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
-    kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, to, p);
+    kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, to, tt, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
@@ -150,7 +180,7 @@ af_status launch_fwd2_variant(const CUtensorMap& tq, const CUtensorMap& tk2, con
 // list of active key blocks of its row block.  An even GQA group pairs two heads per CTA, otherwise one head.
 template <int D, int NQ, bool ROPE>
 af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                                    const CUtensorMap& to, FwdParams p, cudaStream_t stream) {
+                                    const CUtensorMap& to, const CUtensorMap& tt, FwdParams p, cudaStream_t stream) {
     using L = FwdSmem<D, NQ, 2, 2>;
     auto kern = attn_fwd_kernel<D, NQ, ROPE, 2, 2, true>;
     static bool configured = false;
@@ -162,29 +192,30 @@ af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk
     p.pair_heads = NQ == 2 ? 1 : 0;
     p.n_row_blocks = (p.S + BM - 1) / BM;
     dim3 grid(NQ == 2 ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
-    kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, to, p);
+    kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, to, tt, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 template <int D>
-af_status launch_fwd_blocks(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+af_status launch_fwd_blocks(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const CUtensorMap& tt,
                             const FwdParams& p, cudaStream_t stream) {
     if ((p.group % 2) == 0)
-        return p.R > 0 ? launch_fwd_blocks_variant<D, 2, true>(tq, tk, tv, to, p, stream)
-                       : launch_fwd_blocks_variant<D, 2, false>(tq, tk, tv, to, p, stream);
-    return p.R > 0 ? launch_fwd_blocks_variant<D, 1, true>(tq, tk, tv, to, p, stream)
-                   : launch_fwd_blocks_variant<D, 1, false>(tq, tk, tv, to, p, stream);
+        return p.R > 0 ? launch_fwd_blocks_variant<D, 2, true>(tq, tk, tv, to, tt, p, stream)
+                       : launch_fwd_blocks_variant<D, 2, false>(tq, tk, tv, to, tt, p, stream);
+    return p.R > 0 ? launch_fwd_blocks_variant<D, 1, true>(tq, tk, tv, to, tt, p, stream)
+                   : launch_fwd_blocks_variant<D, 1, false>(tq, tk, tv, to, tt, p, stream);
 }
 
 template <int D>
-af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const FwdParams& p,
+af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const CUtensorMap& tt, const FwdParams& p,
                      cudaStream_t stream) {
     const int nq = env_int("AF_FWD_NQ", 2);
     if (nq == 1) {
-        return p.R > 0 ? launch_fwd_variant<D, 1, true, 2, 2>(tq, tk, tv, to, p, stream)
-                       : launch_fwd_variant<D, 1, false, 2, 2>(tq, tk, tv, to, p, stream);
+        return p.R > 0 ? launch_fwd_variant<D, 1, true, 2, 2>(tq, tk, tv, to, tt, p, stream)
+                       : launch_fwd_variant<D, 1, false, 2, 2>(tq, tk, tv, to, tt, p, stream);
     }
-    return p.R > 0 ? launch_fwd_variant<D, 2, true, 2, 2>(tq, tk, tv, to, p, stream)
-                   : launch_fwd_variant<D, 2, false, 2, 2>(tq, tk, tv, to, p, stream);
+    if (p.R > 0 && keys_rotate_in_bf16(p.R)) return launch_fwd_variant<D, 2, true, 2, 2, true>(tq, tk, tv, to, tt, p, stream);
+    return p.R > 0 ? launch_fwd_variant<D, 2, true, 2, 2>(tq, tk, tv, to, tt, p, stream)
+                   : launch_fwd_variant<D, 2, false, 2, 2>(tq, tk, tv, to, tt, p, stream);
 }
 
 template <int D, bool DKV, bool ROT_X, bool ROT_A, bool BS>
@@ -318,7 +349,8 @@ af_status attnfuse_device_status(unsigned int* detail) {
 
 size_t attnfuse_rope_table_bytes(int S, int rotary_dim) {
     if (S < 1 || rotary_dim < 1) return 0;
-    return static_cast<size_t>(S + 1) * (rotary_dim / 2) * sizeof(float2);  // + one trailer row
+    // fp32 rows (+ one trailer row), then the bf16 copy the forward kernel streams by TMA
+    return table_bf16_offset(S, rotary_dim) + static_cast<size_t>(S) * rotary_dim * 2;
 }
 
 af_status attnfuse_rope_table(const af_rope* rope, int S, void* table, void* cuda_stream) {
@@ -333,7 +365,9 @@ af_status attnfuse_rope_table(const af_rope* rope, int S, void* table, void* cud
     const int threads = 256;
     const unsigned blocks = static_cast<unsigned>((n + threads - 1) / threads);
     rope_table_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-        static_cast<float2*>(table), S, rope->rotary_dim, static_cast<double>(rope->theta), rope->pos_offset);
+        static_cast<float2*>(table),
+        reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(table) + table_bf16_offset(S, rope->rotary_dim)), S,
+        rope->rotary_dim, static_cast<double>(rope->theta), rope->pos_offset);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
@@ -390,6 +424,11 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
         if ((st = make_tmap(&to, o, shape->B, shape->Hq, shape->S, shape->D, sto, BM)) != AF_OK) return st;
     }
 
+    // (optional mode) key tiles receive the 128 rows of the table's bf16 copy that belong to them by TMA
+    const int Rr = rope->rotary_dim;
+    CUtensorMap tt = tq;
+    if (keys_rotate_in_bf16(Rr) && (st = make_tmap_table(&tt, rope_table, shape->S, Rr)) != AF_OK) return st;
+
     FwdParams p;
     p.B = shape->B; p.Hq = shape->Hq; p.Hkv = shape->Hkv; p.S = shape->S; p.group = gqa_group;
     p.R = rope->rotary_dim;
@@ -410,7 +449,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
 #endif
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (bs_row_ptr)
-        return shape->D == 128 ? launch_fwd_blocks<128>(tq, tk, tv, to, p, stream) : launch_fwd_blocks<64>(tq, tk, tv, to, p, stream);
+        return shape->D == 128 ? launch_fwd_blocks<128>(tq, tk, tv, to, tt, p, stream) : launch_fwd_blocks<64>(tq, tk, tv, to, tt, p, stream);
     const int R = rope->rotary_dim;
     const bool pair_ok = shape->D == 128 && (gqa_group % 4) == 0 && (R == 0 || R == 16 || R == 32 || R == 64 || R == 128);
     if (pair_ok && env_int("AF_FWD_2CTA", 0)) {
@@ -418,7 +457,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
         if ((st = make_tmap(&tk2, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, 64)) != AF_OK) return st;
         return R > 0 ? launch_fwd2_variant<true>(tq, tk2, tv, p, stream) : launch_fwd2_variant<false>(tq, tk2, tv, p, stream);
     }
-    return shape->D == 128 ? launch_fwd<128>(tq, tk, tv, to, p, stream) : launch_fwd<64>(tq, tk, tv, to, p, stream);
+    return shape->D == 128 ? launch_fwd<128>(tq, tk, tv, to, tt, p, stream) : launch_fwd<64>(tq, tk, tv, to, tt, p, stream);
 }
 }  // namespace
 

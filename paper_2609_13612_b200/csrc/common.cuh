@@ -224,6 +224,54 @@ __device__ __forceinline__ void rotate_tile_fast(uint8_t* tile, RotState<CP>& st
     }
 }
 
+// Table-tile variant of the same rotation, an optional mode for the streamed key tiles of the forward kernel:
+// the cos/sin values of the tile's 128 positions arrive by TMA from the bf16 copy of the table (row layout
+// [R/2 cos | R/2 sin], densely packed, row r at byte 2 R r) and the arithmetic runs on packed bf16 pairs, four
+// multiply-adds per pair of words.  It needs about a quarter of the issue slots of rotate_tile_fast, which
+// matters because the rotation shares its schedulers with the softmax warps.  The result is rounded to bf16 in
+// either variant; here the table entries and the sine product carry one more bf16 rounding each, which makes the
+// rounding error of a rotated key about 1.4 times that of the fp32 arithmetic.
+__device__ __forceinline__ void rotate_word_bf16(uint32_t& a, uint32_t& b, uint32_t c, uint32_t s) {
+    const __nv_bfloat162 A = *reinterpret_cast<const __nv_bfloat162*>(&a), B = *reinterpret_cast<const __nv_bfloat162*>(&b);
+    const __nv_bfloat162 C = *reinterpret_cast<const __nv_bfloat162*>(&c), Sn = *reinterpret_cast<const __nv_bfloat162*>(&s);
+    const __nv_bfloat162 na = __hfma2(__hneg2(B), Sn, __hmul2(A, C));   // a cos - b sin
+    const __nv_bfloat162 nb = __hfma2(A, Sn, __hmul2(B, C));            // b cos + a sin
+    a = *reinterpret_cast<const uint32_t*>(&na);
+    b = *reinterpret_cast<const uint32_t*>(&nb);
+}
+template <int CP>
+__device__ __forceinline__ void rotate_tile_tab(uint8_t* tile, const uint8_t* tab, int tid) {
+    constexpr int RP = 128 / CP;
+    constexpr int ROW_BYTES = CP * 32;       // 2 R
+    constexpr int NB = CP < 2 ? CP : 2;      // rows in flight per thread
+    const int rg = tid / CP, cp = tid % CP;
+#pragma unroll
+    for (int k0 = 0; k0 < CP; k0 += NB) {
+        uint4 lo[NB], hi[NB], c[NB], s[NB];
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+            const int r = rg + RP * (k0 + u);
+            lo[u] = *reinterpret_cast<const uint4*>(tile + swz_chunk_offset(r, cp));
+            hi[u] = *reinterpret_cast<const uint4*>(tile + swz_chunk_offset(r, cp + CP));
+            c[u] = *reinterpret_cast<const uint4*>(tab + r * ROW_BYTES + cp * 16);
+            s[u] = *reinterpret_cast<const uint4*>(tab + r * ROW_BYTES + CP * 16 + cp * 16);
+        }
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+            rotate_word_bf16(lo[u].x, hi[u].x, c[u].x, s[u].x);
+            rotate_word_bf16(lo[u].y, hi[u].y, c[u].y, s[u].y);
+            rotate_word_bf16(lo[u].z, hi[u].z, c[u].z, s[u].z);
+            rotate_word_bf16(lo[u].w, hi[u].w, c[u].w, s[u].w);
+        }
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+            const int r = rg + RP * (k0 + u);
+            *reinterpret_cast<uint4*>(tile + swz_chunk_offset(r, cp)) = lo[u];
+            *reinterpret_cast<uint4*>(tile + swz_chunk_offset(r, cp + CP)) = hi[u];
+        }
+    }
+}
+
 // The same walk restricted to a share of the rows: with PARTS warpgroups working on one tile, part p
 // takes the rows rg + RP * k for k in [p * CP / PARTS, (p + 1) * CP / PARTS).  Used where otherwise idle
 // warpgroups rotate a stationary tile together.  (CP < PARTS: part 0 does everything.)

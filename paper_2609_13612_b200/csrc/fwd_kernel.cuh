@@ -34,18 +34,21 @@ struct FwdParams {
 #endif
 };
 
-template <int D, int NQ, int KS, int VS>
+template <int D, int NQ, int KS, int VS, bool TAB = false>
 struct FwdSmem {
     static constexpr int TILE = 128 * D * 2;
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + NQ * TILE;
     static constexpr int OFF_V = OFF_K + KS * TILE;
-    static constexpr int OFF_BAR = OFF_V + VS * TILE;
+    // TAB: one stage for the bf16 cos/sin rows of a key tile's 128 positions ([R/2 cos | R/2 sin] per row, R <= D)
+    static constexpr int OFF_T = OFF_V + VS * TILE;
+    static constexpr int T_BYTES = TAB ? 128 * 2 * D : 0;
+    static constexpr int OFF_BAR = OFF_T + T_BYTES;
     // barrier slots
     static constexpr int B_QFULL = 0, B_QROT = B_QFULL + NQ, B_KFULL = B_QROT + NQ, B_KROT = B_KFULL + KS,
                          B_KEMPTY = B_KROT + KS, B_VFULL = B_KEMPTY + KS, B_VEMPTY = B_VFULL + VS,
                          B_SFULL = B_VEMPTY + VS, B_PREADY = B_SFULL + 2 * NQ, B_ODONE = B_PREADY + 4 * NQ,   // SFULL: per column half; PREADY: per P part (up to 4)
-                         N_BARS = B_ODONE + NQ;
+                         B_TFULL = B_ODONE + NQ, B_TEMPTY = B_TFULL + 1, N_BARS = B_TEMPTY + 1;
     static constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;
     static constexpr int BYTES = OFF_MISC + 16 + 1024;  // + alignment slack
 };
@@ -188,11 +191,14 @@ __device__ __forceinline__ bool softmax_tile_halves(uint32_t tS, uint32_t tO, in
     return true;
 }
 
-template <int D, int NQ, bool ROPE, int KS, int VS, bool BS = false>
+// TAB (with ROPE): key tiles are rotated in packed bf16 arithmetic from table tiles that arrive by TMA through
+// tm_t (the bf16 copy of the cos/sin table); otherwise in fp32 arithmetic from the fp32 table rows.
+template <int D, int NQ, bool ROPE, int KS, int VS, bool BS = false, bool TAB = false>
 __global__ void __launch_bounds__(128 * (2 + NQ), 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const FwdParams p) {
-    using L = FwdSmem<D, NQ, KS, VS>;
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                const __grid_constant__ CUtensorMap tm_t, const FwdParams p) {
+    using L = FwdSmem<D, NQ, KS, VS, ROPE && TAB>;
     constexpr int TILE = L::TILE;
     constexpr int NBOX = D / BOX_COLS;
     constexpr uint32_t TMEM_COLS = (NQ * (BN + D) <= 256) ? 256u : 512u;
@@ -204,6 +210,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     uint8_t* sQ = smem + L::OFF_Q;
     uint8_t* sK = smem + L::OFF_K;
     uint8_t* sV = smem + L::OFF_V;
+    uint8_t* sT = smem + L::OFF_T;
+    constexpr bool tab_tiles = ROPE && TAB;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_MISC + 4);
@@ -258,7 +266,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int i = 0; i < L::N_BARS; ++i) {
             uint32_t cnt = 1;
             if ((i >= L::B_QROT && i < L::B_QROT + NQ) || (i >= L::B_KROT && i < L::B_KROT + KS) ||
-                (i >= L::B_PREADY && i < L::B_PREADY + 4 * NQ))
+                (i >= L::B_PREADY && i < L::B_PREADY + 4 * NQ) || i == L::B_TEMPTY)
                 cnt = 4;  // one elected arrive per warp of the producing warpgroup
             mbar_init(&bars[i], cnt);
         }
@@ -287,6 +295,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             prefetch_tmap(&tm_q);
             prefetch_tmap(&tm_k);
             prefetch_tmap(&tm_v);
+            if (tab_tiles) prefetch_tmap(&tm_t);
 #pragma unroll
             for (int q = 0; q < NQ; ++q) {
                 if (jhi[q] < jlo[q]) continue;
@@ -303,6 +312,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                 for (int bx = 0; bx < NBOX; ++bx)
                     tma_load_4d(sK + ks * TILE + bx * BOX_BYTES, &tm_k, &bars[L::B_KFULL + ks], bx * BOX_COLS, j0, hk, b);
+                if (tab_tiles) {
+                    // the single table stage is free once the previous tile has been rotated
+                    if (!mbar_wait(&bars[L::B_TEMPTY], (it & 1) ^ 1, abort_flag, 12)) break;
+                    mbar_arrive_expect_tx(&bars[L::B_TFULL], 256u * p.R);
+                    tma_load_2d(sT, &tm_t, &bars[L::B_TFULL], 0, j0);
+                }
                 if (!mbar_wait(&bars[L::B_VEMPTY + vs], ((it / VS) & 1) ^ 1, abort_flag, 2)) break;
                 mbar_arrive_expect_tx(&bars[L::B_VFULL + vs], TILE);
 #pragma unroll
@@ -419,6 +434,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         setmaxnreg_dec<kRotRegs>();
         if (ROPE) {
             const int t = threadIdx.x - 128;
+            // packed bf16 arithmetic on TMA-fed table tiles (rotary widths with a fast path)
+            auto run_tab = [&](auto cp_tag) {
+                constexpr int CP = decltype(cp_tag)::value;
+                bool ok = true;
+                for (int it = 0; ok && it < n_it; ++it) {
+                    const int ks = it % KS;
+                    AF_STAMP(1, it, 0);
+                    ok = mbar_wait_warp(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
+                    if (ok) ok = mbar_wait_warp(&bars[L::B_TFULL], it & 1, abort_flag, 13);
+                    AF_STAMP(1, it, 1);
+                    if (!ok) break;
+                    rotate_tile_tab<CP>(sK + ks * TILE, sT, t);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(&bars[L::B_KROT + ks]);
+                        mbar_arrive(&bars[L::B_TEMPTY]);
+                    }
+                    AF_STAMP(1, it, 2);
+                }
+            };
+            // fp32 arithmetic from the fp32 table rows
             auto run = [&](auto cp_tag) {
                 constexpr int CP = decltype(cp_tag)::value;  // 0: generic path (table read per row)
                 bool ok = true;
@@ -430,7 +467,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int it = 0; ok && it < n_it; ++it) {
                     const int ks = it % KS;
                     // (listed tiles need not be consecutive: the cos/sin state is read for every tile)
-                    if (CP > 0 && (BS || (it % kRotResync) == 0)) rotate_prefetch(st, p.table, tile_at(jlo_c + it) * BN, p.S, p.R, t);
+                    if (CP > 0 && (BS || (it % kRotResync) == 0))
+                        rotate_prefetch(st, p.table, tile_at(jlo_c + it) * BN, p.S, p.R, t);
                     AF_STAMP(1, it, 0);
                     ok = mbar_wait_warp(&bars[L::B_KFULL + ks], (it / KS) & 1, abort_flag, 9);
                     AF_STAMP(1, it, 1);
@@ -443,7 +481,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     AF_STAMP(1, it, 2);
                 }
             };
-            if (p.R == 128) run(std::integral_constant<int, 8>{});
+            if constexpr (tab_tiles) {
+                if (p.R == 128) run_tab(std::integral_constant<int, 8>{});
+                else if (p.R == 64) run_tab(std::integral_constant<int, 4>{});
+                else if (p.R == 32) run_tab(std::integral_constant<int, 2>{});
+                else run_tab(std::integral_constant<int, 1>{});
+            } else if (p.R == 128) run(std::integral_constant<int, 8>{});
             else if (p.R == 64) run(std::integral_constant<int, 4>{});
             else if (p.R == 32) run(std::integral_constant<int, 2>{});
             else if (p.R == 16) run(std::integral_constant<int, 1>{});
@@ -471,6 +514,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             auto rot_q = [&](auto cp_tag) {
                 constexpr int CP = decltype(cp_tag)::value;
                 constexpr int CPT = CP > 0 ? CP : 1;
+                // (fp32 arithmetic: the query tile is rotated once, and every score inherits its rounding)
                 RotStep step;
                 RotState<CPT> st;
                 if (CP > 0) {

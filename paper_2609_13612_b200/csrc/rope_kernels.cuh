@@ -8,7 +8,8 @@ namespace af {
 // table[s][i] = {cos, sin}((p0 + s) * theta^(-2i/R)); the angle is formed in fp64 so that large
 // positions do not lose the fraction of a turn, then rounded to fp32.  One trailer row [S][i] holds
 // {cos, sin}(stride * theta^(-2i/R)), the constant the fused kernels use to walk from row to row.
-__global__ void rope_table_kernel(float2* __restrict__ table, int S, int R, double theta, int p0) {
+__global__ void rope_table_kernel(float2* __restrict__ table, __nv_bfloat16* __restrict__ table_bf16, int S, int R,
+                                  double theta, int p0) {
     const int half = R >> 1;
     const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
     if (idx >= static_cast<long long>(S + 1) * half) return;
@@ -18,6 +19,10 @@ __global__ void rope_table_kernel(float2* __restrict__ table, int S, int R, doub
     double sn, cs;
     sincos(pos * freq, &sn, &cs);
     table[idx] = make_float2(static_cast<float>(cs), static_cast<float>(sn));
+    if (s < S) {   // bf16 copy, row layout [R/2 cos | R/2 sin]
+        table_bf16[static_cast<size_t>(s) * R + i] = __float2bfloat16_rn(static_cast<float>(cs));
+        table_bf16[static_cast<size_t>(s) * R + half + i] = __float2bfloat16_rn(static_cast<float>(sn));
+    }
 }
 
 // x [B, H, S, D] (element strides xb, xh, xs; D contiguous) -> y [B*H, S, D] contiguous, rows rotated by their position; NH = B * H.  One thread owns the 16-byte chunk pair

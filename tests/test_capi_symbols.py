@@ -39,7 +39,8 @@ def test_host_only_calls(libpath):
     L = af.lib()
     assert L.attnfuse_strerror(0) == b"ok"
     assert L.attnfuse_strerror(2) != L.attnfuse_strerror(3)
-    assert L.attnfuse_rope_table_bytes(4096, 128) == 4097 * 64 * 8
+    # fp32 rows with one trailer row, padded to 256 bytes, then the bf16 copy (2 * rotary_dim bytes per position)
+    assert L.attnfuse_rope_table_bytes(4096, 128) == 4097 * 64 * 8 + 4096 * 128 * 2
     assert L.attnfuse_rope_table_bytes(4096, 0) == 0
 
 
