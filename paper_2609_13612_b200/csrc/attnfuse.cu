@@ -1,6 +1,7 @@
 // Host side of the C-ABI declared in include/attnfuse.h: argument validation, tensor-map
 // encoding, variant selection and launches.  All arithmetic of the path runs in the kernels.
 #include <cuda.h>
+#include <atomic>
 #include <cuda_runtime.h>
 #include <math.h>
 #include <mutex>
@@ -87,17 +88,35 @@ bool keys_rotate_in_bf16(int R) {
     return (R == 16 || R == 32 || R == 64 || R == 128) && env_int("AF_FWD_KEYS_BF16", 0);
 }
 
+// Opt a kernel in to its dynamic shared-memory size once per device (the attribute is per device and per
+// function; `done` is the call site's own bit mask over device ordinals).
+template <typename Kernel>
+af_status allow_dynamic_smem(Kernel kern, int bytes, std::atomic<unsigned long long>& done) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return AF_ERR_CUDA;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (!(done.load(std::memory_order_acquire) & bit)) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+            return AF_ERR_CUDA;
+        done.fetch_or(bit, std::memory_order_release);
+    }
+    return AF_OK;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 af_status check_arch() {
-    static int cached = -1;
-    if (cached < 0) {
-        int dev = 0, major = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return AF_ERR_CUDA;
+    static std::atomic<int> cached[64];   // per device ordinal: 0 = not asked yet, else major + 1
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return AF_ERR_CUDA;
+    int major1 = cached[dev & 63].load(std::memory_order_relaxed);
+    if (major1 == 0) {
+        int major = 0;
         if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return AF_ERR_CUDA;
-        cached = major;
+        major1 = major + 1;
+        cached[dev & 63].store(major1, std::memory_order_relaxed);
     }
-    return cached == 10 ? AF_OK : AF_ERR_ARCH;
+    return major1 == 11 ? AF_OK : AF_ERR_ARCH;
 }
 
 af_status check_common(const af_shape* sh, const af_rope* rope, const void* table, const af_mask* mask, int group) {
@@ -130,12 +149,8 @@ af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const
                              FwdParams p, cudaStream_t stream) {
     using L = FwdSmem<D, NQ, KS, VS, ROPE && TAB>;
     auto kern = attn_fwd_kernel<D, NQ, ROPE, KS, VS, false, TAB>;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
-            return AF_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<unsigned long long> configured{0};
+    if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
     // an even GQA group lets the two query tiles of a CTA be two heads of one kv head (same key range)
     p.pair_heads = (NQ == 2 && (p.group % 2) == 0 && env_int("AF_FWD_PAIR", 1)) ? 1 : 0;
     const int rows_per_cta = p.pair_heads ? BM : BM * NQ;
@@ -153,12 +168,8 @@ af_status launch_fwd2_variant(const CUtensorMap& tq, const CUtensorMap& tk2, con
     constexpr int KS = 3, VS = 3;
     using L = Fwd2Smem<128, KS, VS>;
     auto kern = attn_fwd2_kernel<128, ROPE, KS, VS>;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
-            return AF_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<unsigned long long> configured{0};
+    if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
     p.pair_heads = 0;
     p.n_row_blocks = (p.S + BM - 1) / BM;
     cudaLaunchConfig_t cfg = {};
@@ -183,12 +194,8 @@ af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk
                                     const CUtensorMap& to, const CUtensorMap& tt, FwdParams p, cudaStream_t stream) {
     using L = FwdSmem<D, NQ, 2, 2>;
     auto kern = attn_fwd_kernel<D, NQ, ROPE, 2, 2, true>;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
-            return AF_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<unsigned long long> configured{0};
+    if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
     p.pair_heads = NQ == 2 ? 1 : 0;
     p.n_row_blocks = (p.S + BM - 1) / BM;
     dim3 grid(NQ == 2 ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
@@ -223,12 +230,8 @@ af_status launch_bwd_variant_bs(const CUtensorMap& tx, const CUtensorMap& ty, co
                                 const CUtensorMap& ts, const BwdParams& p, dim3 grid, cudaStream_t stream) {
     using L = BwdSmem<D>;
     auto kern = attn_bwd_kernel<D, DKV, ROT_X, ROT_A, BS>;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES) != cudaSuccess)
-            return AF_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<unsigned long long> configured{0};
+    if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
     kern<<<grid, 512, L::BYTES, stream>>>(tx, ty, ta, tb, ts, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
@@ -564,22 +567,12 @@ af_status attnfuse_decode(const af_shape* shape, const void* q, const void* k, c
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     dim3 grid(n_splits, shape->B * shape->Hkv, 1);
     if (shape->D == 128) {
-        static bool configured = false;
-        if (!configured) {
-            if (cudaFuncSetAttribute(decode_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     DecodeSmem<128>::BYTES) != cudaSuccess)
-                return AF_ERR_CUDA;
-            configured = true;
-        }
+        static std::atomic<unsigned long long> configured{0};
+        if (allow_dynamic_smem(decode_split_kernel<128>, DecodeSmem<128>::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
         decode_split_kernel<128><<<grid, kDecWarps * 32, DecodeSmem<128>::BYTES, stream>>>(tk, tv, p);
     } else {
-        static bool configured = false;
-        if (!configured) {
-            if (cudaFuncSetAttribute(decode_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     DecodeSmem<64>::BYTES) != cudaSuccess)
-                return AF_ERR_CUDA;
-            configured = true;
-        }
+        static std::atomic<unsigned long long> configured{0};
+        if (allow_dynamic_smem(decode_split_kernel<64>, DecodeSmem<64>::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
         decode_split_kernel<64><<<grid, kDecWarps * 32, DecodeSmem<64>::BYTES, stream>>>(tk, tv, p);
     }
     if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
