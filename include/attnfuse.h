@@ -95,6 +95,22 @@ af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, cons
                        int gqa_group, float softmax_scale,
                        void* o, af_dtype o_dtype, float* lse, void* cuda_stream);
 
+/* ---- hybrid arm of Section 5.3: rotate K once, fuse only the Q rotation -------------------------------
+ * Same result as attnfuse_fwd (up to the bf16 rounding of a few rotated elements).  A RoPE pass writes
+ * K' = RoPE(K) into the workspace (contiguous [B,Hkv,S,D] bf16), then the forward kernel runs with the
+ * on-chip rotation of key tiles switched off and the query tiles still rotated on chip.  With grouped
+ * queries K is the small operand (Hkv heads against Hq), so rotating it once costs little HBM traffic
+ * and spares every CTA the rotation of each key tile it streams.  rotary_dim = 0: plain attnfuse_fwd.
+ * workspace (device): attnfuse_fwd_hybrid_workspace_bytes(shape) bytes, 16-byte aligned, caller-owned;
+ * AF_ERR_WORKSPACE when missing or too small. */
+size_t    attnfuse_fwd_hybrid_workspace_bytes(const af_shape* shape);
+af_status attnfuse_fwd_hybrid(const af_shape* shape, const void* q, const void* k, const void* v,
+                              const af_strides* sq, const af_strides* skv,
+                              const af_rope* rope, const void* rope_table, const af_mask* mask,
+                              int gqa_group, float softmax_scale,
+                              void* o, af_dtype o_dtype, float* lse,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* ---- block-sparse attention (Section 4.6) ------------------------------------------------------------
  * The caller evaluates its block predicate once and passes the active 128 x 128 blocks as index lists
  * (device memory, int32): by query row block (CSR: row_ptr [nb + 1], col_idx [row_ptr[nb]], nb = ceil(S/128))

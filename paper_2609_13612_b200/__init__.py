@@ -4,8 +4,8 @@ Argument marshalling only: every step of the path runs in the CUDA kernels.  PyT
 device memory and streams.  There is no CPU fallback: without the compiled library, or without
 a CUDA device, the calls raise.
 """
-from .binding import (AttnFuseError, BlockMask, RopeSpec, MaskSpec, bwd, bwd_static, decode, device_status, fwd, fwd_blocks, fwd_host, lib, rope,
+from .binding import (AttnFuseError, BlockMask, RopeSpec, MaskSpec, bwd, bwd_static, decode, device_status, fwd, fwd_blocks, fwd_host, fwd_hybrid, lib, rope,
                       rope_table, version)
 
-__all__ = ["AttnFuseError", "BlockMask", "RopeSpec", "MaskSpec", "bwd", "bwd_static", "decode", "device_status", "fwd", "fwd_blocks", "fwd_host", "lib",
+__all__ = ["AttnFuseError", "BlockMask", "RopeSpec", "MaskSpec", "bwd", "bwd_static", "decode", "device_status", "fwd", "fwd_blocks", "fwd_host", "fwd_hybrid", "lib",
            "rope", "rope_table", "version"]

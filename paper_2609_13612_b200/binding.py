@@ -83,6 +83,11 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_fwd.restype = i
         L.attnfuse_fwd.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp, P(_Mask), i, f,
                                    vp, i, vp, vp]
+        L.attnfuse_fwd_hybrid_workspace_bytes.restype = sz
+        L.attnfuse_fwd_hybrid_workspace_bytes.argtypes = [P(_Shape)]
+        L.attnfuse_fwd_hybrid.restype = i
+        L.attnfuse_fwd_hybrid.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp, P(_Mask), i, f,
+                                          vp, i, vp, vp, sz, vp]
         L.attnfuse_fwd_host_staging_bytes.restype = sz
         L.attnfuse_fwd_host_staging_bytes.argtypes = [P(_Shape)]
         L.attnfuse_fwd_host.restype = i
@@ -201,6 +206,39 @@ def fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, 
                               ctypes.byref(m), Hq // Hkv, float(softmax_scale), out.data_ptr(),
                               AF_F32 if out.dtype == torch.float32 else AF_BF16,
                               lse.data_ptr() if lse is not None else None, _stream()))
+    return out, lse
+
+
+def fwd_hybrid(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor],
+               mask: MaskSpec, softmax_scale: float, out: Optional[torch.Tensor] = None,
+               lse: Optional[torch.Tensor] = None, out_dtype: torch.dtype = torch.bfloat16, want_lse: bool = True,
+               workspace: Optional[torch.Tensor] = None):
+    """Hybrid forward (Section 5.3): K rotated once by a RoPE pass into `workspace` (uint8, at least
+    attnfuse_fwd_hybrid_workspace_bytes; allocated when None), Q rotated inside the kernel.  Returns (o, lse)."""
+    _need_cuda(q, k, v, table, out, lse, workspace)
+    assert q.dtype == k.dtype == v.dtype == torch.bfloat16
+    B, Hq, S, D = q.shape
+    Hkv = k.shape[1]
+    assert k.shape == v.shape == (B, Hkv, S, D) and k.stride() == v.stride()
+    if out is None:
+        out = torch.empty((B, Hq, S, D), dtype=out_dtype, device=q.device)
+    if lse is None and want_lse:
+        lse = torch.empty((B, Hq, S), dtype=torch.float32, device=q.device)
+    assert out.is_contiguous() and out.dtype in (torch.bfloat16, torch.float32)
+    sh = _Shape(B, Hq, Hkv, S, D)
+    if workspace is None:
+        workspace = torch.empty(lib().attnfuse_fwd_hybrid_workspace_bytes(ctypes.byref(sh)), dtype=torch.uint8,
+                                device=q.device)
+    sq, skv = _strides(q), _strides(k)
+    r = _Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset)
+    m = _mask_struct(mask)
+    _check(lib().attnfuse_fwd_hybrid(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), ctypes.byref(sq),
+                                     ctypes.byref(skv), ctypes.byref(r),
+                                     table.data_ptr() if table is not None else None, ctypes.byref(m), Hq // Hkv,
+                                     float(softmax_scale), out.data_ptr(),
+                                     AF_F32 if out.dtype == torch.float32 else AF_BF16,
+                                     lse.data_ptr() if lse is not None else None, workspace.data_ptr(),
+                                     workspace.numel() * workspace.element_size(), _stream()))
     return out, lse
 
 

@@ -220,7 +220,7 @@ af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
         return p.R > 0 ? launch_fwd_variant<D, 1, true, 2, 2>(tq, tk, tv, to, tt, p, stream)
                        : launch_fwd_variant<D, 1, false, 2, 2>(tq, tk, tv, to, tt, p, stream);
     }
-    if (p.R > 0 && keys_rotate_in_bf16(p.R)) return launch_fwd_variant<D, 2, true, 2, 2, true>(tq, tk, tv, to, tt, p, stream);
+    if (p.R > 0 && p.keys_bf16) return launch_fwd_variant<D, 2, true, 2, 2, true>(tq, tk, tv, to, tt, p, stream);
     return p.R > 0 ? launch_fwd_variant<D, 2, true, 2, 2>(tq, tk, tv, to, tt, p, stream)
                    : launch_fwd_variant<D, 2, false, 2, 2>(tq, tk, tv, to, tt, p, stream);
 }
@@ -403,7 +403,7 @@ namespace {
 af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
                    const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
                    int gqa_group, float softmax_scale, const int* bs_row_ptr, const int* bs_col_idx,
-                   const int* bs_order, void* o, af_dtype o_dtype, float* lse, void* cuda_stream) {
+                   const int* bs_order, void* o, af_dtype o_dtype, float* lse, bool k_prerotated, void* cuda_stream) {
     af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
     if (st != AF_OK) return st;
     if (!q || !k || !v || !o) return AF_ERR_NULL;
@@ -417,7 +417,9 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
 
     CUtensorMap tq, tk, tv, to;
     if ((st = make_tmap(&tq, q, shape->B, shape->Hq, shape->S, shape->D, stq, BM)) != AF_OK) return st;
-    if ((st = make_tmap(&tk, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, BN)) != AF_OK) return st;
+    af_strides stk = stkv;
+    if (k_prerotated) resolve_strides(nullptr, shape->Hkv, shape->S, shape->D, &stk);   // K' is contiguous
+    if ((st = make_tmap(&tk, k, shape->B, shape->Hkv, shape->S, shape->D, stk, BN)) != AF_OK) return st;
     if ((st = make_tmap(&tv, v, shape->B, shape->Hkv, shape->S, shape->D, stkv, BN)) != AF_OK) return st;
     // bf16 output goes out through TMA (contiguous [B,Hq,S,D]); with fp32 output the map is not used
     to = tq;
@@ -430,7 +432,8 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     // (optional mode) key tiles receive the 128 rows of the table's bf16 copy that belong to them by TMA
     const int Rr = rope->rotary_dim;
     CUtensorMap tt = tq;
-    if (keys_rotate_in_bf16(Rr) && (st = make_tmap_table(&tt, rope_table, shape->S, Rr)) != AF_OK) return st;
+    const bool keys_bf16 = !k_prerotated && keys_rotate_in_bf16(Rr);
+    if (keys_bf16 && (st = make_tmap_table(&tt, rope_table, shape->S, Rr)) != AF_OK) return st;
 
     FwdParams p;
     p.B = shape->B; p.Hq = shape->Hq; p.Hkv = shape->Hkv; p.S = shape->S; p.group = gqa_group;
@@ -446,6 +449,8 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     p.bs_row_ptr = bs_row_ptr;
     p.bs_col_idx = bs_col_idx;
     p.bs_order = bs_order;
+    p.rot_k = k_prerotated ? 0 : 1;
+    p.keys_bf16 = keys_bf16 ? 1 : 0;
 #ifdef AF_TRACE
     p.trace = reinterpret_cast<long long*>(getenv("AF_TRACE_PTR") ? strtoull(getenv("AF_TRACE_PTR"), nullptr, 0) : 0ull);
     cudaMemcpyToSymbol(af::g_trace, &p.trace, sizeof(p.trace));
@@ -455,7 +460,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
         return shape->D == 128 ? launch_fwd_blocks<128>(tq, tk, tv, to, tt, p, stream) : launch_fwd_blocks<64>(tq, tk, tv, to, tt, p, stream);
     const int R = rope->rotary_dim;
     const bool pair_ok = shape->D == 128 && (gqa_group % 4) == 0 && (R == 0 || R == 16 || R == 32 || R == 64 || R == 128);
-    if (pair_ok && env_int("AF_FWD_2CTA", 0)) {
+    if (pair_ok && !k_prerotated && env_int("AF_FWD_2CTA", 0)) {
         CUtensorMap tk2;
         if ((st = make_tmap(&tk2, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, 64)) != AF_OK) return st;
         return R > 0 ? launch_fwd2_variant<true>(tq, tk2, tv, p, stream) : launch_fwd2_variant<false>(tq, tk2, tv, p, stream);
@@ -470,7 +475,35 @@ af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, cons
                        const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
                        int gqa_group, float softmax_scale, void* o, af_dtype o_dtype, float* lse, void* cuda_stream) {
     return fwd_impl(shape, q, k, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, nullptr, nullptr, nullptr,
-                    o, o_dtype, lse, cuda_stream);
+                    o, o_dtype, lse, false, cuda_stream);
+}
+
+size_t attnfuse_fwd_hybrid_workspace_bytes(const af_shape* shape) {
+    if (!shape || shape->B < 1 || shape->Hkv < 1 || shape->S < 1 || shape->D < 1) return 0;
+    return static_cast<size_t>(shape->B) * shape->Hkv * shape->S * shape->D * 2;
+}
+
+af_status attnfuse_fwd_hybrid(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
+                              const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
+                              int gqa_group, float softmax_scale, void* o, af_dtype o_dtype, float* lse,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
+    if (st != AF_OK) return st;
+    if (rope->rotary_dim == 0)   // nothing to rotate: the plain kernel
+        return fwd_impl(shape, q, k, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, nullptr, nullptr,
+                        nullptr, o, o_dtype, lse, false, cuda_stream);
+    if (!k || !workspace) return AF_ERR_NULL;
+    if (workspace_bytes < attnfuse_fwd_hybrid_workspace_bytes(shape)) return AF_ERR_WORKSPACE;
+    if (!aligned16(k) || !aligned16(workspace)) return AF_ERR_ALIGN;
+    af_strides stkv;
+    if ((st = resolve_strides(skv, shape->Hkv, shape->S, shape->D, &stkv)) != AF_OK) return st;
+    if ((st = check_arch()) != AF_OK) return st;
+    // K' = RoPE(K) once, contiguous, into the workspace; the kernel then rotates only its Q tiles
+    if ((st = launch_rope(k, stkv, workspace, shape->B, shape->Hkv, shape->S, shape->D, rope->rotary_dim, rope_table, 0,
+                          static_cast<cudaStream_t>(cuda_stream))) != AF_OK)
+        return st;
+    return fwd_impl(shape, q, workspace, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, nullptr, nullptr,
+                    nullptr, o, o_dtype, lse, true, cuda_stream);
 }
 
 af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
@@ -480,7 +513,7 @@ af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* 
     if (!blocks || !blocks->row_ptr || !blocks->col_idx) return AF_ERR_NULL;
     if (blocks->block != 128) return AF_ERR_SPEC;
     return fwd_impl(shape, q, k, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, blocks->row_ptr,
-                    blocks->col_idx, blocks->row_order, o, o_dtype, lse, cuda_stream);
+                    blocks->col_idx, blocks->row_order, o, o_dtype, lse, false, cuda_stream);
 }
 
 size_t attnfuse_fwd_host_staging_bytes(const af_shape* shape) {

@@ -29,6 +29,9 @@ struct FwdParams {
     const int* bs_row_ptr;
     const int* bs_col_idx;
     const int* bs_order;   // optional launch order of the row blocks (longest lists first), or nullptr
+    int keys_bf16;         // host-side choice of the TAB instantiation (packed-bf16 key rotation)
+    int rot_k;             // ROPE kernels: 1 = rotate the key tiles on chip; 0 = the keys arrive rotated (hybrid
+                           // arm of Section 5.3: K rotated once by a RoPE pass, only Q rotated in the kernel)
 #ifdef AF_TRACE
     long long* trace;
 #endif
@@ -328,7 +331,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr int B_KREADY = ROPE ? L::B_KROT : L::B_KFULL;
+            const int B_KREADY = (ROPE && p.rot_k) ? L::B_KROT : L::B_KFULL;
             constexpr int B_QREADY = ROPE ? L::B_QROT : L::B_QFULL;
             int cnt[NQ];
             bool ok = true;
@@ -432,7 +435,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------ rotation warpgroup (Section 4.1)
         setmaxnreg_dec<kRotRegs>();
-        if (ROPE) {
+        if (ROPE && p.rot_k) {
             const int t = threadIdx.x - 128;
             // packed bf16 arithmetic on TMA-fed table tiles (rotary widths with a fast path)
             auto run_tab = [&](auto cp_tag) {

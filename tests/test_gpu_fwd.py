@@ -74,6 +74,46 @@ def test_forward_small_one_query_tile_per_cta(w, monkeypatch):
     run_case(w)
 
 
+@pytest.mark.parametrize("w", [SMALL[i] for i in (1, 3, 4, 6, 7, 9, 12, 14, 15, 17)] + [synth.CONFIGS[1]],
+                         ids=lambda w: w.name)
+def test_forward_hybrid_prerotated_keys(w):
+    """Hybrid arm of the fuse-or-not experiment: K rotated once by the RoPE pass into a workspace, Q rotated in
+    the kernel.  Held to the oracle like the fused call, and to the fused call itself up to bf16 roundings."""
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S) if w.R > 0 else None
+    o, lse = af.fwd_hybrid(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale)
+    o_f, lse_f = af.fwd(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    want_o, want_l = oracle.run_workload(w, t)
+    pu.assert_close(w.name + " O hybrid", pu.to_np(o), want_o)
+    assert np.abs(pu.to_np(lse) - want_l).max() <= pu.LSE_TOL
+    assert (o.float() - o_f.float()).abs().max().item() <= 8e-3
+    assert (lse - lse_f).abs().max().item() <= 2e-3
+
+
+def test_forward_hybrid_strided_inputs_and_small_workspace():
+    w = W("hybrid_strided", 2, 4, 2, 300, 128, theta=1e4, seed_id=131)
+    t = synth.draw_all(w)
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S)
+    # K and V as slices of one packed [B, S, 2, Hkv, D] buffer
+    kv = torch.empty((w.B, w.S, 2, w.Hkv, w.D), dtype=torch.bfloat16, device="cuda")
+    kv[:, :, 0] = pu.to_dev(t["k"]).permute(0, 2, 1, 3)
+    kv[:, :, 1] = pu.to_dev(t["v"]).permute(0, 2, 1, 3)
+    k = kv[:, :, 0].permute(0, 2, 1, 3)
+    v = kv[:, :, 1].permute(0, 2, 1, 3)
+    o, _ = af.fwd_hybrid(pu.to_dev(t["q"]), k, v, rope, table, mask, w.scale)
+    torch.cuda.synchronize()
+    want_o, _ = oracle.run_workload(w, t)
+    pu.assert_close("hybrid strided O", pu.to_np(o), want_o)
+    with pytest.raises(af.AttnFuseError):
+        af.fwd_hybrid(pu.to_dev(t["q"]), k, v, rope, table, mask, w.scale,
+                      workspace=torch.empty(1024, dtype=torch.uint8, device="cuda"))
+
+
 def test_forward_fp32_output():
     run_case(W("fp32_out", 1, 4, 2, 300, 128, theta=1e4, seed_id=120), out_dtype=torch.float32)
 
