@@ -333,13 +333,18 @@ def main():
         ex = {}
         k_ex, w_ex = 20, 5
 
-        def fwd_ms(wl, fused=True, sets_=None):
+        def fwd_ms(wl, fused=True, sets_=None, hybrid=False):
             r, m, tb = specs(wl)
             ss = sets_ or make_sets(wl, n_sets_for(wl))
             oo = torch.empty((wl.B, wl.Hq, wl.S, wl.D), dtype=torch.bfloat16, device=dev)
             ll = torch.empty((wl.B, wl.Hq, wl.S), dtype=torch.float32, device=dev)
             norope = af.RopeSpec()
-            if fused:
+            if hybrid:
+                # third arm: K rotated once by the RoPE pass (into a workspace), Q rotated inside the kernel
+                wsk = torch.empty(ss[0]["k"].numel() * 2, dtype=torch.uint8, device=dev)
+                f = lambda i: af.fwd_hybrid(ss[i % len(ss)]["q"], ss[i % len(ss)]["k"], ss[i % len(ss)]["v"], r, tb, m,
+                                            wl.scale, out=oo, lse=ll, workspace=wsk)
+            elif fused:
                 f = lambda i: af.fwd(ss[i % len(ss)]["q"], ss[i % len(ss)]["k"], ss[i % len(ss)]["v"], r, tb, m,
                                      wl.scale, out=oo, lse=ll)
             else:
@@ -369,12 +374,15 @@ def main():
                                                 "mode_frac_of_measured_burst_peak": wl.fwd_flops() / ms_b / 1e9 / peaks["bf16_tflops"]}
         del ss
         torch.cuda.empty_cache()
-        for wl in synth.CONFIGS[2:4]:
+        for wl in synth.CONFIGS[1:4]:
             ms_f, ss = fwd_ms(wl, True)
             ms_s, _ = fwd_ms(wl, False, ss)
+            ms_h, _ = fwd_ms(wl, True, ss, hybrid=True)
             ex[wl.name] = {"fused_fwd_ms": ms_f, "fused_fwd_tflops": wl.fwd_flops() / ms_f / 1e9,
                            "separate_rope_fwd_ms": ms_s, "separate_rope_fwd_tflops": wl.fwd_flops() / ms_s / 1e9,
-                           "fused_over_separate_speedup": ms_s / ms_f}
+                           "fused_over_separate_speedup": ms_s / ms_f,
+                           "hybrid_fwd_ms": ms_h, "hybrid_fwd_tflops": wl.fwd_flops() / ms_h / 1e9,
+                           "hybrid_frac_of_measured_burst_peak": wl.fwd_flops() / ms_h / 1e9 / peaks["bf16_tflops"]}
             del ss
             torch.cuda.empty_cache()
         # config 5: forward + backward
@@ -506,8 +514,10 @@ def main():
             wl = synth.Workload("sweep_S%d" % S, 32768 // S, 32, 8, S, 128, theta=5.0e5, seed_id=50)
             ms_f, ss = fwd_ms(wl, True)
             ms_s, _ = fwd_ms(wl, False, ss)
-            sweep.append({"S": S, "B": wl.B, "fused_ms": ms_f, "separate_ms": ms_s, "speedup_fused": ms_s / ms_f,
-                          "fused_tflops": wl.fwd_flops() / ms_f / 1e9})
+            ms_h, _ = fwd_ms(wl, True, ss, hybrid=True)
+            sweep.append({"S": S, "B": wl.B, "fused_ms": ms_f, "separate_ms": ms_s, "hybrid_ms": ms_h,
+                          "speedup_fused": ms_s / ms_f, "speedup_hybrid_over_fused": ms_f / ms_h,
+                          "fused_tflops": wl.fwd_flops() / ms_f / 1e9, "hybrid_tflops": wl.fwd_flops() / ms_h / 1e9})
             del ss
             torch.cuda.empty_cache()
         ex["rotation_calculus_sweep"] = sweep
