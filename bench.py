@@ -159,7 +159,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--extras", type=int, default=1, help="also time configs 3-5, the separate-RoPE arm and the sweep")
     ap.add_argument("--cpu-baseline", type=int, default=1)
-    ap.add_argument("--profile", default="", choices=["", "fwd", "bwd", "rope", "decode"],
+    ap.add_argument("--profile", default="", choices=["", "fwd", "hybrid", "bwd", "rope", "decode"],
                     help="run only a few launches of one path (for ncu captures) and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -252,12 +252,15 @@ def main():
         return
     if args.profile:
         # a handful of launches of one path on its configuration, nothing else: the target of ncu captures
-        wl = {"fwd": synth.CONFIGS[1], "bwd": synth.CONFIGS[4], "rope": synth.CONFIGS[3]}[args.profile]
+        wl = {"fwd": synth.CONFIGS[1], "hybrid": synth.CONFIGS[1], "bwd": synth.CONFIGS[4],
+              "rope": synth.CONFIGS[3]}[args.profile]
         r, m, tb = specs(wl)
         t = {k: to_dev(v) for k, v in synth.draw_all(wl).items()}
         for _ in range(3):
             if args.profile == "rope":
                 af.rope(t["q"], r, tb)
+            elif args.profile == "hybrid":
+                af.fwd_hybrid(t["q"], t["k"], t["v"], r, tb, m, wl.scale)
             else:
                 o_, l_ = af.fwd(t["q"], t["k"], t["v"], r, tb, m, wl.scale)
                 if args.profile == "bwd":
