@@ -156,6 +156,21 @@ af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const
     const int rows_per_cta = p.pair_heads ? BM : BM * NQ;
     p.n_row_blocks = (p.S + rows_per_cta - 1) / rows_per_cta;
     dim3 grid(p.pair_heads ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
+    if (ROPE && !p.rot_k) {
+        // hybrid arm: launched as a programmatic dependent of the RoPE pass on K that precedes it in the stream;
+        // the kernel waits for that pass only before its first key-tile load
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(128 * (2 + NQ), 1, 1);
+        cfg.dynamicSmemBytes = L::BYTES;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, to, tt, p) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+    }
     kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, to, tt, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }

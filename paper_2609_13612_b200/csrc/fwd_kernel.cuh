@@ -307,6 +307,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int bx = 0; bx < NBOX; ++bx)
                     tma_load_4d(sQ + q * TILE + bx * BOX_BYTES, &tm_q, &bars[L::B_QFULL + q], bx * BOX_COLS, i0[q], hq[q], b);
             }
+            // hybrid arm: the keys are written by the RoPE pass launched just before this grid, which may still be
+            // running (programmatic dependent launch); everything above overlaps with its tail
+            if (ROPE && !p.rot_k) grid_dep_wait();
             for (int it = 0; it < n_it; ++it) {
                 const int j0 = tile_at(jlo_c + it) * BN;
                 const int ks = it % KS, vs = it % VS;
