@@ -2,6 +2,7 @@
 // encoding, variant selection and launches.  All arithmetic of the path runs in the kernels.
 #include <cuda.h>
 #include <atomic>
+#include <utility>
 #include <cuda_runtime.h>
 #include <math.h>
 #include <mutex>
@@ -103,6 +104,25 @@ af_status allow_dynamic_smem(Kernel kern, int bytes, std::atomic<unsigned long l
     return AF_OK;
 }
 
+// Launch as a programmatic dependent of the kernel that precedes it in the stream: the grid may be scheduled
+// while that kernel drains and runs its set-up, then waits (griddepcontrol.wait in the kernel) for the
+// predecessor's completion before it touches global memory.  dependent = false: a plain launch.
+template <typename... KArgs, typename... Args>
+af_status launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool dependent,
+                        Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 af_status check_arch() {
@@ -159,17 +179,7 @@ af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const
     if (ROPE && !p.rot_k) {
         // hybrid arm: launched as a programmatic dependent of the RoPE pass on K that precedes it in the stream;
         // the kernel waits for that pass only before its first key-tile load
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = grid;
-        cfg.blockDim = dim3(128 * (2 + NQ), 1, 1);
-        cfg.dynamicSmemBytes = L::BYTES;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, kern, tq, tk, tv, to, tt, p) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+        return launch_kernel(kern, grid, dim3(128 * (2 + NQ), 1, 1), L::BYTES, stream, true, tq, tk, tv, to, tt, p);
     }
     kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, to, tt, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
@@ -247,8 +257,8 @@ af_status launch_bwd_variant_bs(const CUtensorMap& tx, const CUtensorMap& ty, co
     auto kern = attn_bwd_kernel<D, DKV, ROT_X, ROT_A, BS>;
     static std::atomic<unsigned long long> configured{0};
     if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
-    kern<<<grid, 512, L::BYTES, stream>>>(tx, ty, ta, tb, ts, p);
-    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+    // every gradient kernel follows the delta kernel or another kernel of the backward sequence in the stream
+    return launch_kernel(kern, grid, dim3(512, 1, 1), L::BYTES, stream, true, tx, ty, ta, tb, ts, p);
 }
 // dense or, when the parameters carry block lists, block-sparse instantiation
 template <int D, bool DKV, bool ROT_X, bool ROT_A>
@@ -259,18 +269,19 @@ af_status launch_bwd_variant(const CUtensorMap& tx, const CUtensorMap& ty, const
 }
 
 // RoPE pass x [B, H, S, D] (strided) -> x_out (contiguous); R > 0.
+// dependent: launch as a programmatic dependent of the preceding kernel (only inside this library's own sequences).
 af_status launch_rope(const void* x_in, const af_strides& st, void* x_out, int B, int H, int S, int D, int R,
-                      const void* rope_table, int inverse, cudaStream_t stream) {
+                      const void* rope_table, int inverse, cudaStream_t stream, bool dependent = false) {
     constexpr int HPT = 4;
     const long long NH = static_cast<long long>(B) * H;
     const int per_row = (R >> 4) + ((D - R) >> 3);
     const long long items = static_cast<long long>(S) * per_row;
     dim3 grid(static_cast<unsigned>((items + 255) / 256), static_cast<unsigned>((NH + HPT - 1) / HPT), 1);
     if (grid.y > 65535) return AF_ERR_SHAPE;
-    rope_apply_kernel<HPT><<<grid, 256, 0, stream>>>(static_cast<const uint4*>(x_in), static_cast<uint4*>(x_out),
-                                                     static_cast<const float2*>(rope_table), static_cast<int>(NH), H, S,
-                                                     D, R, inverse ? -1.f : 1.f, st.b, st.h, st.s);
-    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+    return launch_kernel(rope_apply_kernel<HPT>, grid, dim3(256, 1, 1), 0, stream, dependent,
+                         static_cast<const uint4*>(x_in), static_cast<uint4*>(x_out),
+                         static_cast<const float2*>(rope_table), static_cast<int>(NH), H, S, D, R, inverse ? -1.f : 1.f,
+                         static_cast<long long>(st.b), static_cast<long long>(st.h), static_cast<long long>(st.s));
 }
 
 // delta, then the two gradient kernels.  tkp / tqp: tensor maps over the rotated-K and rotated-Q caches in
@@ -300,7 +311,7 @@ af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMa
     dim3 gkv(sh->B * sh->Hkv, tiles, 1), gq(sh->B * sh->Hq, tiles, 1);
     if (p.R > 0 && tkp && tqp && only == 0) {
         // both caches: K' by the RoPE pass, Q' by the dQ kernel, no on-chip rotation in the dK/dV loop
-        if ((st = launch_rope(k, stkv, kcache, sh->B, sh->Hkv, sh->S, D, p.R, p.table, 0, stream)) != AF_OK) return st;
+        if ((st = launch_rope(k, stkv, kcache, sh->B, sh->Hkv, sh->S, D, p.R, p.table, 0, stream, true)) != AF_OK) return st;
         p.out1 = dq; p.out2 = nullptr; p.out_f32 = dq_f32; p.store_x = 1;
         role_lists(false);
         if ((st = launch_bwd_variant<D, false, true, false>(tq, tdo, *tkp, tv, *tqp, p, gq, stream)) != AF_OK) return st;

@@ -50,6 +50,7 @@ template <int D>
 __global__ void __launch_bounds__(256) bwd_delta_kernel(const uint4* __restrict__ o, const uint4* __restrict__ d_o,
                                                         float* __restrict__ delta, long long rows) {
     constexpr int TPR = D / 8;
+    grid_dep_launch();   // the next kernel of the backward sequence may be scheduled while this one runs
     const long long idx = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
     const long long row = idx / TPR;
     float acc = 0.f;
@@ -319,6 +320,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Programmatic dependent launch: this grid may have been scheduled while its predecessor in the backward
+    // sequence (delta, RoPE pass or the other gradient kernel) was still running; from here on it reads what
+    // they wrote.  The next kernel of the sequence may in turn be scheduled from now on.
+    grid_dep_wait();
+    grid_dep_launch();
     AF_BSTAMP(5, 0, 0);
 
     if (warp == 0) {

@@ -33,7 +33,11 @@ template <int HPT>
 __global__ void __launch_bounds__(256)
 rope_apply_kernel(const uint4* x, uint4* y, const float2* __restrict__ table, int NH, int H, int S,
                   int D, int R, float sgn, long long xb, long long xh, long long xs) {
-    grid_dep_launch();   // a dependent grid (the hybrid forward) may start its set-up while this pass runs
+    // programmatic dependent launch, both ways: as a dependent (inside the backward sequence) wait for the
+    // predecessor before touching memory; as a predecessor (of the hybrid forward or of a gradient kernel) let
+    // the next grid be scheduled and run its set-up while this pass runs
+    grid_dep_wait();
+    grid_dep_launch();
     const int CP = R >> 4;                 // rotated chunk pairs per row
     const int PT = (D - R) >> 3;           // pass-through chunks per row
     const int per_row = CP + PT;
