@@ -139,9 +139,14 @@ af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* 
                               void* o, af_dtype o_dtype, float* lse, void* cuda_stream);
 
 /* Same computation with HOST buffers: q, k, v, o (bf16) and lse (nullable) are host pointers
- * (pinned memory recommended).  `staging` is a DEVICE buffer of at least attnfuse_fwd_host_staging_bytes()
- * bytes; the call enqueues host-to-device copies, the kernel and device-to-host copies on the stream.
- * alibi slopes inside `mask` remain a DEVICE pointer. */
+ * (pinned memory: with pageable memory the copies are not asynchronous).  `staging` is a DEVICE buffer
+ * of at least attnfuse_fwd_host_staging_bytes() bytes, caller-owned.  The work is cut into chunks of
+ * consecutive (batch element, kv head) units and pipelined: host-to-device copies on the caller's stream,
+ * the kernels and the device-to-host copies on two internal streams of the library (created once per
+ * device), so that the two copy directions and the kernels overlap; the caller's stream waits for the
+ * last result at the end of the call, so work enqueued on it afterwards sees o_host and lse_host complete
+ * and may reuse `staging`.  Results are bit-identical to attnfuse_fwd on the same data.  Calls are
+ * serialised on the host by a lock.  alibi slopes inside `mask` remain a DEVICE pointer. */
 size_t    attnfuse_fwd_host_staging_bytes(const af_shape* shape);
 af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const void* k_host, const void* v_host,
                             const af_rope* rope, const void* rope_table, const af_mask* mask,

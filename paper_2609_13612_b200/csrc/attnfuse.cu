@@ -123,6 +123,31 @@ af_status launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t sm
     return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
+// Internal streams and events of attnfuse_fwd_host, per device, created on first use and kept.
+struct HostPipe {
+    static constexpr int kEvents = 64;
+    cudaStream_t compute = nullptr, d2h = nullptr;
+    cudaEvent_t ev[kEvents] = {};
+    int next = 0;
+    bool ready = false;
+};
+std::mutex g_pipe_mutex;
+HostPipe g_pipes[64];
+// (caller holds g_pipe_mutex)
+HostPipe* get_pipe() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    HostPipe* p = &g_pipes[dev & 63];
+    if (!p->ready) {
+        if (cudaStreamCreateWithFlags(&p->compute, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaStreamCreateWithFlags(&p->d2h, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        for (int i = 0; i < HostPipe::kEvents; ++i)
+            if (cudaEventCreateWithFlags(&p->ev[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        p->ready = true;
+    }
+    return p;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 af_status check_arch() {
@@ -559,20 +584,90 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
     if (st != AF_OK) return st;
     if (staging_bytes < attnfuse_fwd_host_staging_bytes(shape)) return AF_ERR_WORKSPACE;
     if (!aligned16(staging)) return AF_ERR_ALIGN;
-    const size_t qn = static_cast<size_t>(shape->B) * shape->Hq * shape->S * shape->D * 2;
-    const size_t kn = static_cast<size_t>(shape->B) * shape->Hkv * shape->S * shape->D * 2;
-    const size_t ln = static_cast<size_t>(shape->B) * shape->Hq * shape->S * 4;
+    const size_t row = static_cast<size_t>(shape->S) * shape->D * 2;   // bytes of one head of Q, K, V or O
+    const size_t qn = static_cast<size_t>(shape->B) * shape->Hq * row;
+    const size_t kn = static_cast<size_t>(shape->B) * shape->Hkv * row;
     uint8_t* base = static_cast<uint8_t*>(staging);
     uint8_t *dq = base, *dk = dq + qn, *dv = dk + kn, *dob = dv + kn, *dl = dob + qn;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (cudaMemcpyAsync(dq, q_host, qn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return AF_ERR_CUDA;
-    if (cudaMemcpyAsync(dk, k_host, kn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return AF_ERR_CUDA;
-    if (cudaMemcpyAsync(dv, v_host, kn, cudaMemcpyHostToDevice, stream) != cudaSuccess) return AF_ERR_CUDA;
-    st = attnfuse_fwd(shape, dq, dk, dv, nullptr, nullptr, rope, rope_table, mask, gqa_group, softmax_scale, dob,
-                      AF_BF16, lse_host ? reinterpret_cast<float*>(dl) : nullptr, cuda_stream);
-    if (st != AF_OK) return st;
-    if (cudaMemcpyAsync(o_host, dob, qn, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return AF_ERR_CUDA;
-    if (lse_host && cudaMemcpyAsync(lse_host, dl, ln, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+
+    // Work units (batch element, kv head with its query heads) are independent and contiguous in every tensor, so
+    // the call is cut into chunks of consecutive units and pipelined: the host-to-device copies of chunk c + 1 (on
+    // the caller's stream), the kernel of chunk c (internal stream) and the device-to-host copies of chunk c - 1
+    // (second internal stream) run at the same time; the two copy directions use different DMA engines.
+    // Chunking: whole batch elements when there are at least 8 of them, else groups of kv heads per batch element.
+    int nb = 1, nh = shape->Hkv;   // a chunk = nb batch elements x nh kv heads
+    if (shape->B >= 8) {
+        nb = (shape->B + 7) / 8;
+    } else {
+        int per_batch = (8 + shape->B - 1) / shape->B;
+        if (per_batch > shape->Hkv) per_batch = shape->Hkv;
+        while (shape->Hkv % per_batch) --per_batch;
+        nh = shape->Hkv / per_batch;
+    }
+    const int chunks_b = (shape->B + nb - 1) / nb, chunks_h = shape->Hkv / nh;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe* pipe = get_pipe();
+    if (!pipe) return AF_ERR_CUDA;
+    auto next_event = [&]() {
+        cudaEvent_t e = pipe->ev[pipe->next];
+        pipe->next = (pipe->next + 1) % HostPipe::kEvents;
+        return e;
+    };
+    // the internal streams start after whatever the caller's stream holds so far (e.g. the table build)
+    cudaEvent_t e0 = next_event();
+    if (cudaEventRecord(e0, stream) != cudaSuccess || cudaStreamWaitEvent(pipe->compute, e0, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(pipe->d2h, e0, 0) != cudaSuccess)
+        return AF_ERR_CUDA;
+    // K and V go first, each as one copy, then one copy of Q per chunk: several small host-to-device copies per
+    // chunk interleaved with the device-to-host copies of earlier chunks overlapped poorly (1.42 ms against 1.07 ms
+    // for the same bytes at config 2)
+    if (cudaMemcpyAsync(dk, k_host, kn, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(dv, v_host, kn, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return AF_ERR_CUDA;
+    for (int cb = 0; cb < chunks_b; ++cb) {
+        const int b0 = cb * nb, bn = (b0 + nb <= shape->B) ? nb : shape->B - b0;
+        for (int ch = 0; ch < chunks_h; ++ch) {
+            const int hk0 = ch * nh, hq0 = hk0 * gqa_group;
+            // with nh < Hkv a chunk lies inside one batch element (bn = 1), so it is contiguous in every tensor
+            const size_t q_off = (static_cast<size_t>(b0) * shape->Hq + hq0) * row;
+            const size_t k_off = (static_cast<size_t>(b0) * shape->Hkv + hk0) * row;
+            const size_t q_bytes = static_cast<size_t>(bn) * nh * gqa_group * row;
+            const size_t l_off = (static_cast<size_t>(b0) * shape->Hq + hq0) * shape->S * 4;
+            const uint8_t* qh = static_cast<const uint8_t*>(q_host);
+            if (cudaMemcpyAsync(dq + q_off, qh + q_off, q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+                return AF_ERR_CUDA;
+            cudaEvent_t e_in = next_event(), e_k = next_event();
+            if (cudaEventRecord(e_in, stream) != cudaSuccess || cudaStreamWaitEvent(pipe->compute, e_in, 0) != cudaSuccess)
+                return AF_ERR_CUDA;
+            af_shape cs = {bn, nh * gqa_group, nh, shape->S, shape->D};
+            af_mask cm = *mask;
+            if (cm.alibi_slopes) cm.alibi_slopes += hq0;
+            // strides of the full tensors: a chunk of kv heads inside a batch element keeps the batch stride
+            af_strides sq, skv;
+            sq.s = skv.s = shape->D;
+            sq.h = skv.h = static_cast<int64_t>(shape->S) * shape->D;
+            sq.b = static_cast<int64_t>(shape->Hq) * shape->S * shape->D;
+            skv.b = static_cast<int64_t>(shape->Hkv) * shape->S * shape->D;
+            // the output of a chunk is contiguous [bn, heads, S, D] only if the chunk covers whole batch elements or
+            // a single one; both hold here (bn = 1 when nh < Hkv)
+            st = attnfuse_fwd(&cs, dq + q_off, dk + k_off, dv + k_off, &sq, &skv, rope, rope_table, &cm, gqa_group,
+                              softmax_scale, dob + q_off, AF_BF16, lse_host ? reinterpret_cast<float*>(dl + l_off) : nullptr,
+                              pipe->compute);
+            if (st != AF_OK) return st;
+            if (cudaEventRecord(e_k, pipe->compute) != cudaSuccess || cudaStreamWaitEvent(pipe->d2h, e_k, 0) != cudaSuccess)
+                return AF_ERR_CUDA;
+            if (cudaMemcpyAsync(static_cast<uint8_t*>(o_host) + q_off, dob + q_off, q_bytes, cudaMemcpyDeviceToHost,
+                                pipe->d2h) != cudaSuccess)
+                return AF_ERR_CUDA;
+        }
+    }
+    // L in one copy at the end (small copies between the large ones cost overlap, as above)
+    const size_t ln = static_cast<size_t>(shape->B) * shape->Hq * shape->S * 4;
+    if (lse_host && cudaMemcpyAsync(lse_host, dl, ln, cudaMemcpyDeviceToHost, pipe->d2h) != cudaSuccess) return AF_ERR_CUDA;
+    // the caller's stream continues once the last results are on the host
+    cudaEvent_t e_done = next_event();
+    if (cudaEventRecord(e_done, pipe->d2h) != cudaSuccess || cudaStreamWaitEvent(stream, e_done, 0) != cudaSuccess)
         return AF_ERR_CUDA;
     return AF_OK;
 }

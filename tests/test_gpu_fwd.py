@@ -114,6 +114,35 @@ def test_forward_hybrid_strided_inputs_and_small_workspace():
                       workspace=torch.empty(1024, dtype=torch.uint8, device="cuda"))
 
 
+@pytest.mark.parametrize("w", [
+    W("host_gqa_chunks", 1, 8, 4, 300, 128, theta=5e5, seed_id=141),                     # 4 chunks of one kv head
+    W("host_batches", 9, 4, 2, 200, 64, theta=1e4, seed_id=142),                          # chunks of two batch elements
+    W("host_alibi", 2, 8, 4, 260, 128, theta=1e4, window=100, alibi=True, seed_id=143),   # slopes offset per chunk
+    W("host_single_chunk", 1, 2, 1, 150, 128, theta=1e4, seed_id=144),
+], ids=lambda w: w.name)
+def test_forward_from_host_buffers(w):
+    """attnfuse_fwd_host: pinned host tensors in and out, the copies and the kernels of consecutive chunks of
+    (batch, kv head) units pipelined on internal streams.  Same bounds as the device call, and bit-identical to it."""
+    t = synth.draw_all(w)
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S)
+    hq, hk, hv = (pu.to_dev(t[k]).cpu().pin_memory() for k in ("q", "k", "v"))
+    ho = torch.full(hq.shape, float("nan"), dtype=torch.bfloat16).pin_memory()
+    hl = torch.full((w.B, w.Hq, w.S), float("nan"), dtype=torch.float32).pin_memory()
+    from paper_2609_13612_b200 import binding
+    staging = torch.empty(binding.fwd_host_staging_bytes(w.B, w.Hq, w.Hkv, w.S, w.D), dtype=torch.uint8, device="cuda")
+    for _ in range(2):   # a second call reuses the staging buffer behind the first
+        af.fwd_host(hq, hk, hv, rope, table, mask, w.scale, ho, hl, staging)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    want_o, want_l = oracle.run_workload(w, t)
+    pu.assert_close(w.name + " O from host", pu.to_np(ho), want_o)
+    assert np.abs(hl.numpy() - want_l).max() <= pu.LSE_TOL
+    o_dev, l_dev = af.fwd(hq.cuda(), hk.cuda(), hv.cuda(), rope, table, mask, w.scale)
+    torch.cuda.synchronize()
+    assert torch.equal(o_dev.cpu(), ho) and torch.equal(l_dev.cpu(), hl)
+
+
 def test_forward_fp32_output():
     run_case(W("fp32_out", 1, 4, 2, 300, 128, theta=1e4, seed_id=120), out_dtype=torch.float32)
 
