@@ -405,10 +405,20 @@ def main():
             s = s5[i % len(s5)]
             af.bwd(s["q"], s["k"], s["v"], o5, l5, s["do"], r5, t5, m5, w5.scale, workspace=ws)
 
+        wsk5 = torch.empty(s5[0]["k"].numel() * 2, dtype=torch.uint8, device=dev)
+
+        def fb_hybrid(i):   # the same step with the hybrid forward (K rotated once by the RoPE pass)
+            s = s5[i % len(s5)]
+            af.fwd_hybrid(s["q"], s["k"], s["v"], r5, t5, m5, w5.scale, out=o5, lse=l5, workspace=wsk5)
+            af.bwd(s["q"], s["k"], s["v"], o5, l5, s["do"], r5, t5, m5, w5.scale, workspace=ws)
+
         t_fb, _, _ = timed(fb, k_ex, w_ex)
+        t_fbh, _, _ = timed(fb_hybrid, k_ex, w_ex)
         t_b, _, _ = timed(bonly, k_ex, w_ex)
         ex[w5.name] = {"fwd_bwd_ms": t_fb / k_ex,
                        "fwd_bwd_tflops": (w5.fwd_flops() + w5.bwd_flops()) / (t_fb / k_ex) / 1e9,
+                       "hybrid_fwd_bwd_ms": t_fbh / k_ex,
+                       "hybrid_fwd_bwd_tflops": (w5.fwd_flops() + w5.bwd_flops()) / (t_fbh / k_ex) / 1e9,
                        "bwd_ms": t_b / k_ex, "bwd_tflops": w5.bwd_flops() / (t_b / k_ex) / 1e9,
                        "bwd_pct_of_measured_peak": 100 * w5.bwd_flops() / (t_b / k_ex) / 1e9 / peaks["bf16_tflops"]}
         del s5
