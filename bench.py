@@ -519,6 +519,17 @@ def main():
                        "dense_fwd_ms_same_shape": t_df / k_ex, "speedup_over_dense": t_df / t_bf,
                        "bwd_ms": t_bb / k_ex, "bwd_tflops_on_kept_pairs": 2.5 * fl_b / (t_bb / k_ex) / 1e9,
                        "paper_fwd_ms_other_hardware": 0.084}
+        # a second mask at the density the paper quotes (about 7.7 % of the blocks): diagonal, global block column,
+        # and a seeded random block in every second row
+        act2 = _np.eye(nb_, dtype=bool)
+        act2[:, 0] = True
+        rows2 = _np.arange(0, nb_, 2)
+        act2[rows2, rng_.integers(1, nb_, size=rows2.size)] = True
+        bmask2 = af.BlockMask(act2, device=dev)
+        t_bf2, _, _ = timed(lambda i: af.fwd_blocks(sb[i % 2]["q"], sb[i % 2]["k"], sb[i % 2]["v"], rb_, tbb, mb_, wb.scale,
+                                                    bmask2, out=ob, lse=lb), k_ex, w_ex)
+        ex[wb.name]["at_paper_density"] = {"active_blocks": int(act2.sum()), "density": float(act2.mean()),
+                                           "fwd_ms": t_bf2 / k_ex, "speedup_over_dense": t_df / t_bf2}
         del sb
         torch.cuda.empty_cache()
         # Rotation Calculus sweep (Section 5.3): fused vs separate RoPE at constant B*S = 32768 tokens
