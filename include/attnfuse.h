@@ -129,6 +129,14 @@ typedef struct {
     const int* row_order; /* optional (NULL = 0, 1, 2, ...): the query row blocks in the order in which CTAs should be
                              launched, normally by decreasing list length so that the longest lists start first */
     const int* col_order; /* the same for key blocks (dK/dV kernel of the backward) */
+    /* Optional (all three NULL = not given), used by attnfuse_fwd_blocks when the GQA group is odd, where no two
+     * query heads share K and V: lists by PAIR of query row blocks (2r, 2r + 1), so that one CTA can work on two
+     * row blocks of a head at once.  pair_ptr [ceil(nb/2) + 1]; pair_idx: per pair the sorted union of the two
+     * row blocks' lists, each entry = key block | (1 << 28 if row block 2r lists it) | (1 << 29 if 2r + 1 does);
+     * pair_order: optional launch order of the pairs (NULL = 0, 1, 2, ...). */
+    const int* pair_ptr;
+    const int* pair_idx;
+    const int* pair_order;
 } af_blocks;
 
 /* attnfuse_fwd over the listed blocks. */

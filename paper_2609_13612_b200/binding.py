@@ -32,7 +32,8 @@ class _Strides(ctypes.Structure):
 class _Blocks(ctypes.Structure):
     _fields_ = [("block", ctypes.c_int), ("row_ptr", ctypes.c_void_p), ("col_idx", ctypes.c_void_p),
                 ("col_ptr", ctypes.c_void_p), ("row_idx", ctypes.c_void_p), ("row_order", ctypes.c_void_p),
-                ("col_order", ctypes.c_void_p)]
+                ("col_order", ctypes.c_void_p), ("pair_ptr", ctypes.c_void_p), ("pair_idx", ctypes.c_void_p),
+                ("pair_order", ctypes.c_void_p)]
 
 
 class _Rope(ctypes.Structure):
@@ -261,13 +262,27 @@ class BlockMask:
         # launch orders: longest lists first
         self.row_order = torch.argsort(counts, descending=True, stable=True).to(torch.int32).to(device)
         self.col_order = torch.argsort(counts_t, descending=True, stable=True).to(torch.int32).to(device)
+        # lists by pair of row blocks (2r, 2r + 1): sorted union, bit 28 / 29 = listed by the first / second row block
+        an = a.numpy()
+        ptr, idx = [0], []
+        for r in range(0, self.nb, 2):
+            first = an[r]
+            second = an[r + 1] if r + 1 < self.nb else first & False
+            for j in (first | second).nonzero()[0]:
+                idx.append(int(j) | (int(first[j]) << 28) | (int(second[j]) << 29))
+            ptr.append(len(idx))
+        self.pair_ptr = torch.tensor(ptr, dtype=torch.int32).to(device)
+        self.pair_idx = torch.tensor(idx if idx else [0], dtype=torch.int32).to(device)
+        plen = torch.tensor(ptr[1:], dtype=torch.int64) - torch.tensor(ptr[:-1], dtype=torch.int64)
+        self.pair_order = torch.argsort(plen, descending=True, stable=True).to(torch.int32).to(device)
         if self.col_idx.numel() == 0:   # keep the pointers valid
             self.col_idx = torch.zeros(1, dtype=torch.int32, device=device)
             self.row_idx = torch.zeros(1, dtype=torch.int32, device=device)
 
     def struct(self):
         return _Blocks(128, self.row_ptr.data_ptr(), self.col_idx.data_ptr(), self.col_ptr.data_ptr(),
-                       self.row_idx.data_ptr(), self.row_order.data_ptr(), self.col_order.data_ptr())
+                       self.row_idx.data_ptr(), self.row_order.data_ptr(), self.col_order.data_ptr(),
+                       self.pair_ptr.data_ptr(), self.pair_idx.data_ptr(), self.pair_order.data_ptr())
 
 
 def fwd_blocks(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor],

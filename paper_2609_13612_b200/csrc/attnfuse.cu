@@ -246,16 +246,20 @@ af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk
     auto kern = attn_fwd_kernel<D, NQ, ROPE, 2, 2, true>;
     static std::atomic<unsigned long long> configured{0};
     if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
-    p.pair_heads = NQ == 2 ? 1 : 0;
+    // NQ = 2: two heads of one kv head on the same row block (even GQA group), or - with pair lists - the row
+    // blocks 2 rb and 2 rb + 1 of one head
+    p.pair_heads = (NQ == 2 && !p.bs_rowpair) ? 1 : 0;
     p.n_row_blocks = (p.S + BM - 1) / BM;
-    dim3 grid(NQ == 2 ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
+    if (p.bs_rowpair) p.n_row_blocks = (p.n_row_blocks + 1) / 2;
+    dim3 grid(p.pair_heads ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
     kern<<<grid, 128 * (2 + NQ), L::BYTES, stream>>>(tq, tk, tv, to, tt, p);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 template <int D>
 af_status launch_fwd_blocks(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const CUtensorMap& tt,
                             const FwdParams& p, cudaStream_t stream) {
-    if ((p.group % 2) == 0)
+    // (p.bs_rowpair is set only for an odd GQA group, when the caller supplied the lists of row-block pairs)
+    if ((p.group % 2) == 0 || p.bs_rowpair)
         return p.R > 0 ? launch_fwd_blocks_variant<D, 2, true>(tq, tk, tv, to, tt, p, stream)
                        : launch_fwd_blocks_variant<D, 2, false>(tq, tk, tv, to, tt, p, stream);
     return p.R > 0 ? launch_fwd_blocks_variant<D, 1, true>(tq, tk, tv, to, tt, p, stream)
@@ -454,7 +458,8 @@ namespace {
 af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
                    const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
                    int gqa_group, float softmax_scale, const int* bs_row_ptr, const int* bs_col_idx,
-                   const int* bs_order, void* o, af_dtype o_dtype, float* lse, bool k_prerotated, void* cuda_stream) {
+                   const int* bs_order, void* o, af_dtype o_dtype, float* lse, bool k_prerotated, void* cuda_stream,
+                   const af_blocks* blocks = nullptr) {
     af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
     if (st != AF_OK) return st;
     if (!q || !k || !v || !o) return AF_ERR_NULL;
@@ -500,6 +505,14 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     p.bs_row_ptr = bs_row_ptr;
     p.bs_col_idx = bs_col_idx;
     p.bs_order = bs_order;
+    p.bs_rowpair = 0;
+    if (blocks && (gqa_group % 2) == 1 && blocks->pair_ptr && blocks->pair_idx && env_int("AF_BS_ROWPAIR", 1)) {
+        // odd GQA group: no two heads share K and V, so a CTA takes two row blocks of one head instead
+        p.bs_row_ptr = blocks->pair_ptr;
+        p.bs_col_idx = blocks->pair_idx;
+        p.bs_order = blocks->pair_order;
+        p.bs_rowpair = 1;
+    }
     p.rot_k = k_prerotated ? 0 : 1;
     p.keys_bf16 = keys_bf16 ? 1 : 0;
 #ifdef AF_TRACE
@@ -564,7 +577,7 @@ af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* 
     if (!blocks || !blocks->row_ptr || !blocks->col_idx) return AF_ERR_NULL;
     if (blocks->block != 128) return AF_ERR_SPEC;
     return fwd_impl(shape, q, k, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, blocks->row_ptr,
-                    blocks->col_idx, blocks->row_order, o, o_dtype, lse, false, cuda_stream);
+                    blocks->col_idx, blocks->row_order, o, o_dtype, lse, false, cuda_stream, blocks);
 }
 
 size_t attnfuse_fwd_host_staging_bytes(const af_shape* shape) {

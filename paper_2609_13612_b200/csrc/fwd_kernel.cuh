@@ -29,6 +29,10 @@ struct FwdParams {
     const int* bs_row_ptr;
     const int* bs_col_idx;
     const int* bs_order;   // optional launch order of the row blocks (longest lists first), or nullptr
+    // bs_rowpair (BS, NQ = 2, not pair_heads): the two query tiles of a CTA are the row blocks 2 rb and 2 rb + 1 of one
+    // head, and bs_row_ptr / bs_col_idx / bs_order describe PAIRS of row blocks: the list of pair rb is the sorted union
+    // of the two row blocks' lists, each entry = key block | (1 << 28 if row block 2 rb has it) | (1 << 29 if 2 rb + 1).
+    int bs_rowpair;
     int keys_bf16;         // host-side choice of the TAB instantiation (packed-bf16 key rotation)
     int rot_k;             // ROPE kernels: 1 = rotate the key tiles on chip; 0 = the keys arrive rotated (hybrid
                            // arm of Section 5.3: K rotated once by a RoPE pass, only Q rotated in the kernel)
@@ -237,7 +241,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     int jlo_c = 0x7fffffff, jhi_c = -1;
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
-        i0[q] = p.pair_heads ? rb * BM : (rb * NQ + q) * BM;
+        i0[q] = p.pair_heads ? rb * BM : (rb * NQ + q) * BM;   // (also the row-pair mode of the block lists)
         if (i0[q] < p.S) {
             tile_range(ms, i0[q], jlo[q], jhi[q]);
             jlo_c = min(jlo_c, jlo[q]);
@@ -250,9 +254,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // Block-sparse: the loops below run over positions in the row block's list (jlo = 0, jhi = length - 1, the
     // same for both query tiles, which share the row block); tile_at() gives the key tile of a position.
     int bs_base = 0;
+    int last_act[NQ];   // row-pair mode: last list position that is active for query tile q (-1: none)
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) last_act[q] = -1;
+    const bool rowpair = BS && NQ == 2 && p.bs_rowpair;
     if constexpr (BS) {
         bs_base = __ldg(p.bs_row_ptr + rb);
-        const int len = (rb * BM < p.S) ? __ldg(p.bs_row_ptr + rb + 1) - bs_base : 0;
+        const int first_row = rowpair ? rb * NQ * BM : rb * BM;
+        const int len = (first_row < p.S) ? __ldg(p.bs_row_ptr + rb + 1) - bs_base : 0;
 #pragma unroll
         for (int q = 0; q < NQ; ++q) {
             jlo[q] = 0;
@@ -260,8 +269,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         jlo_c = 0;
         jhi_c = len - 1;
+        if (rowpair) {
+            for (int pos = 0; pos < len; ++pos) {
+                const int ent = __ldg(p.bs_col_idx + bs_base + pos);
+#pragma unroll
+                for (int q = 0; q < NQ; ++q)
+                    if ((ent >> (28 + q)) & 1) last_act[q] = pos;
+            }
+#pragma unroll
+            for (int q = 0; q < NQ; ++q)
+                if (last_act[q] < 0 || i0[q] >= p.S) {   // nothing listed for this row block: treated as empty
+                    jlo[q] = 1;
+                    jhi[q] = 0;
+                }
+        }
     }
-    auto tile_at = [&](int pos) { return BS ? __ldg(p.bs_col_idx + bs_base + pos) : pos; };
+    auto tile_at = [&](int pos) { return BS ? (__ldg(p.bs_col_idx + bs_base + pos) & 0x0fffffff) : pos; };
+    // is list position / key tile j part of query tile q's work?
+    auto active = [&](int q, int j) {
+        if (rowpair) return jhi[q] >= jlo[q] && ((__ldg(p.bs_col_idx + bs_base + j) >> (28 + q)) & 1) != 0;
+        return j >= jlo[q] && j <= jhi[q];
+    };
+    auto is_last = [&](int q, int j) { return rowpair ? j == last_act[q] : j == jhi[q]; };
     const int n_it = jhi_c - jlo_c + 1;
     AF_STAMP(0, 63, 0);  // kernel entry
 
@@ -389,7 +418,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (ok && jhi[q] >= jlo[q]) {
                     ok = mbar_wait(&bars[B_QREADY + q], 0, abort_flag, 3);
                     tc_fence_after_sync();
-                    if (ok && jlo_c >= jlo[q] && jlo_c <= jhi[q]) issue_S(q, 0);
+                    if (ok && active(q, jlo_c)) issue_S(q, 0);
                 }
             }
             AF_STAMP(0, 63, 2);  // Q ready
@@ -403,7 +432,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 AF_STAMP(0, it, 1);
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
-                    if (ok && j >= jlo[q] && j <= jhi[q]) {
+                    if (ok && active(q, j)) {
 #pragma unroll
                         for (int pt = 0; pt < kPParts; ++pt) {
                             if (ok) ok = mbar_wait(&bars[L::B_PREADY + 4 * q + pt], cnt[q] & 1, abort_flag, 6);
@@ -416,10 +445,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         if (ok) {
                             AF_STAMP(0, it, 3 + 3 * q);
                             ++cnt[q];
-                            if (j == jhi[q]) mma_commit(&bars[L::B_ODONE + q]);
+                            if (is_last(q, j)) mma_commit(&bars[L::B_ODONE + q]);
                         }
                     }
-                    if (ok && next && j + 1 >= jlo[q] && j + 1 <= jhi[q]) {
+                    if (ok && next && active(q, j + 1)) {
                         if (!kwaited) {
                             ok = mbar_wait(&bars[B_KREADY + ks1], ((it + 1) / KS) & 1, abort_flag, 7);
                             tc_fence_after_sync();
@@ -541,7 +570,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             else if (p.R == 16) rot_q(std::integral_constant<int, 1>{});
             else rot_q(std::integral_constant<int, 0>{});
         }
-        for (int j = jlo[q]; ok && j <= jhi[q]; ++j, ++n) {
+        for (int j = jlo[q]; ok && j <= jhi[q]; ++j) {
+            if (rowpair && !active(q, j)) continue;   // a listed block of the other row block only
             const int j0 = tile_at(j) * BN;
             AF_STAMP(2 + q, n, 0);
             const bool need_mask = tile_needs_mask(ms, i0[q], j0);
@@ -559,6 +589,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 else ok = softmax_tile_halves<D, false, false>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
             }
             AF_STAMP(2 + q, n, 2);
+            ++n;
         }
         // epilogue (Section 4.4: save L = m + ln l)
         if (ok && jhi[q] >= jlo[q]) ok = mbar_wait_warp(&bars[L::B_ODONE + q], 0, abort_flag, 11);

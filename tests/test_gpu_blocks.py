@@ -73,6 +73,26 @@ def test_block_sparse_row_blocks_without_active_blocks_give_zero_rows():
     assert torch.all(o[:, :, 128:256] == 0) and torch.all(torch.isneginf(lse[:, :, 128:256]))
 
 
+def test_block_sparse_row_pairs_of_one_head():
+    """Odd GQA group: a CTA takes the row blocks 2r and 2r + 1 of one head and walks the union of their lists.  An odd
+    number of row blocks, a row block without blocks inside a pair, a pair without any block, causal + window + ALiBi."""
+    w = W("bs_rowpair_mixed", 2, 3, 3, 1100, 128, theta=1e4, window=500, alibi=True, seed_id=412)   # 9 row blocks
+    nb = 9
+    a = np.tril(bigbird_blocks(nb, seed=7, causal=True))
+    a[3, :] = False           # row block 3 (second of pair 1) has nothing
+    a[6, :] = a[7, :] = False   # pair 3 has nothing
+    t, dev, o, lse, _ = run_fwd(w, a)
+    for r in (3, 6, 7):
+        assert torch.all(o[:, :, 128 * r:128 * (r + 1)] == 0) and torch.all(torch.isneginf(lse[:, :, 128 * r:128 * (r + 1)]))
+
+
+@pytest.mark.parametrize("w,pattern", [FWD_CASES[4], FWD_CASES[5]], ids=lambda x: x.name if hasattr(x, "name") else "")
+def test_block_sparse_forward_one_row_block_per_cta(w, pattern, monkeypatch):
+    """The same odd-group cases without the pair lists (one query tile per CTA)."""
+    monkeypatch.setenv("AF_BS_ROWPAIR", "0")
+    run_fwd(w, pattern((w.S + 127) // 128))
+
+
 def test_block_sparse_all_active_equals_the_dense_kernel():
     w = W("bs_vs_dense", 1, 4, 2, 768, 128, theta=5e5, seed_id=411)
     t = synth.draw_all(w)
