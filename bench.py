@@ -555,6 +555,13 @@ def main():
         ex["rope_apply_kernel"] = {"bytes": 2 * x.numel() * 2, "ms": t_r / k_ex, "GB/s": gbs,
                                    "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]}
         line["extras"] = ex
+        # the three arms of the fuse-or-not experiment on the headline workload, side by side (TFLOP/s)
+        c2 = ex[synth.CONFIGS[1].name]
+        line["arms_on_headline_workload"] = {
+            "fused_single_kernel": c2["fused_fwd_tflops"], "separate_rope_then_attention": c2["separate_rope_fwd_tflops"],
+            "hybrid_k_prerotated_q_fused": c2["hybrid_fwd_tflops"],
+            "hybrid_frac_of_measured_burst_peak": c2["hybrid_frac_of_measured_burst_peak"],
+            "note": "value/roofline above are the single fused kernel; the other arms include their RoPE pass"}
 
     if rank == 0 and world == 1 and args.cpu_baseline:
         v, sample, _ = oracle_rate(w, 12.0)
