@@ -363,15 +363,12 @@ def main():
             return t / k_ex, ss
 
         # Optional forward mode: key tiles rotated in packed bf16 arithmetic from TMA-fed tiles of the table's bf16
-        # copy (environment switch read per call).  Faster, about 1.4 times the rounding error on rotated keys;
+        # copy (a tuning option of the library).  Faster, about 1.4 times the rounding error on rotated keys;
         # forward only, off by default - the headline above is the default fp32 rotation.
         wl = synth.CONFIGS[1]
         ms_d, ss = fwd_ms(wl, True)
-        os.environ["AF_FWD_KEYS_BF16"] = "1"
-        try:
+        with af.option(af.OPT_FWD_KEYS_BF16, 1):
             ms_b, _ = fwd_ms(wl, True, ss)
-        finally:
-            del os.environ["AF_FWD_KEYS_BF16"]
         ex["c2_keys_rotated_in_packed_bf16"] = {"default_fwd_ms": ms_d, "default_fwd_tflops": wl.fwd_flops() / ms_d / 1e9,
                                                 "mode_fwd_ms": ms_b, "mode_fwd_tflops": wl.fwd_flops() / ms_b / 1e9,
                                                 "mode_frac_of_measured_burst_peak": wl.fwd_flops() / ms_b / 1e9 / peaks["bf16_tflops"]}
@@ -451,7 +448,7 @@ def main():
         ms_b = bwd_ms(wc)
         ex[wc.name] = {"bwd_ms": ms_b, "bwd_tflops": wc.bwd_flops() / ms_b / 1e9}
         torch.cuda.empty_cache()
-        # Flash Decoding (Section 4.5, the paper's decode table): query length 1, D = 128, B = 1.  HBM-bound: the
+        # Flash Decoding (Section 4.2, the paper's decode table): query length 1, D = 128, B = 1.  HBM-bound: the
         # algorithmic bytes are the K and V caches, read once.  Caches rotate over sets larger than L2 in total.
         # Timed twice: as a replayed CUDA graph (device time per call) and through the C-ABI call from the host.
         dec = []
@@ -487,7 +484,7 @@ def main():
             del kcs, vcs
             torch.cuda.empty_cache()
         ex["flash_decoding"] = dec
-        # Block-sparse attention (Section 4.6): a BigBird-like mask over 32 x 32 blocks at N = 4096 in the geometry
+        # Block-sparse attention (Section 4.3): a BigBird-like mask over 32 x 32 blocks at N = 4096 in the geometry
         # of the paper's single-GPU tables (B = 4, 12 heads, D = 64), RoPE fused, no causal rule.  Diagonal blocks,
         # one global block column and row, one seeded random block per row.  FLOPs are counted on the kept pairs.
         import numpy as _np

@@ -62,9 +62,48 @@ typedef struct { int causal; int window; const float* alibi_slopes; } af_mask;
 int         attnfuse_version(void);
 const char* attnfuse_strerror(af_status st);
 
-/* Reads (and clears) the device status word of the current device; synchronises the device.
- * Returns AF_OK or AF_ERR_DEVICE_TIMEOUT; *detail (HOST, nullable) receives the raw word. */
+/* ---- tuning options ---------------------------------------------------------------------------------
+ * Process-wide switches between kernel variants that compute the same result (Section 3.2 makes such choices
+ * compile-time constants of the generated kernel; here they select among pre-built instantiations).  Each
+ * option starts from the environment variable named beside it, read once when the library first needs an
+ * option, else from its default; afterwards only attnfuse_set_option changes it.  Launches read the table,
+ * not the environment.  Setting an option while calls are in flight on other host threads affects only
+ * calls that start later.  attnfuse_set_option returns AF_ERR_SPEC for an unknown option;
+ * attnfuse_get_option returns -1 for one. */
+typedef enum {
+    AF_OPT_FWD_QTILES = 0,     /* AF_FWD_NQ, default 2: query tiles per CTA of the forward kernel (1 or 2) */
+    AF_OPT_FWD_PAIR_HEADS = 1, /* AF_FWD_PAIR, default 1: with an even GQA group the two query tiles of a CTA are two
+                                  heads of one kv head; 0: two consecutive row blocks of one head */
+    AF_OPT_FWD_KEYS_BF16 = 2,  /* AF_FWD_KEYS_BF16, default 0: key tiles rotated in packed bf16 arithmetic (faster,
+                                  about 1.4 times the rounding error on rotated keys; forward only) */
+    AF_OPT_FWD_CTA_PAIR = 3,   /* AF_FWD_2CTA, default 0: CTA-pair forward kernel for GQA groups that are multiples of 4 */
+    AF_OPT_BS_ROWPAIR = 4,     /* AF_BS_ROWPAIR, default 1: block-sparse forward with an odd GQA group gives a CTA two
+                                  row blocks of one head when the caller supplied pair lists */
+    AF_OPT_COUNT_ = 5
+} af_option;
+af_status attnfuse_set_option(af_option option, int value);
+int       attnfuse_get_option(af_option option);
+
+/* ---- device status (bounded waits) ------------------------------------------------------------------
+ * Every wait inside the kernels (on an mbarrier) gives up after about one second of SM clocks.  The kernel
+ * then records (wait-site code << 16 | low bits of the CTA index) in a status word of the current device,
+ * raises a CTA-wide flag that releases the CTA's other waits, frees its tensor memory and returns; the
+ * outputs of that launch are undefined and the context stays usable.  No entry point reports the word by
+ * itself: poll it with one of the two calls below (e.g. once per step).  Both return AF_OK or
+ * AF_ERR_DEVICE_TIMEOUT, store the raw word in *detail (HOST, nullable) and clear it when it was set.
+ *   attnfuse_device_status  synchronises the whole device first.
+ *   attnfuse_stream_status  reads the word in stream order on `cuda_stream` and synchronises only that
+ *                           stream: it sees every launch enqueued on the stream before the call.
+ * Neither may be called while a stream capture is in progress (they synchronise). */
 af_status attnfuse_device_status(unsigned int* detail);
+af_status attnfuse_stream_status(void* cuda_stream, unsigned int* detail);
+
+/* Self-test of that path (for tests and bring-up; no counterpart in the paper): launches one small CTA in which
+ * one warp waits, with a limit of `limit_cycles` SM clocks (1e3 .. 1e8), on a barrier that nothing ever
+ * arrives on, and a second warp waits on it with the normal limit.  The first wait runs out and records
+ * wait-site code 0x7e; the flag it raises releases the second warp; the kernel returns normally.  Afterwards
+ * attnfuse_stream_status / attnfuse_device_status report AF_ERR_DEVICE_TIMEOUT once, then AF_OK. */
+af_status attnfuse_selftest_wait_timeout(unsigned int limit_cycles, void* cuda_stream);
 
 /* ---- cos/sin table (set-up step of Section 4.1; cached by the caller) --------------------------
  * table: S * rotary_dim/2 pairs of fp32 {cos, sin}(p * theta^(-2i/rotary_dim)), p = pos_offset + s,
@@ -111,7 +150,7 @@ af_status attnfuse_fwd_hybrid(const af_shape* shape, const void* q, const void* 
                               void* o, af_dtype o_dtype, float* lse,
                               void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* ---- block-sparse attention (Section 4.6) ------------------------------------------------------------
+/* ---- block-sparse attention (Section 4.3) ------------------------------------------------------------
  * The caller evaluates its block predicate once and passes the active 128 x 128 blocks as index lists
  * (device memory, int32): by query row block (CSR: row_ptr [nb + 1], col_idx [row_ptr[nb]], nb = ceil(S/128))
  * and, for the backward, by key block (CSC: col_ptr [nb + 1], row_idx [col_ptr[nb]]).  Kernels visit only
@@ -162,7 +201,7 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
                             void* o_host, float* lse_host, void* staging, size_t staging_bytes,
                             void* cuda_stream);
 
-/* ---- Flash Decoding (Section 4.5; Table "Flash Decoding") ---------------------------------------------
+/* ---- Flash Decoding (Section 4.2; Table "Flash Decoding") ---------------------------------------------
  * One query position per head (the last one, N - 1) against a KV cache of N = shape->S keys:
  *   o[b,h,:] = softmax_j( c * <q[b,h], k[b,h/g,j]> + m_h (j - (N - 1)) ) v[b,h/g,j],  j kept iff j >= N - 1 - W.
  * Phase 1 splits the cache over n_splits CTAs per (batch, kv head); each computes a partial (max, sum,
@@ -172,7 +211,9 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
  * cached key precedes the query); window and ALiBi slopes apply as in attnfuse_fwd.
  * q, o: [B,Hq,D] bf16 contiguous (device); k, v: [B,Hkv,N,D] bf16 with strides skv (NULL = contiguous; the
  * rows need 16-byte alignment and strides that are multiples of 8 elements); lse (nullable): [B,Hq] fp32.
- * gqa_group <= 16; D in {64, 128}.  n_splits <= 0: attnfuse_decode_splits(shape) (about two CTAs per SM).
+ * gqa_group <= 16; D in {64, 128}.  n_splits <= 0: attnfuse_decode_splits(shape), the largest count that keeps the
+ * grid of n_splits x B x Hkv CTAs within one CTA per SM of the current device (one wave) with at least 128 keys
+ * per split.  Larger requests are clamped to ceil(S / 128) and to 256 splits.
  * workspace: attnfuse_decode_workspace_bytes(shape, n_splits) device bytes for the partials. */
 int       attnfuse_decode_splits(const af_shape* shape);
 size_t    attnfuse_decode_workspace_bytes(const af_shape* shape, int n_splits);
@@ -204,7 +245,7 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
                        void* dq, af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* attnfuse_bwd over the listed blocks (Section 4.6); needs both the CSR and the CSC lists of `blocks`.
+/* attnfuse_bwd over the listed blocks (Section 4.3); needs both the CSR and the CSC lists of `blocks`.
  * lse must come from attnfuse_fwd_blocks with the same lists; rows whose L is -inf get zero gradients. */
 af_status attnfuse_bwd_blocks(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,
                               const float* lse, const void* d_o,
@@ -220,7 +261,11 @@ af_status attnfuse_bwd_blocks(const af_shape* shape, const void* q, const void* 
  * frozen at start-up, code that runs while the allocator is locked by someone else.  For them this
  * variant of attnfuse_bwd keeps the one piece of scratch the backward needs (delta, one fp32 per
  * query row) in a fixed array inside the library instead of a caller workspace.  Inputs and outputs
- * are still the caller's, exactly as for attnfuse_bwd, and the results are the same.
+ * are still the caller's, exactly as for attnfuse_bwd.  The call always runs the delta-only set-up of
+ * attnfuse_bwd (both gradient kernels rotate what they touch on chip, nothing else is cached), whatever
+ * the problem size: its results are bit-identical to attnfuse_bwd given a workspace of exactly
+ * 4 * B*Hq*S bytes rounded up to 256, and equal to attnfuse_bwd with a full workspace up to the bf16
+ * rounding of a few rotated elements.
  *
  *  - Limit: B*Hq*S <= AF_BWD_STATIC_MAX_ROWS (4 MiB of scratch, which every GPU that loads the library
  *    holds until the process exits).  Larger problems return AF_ERR_STATIC_LIMIT and launch nothing.

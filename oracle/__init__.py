@@ -36,6 +36,10 @@ def _load():
         lib.af_oracle_fwd_blocks.restype = None
         lib.af_oracle_bwd_blocks.argtypes = [dp, dp, dp, dp, i, i, i, i, i, d, i, i, i, i, dp, d, bp, i, dp, dp, dp]
         lib.af_oracle_bwd_blocks.restype = None
+        lib.af_oracle_fwd_variant.argtypes = [dp, dp, dp, i, i, i, i, i, d, i, i, i, i, dp, d, bp, i, dp, i, i, i, ip, i, dp, dp]
+        lib.af_oracle_fwd_variant.restype = None
+        lib.af_oracle_bwd_variant.argtypes = [dp, dp, dp, dp, i, i, i, i, i, d, i, i, i, i, dp, d, bp, i, dp, i, i, i, dp, dp, dp]
+        lib.af_oracle_bwd_variant.restype = None
         _lib = lib
     return _lib
 
@@ -69,7 +73,7 @@ def _check(q, k, v):
 
 
 def _blocks(blocks, block_size, S):
-    """Active-block matrix [nb, nb] (Section 4.6) as contiguous bytes, or None."""
+    """Active-block matrix [nb, nb] (Section 4.3) as contiguous bytes, or None."""
     if blocks is None:
         return None, None
     nb = (S + block_size - 1) // block_size
@@ -78,12 +82,24 @@ def _blocks(blocks, block_size, S):
     return a, a.ctypes.data_as(ctypes.POINTER(ctypes.c_ubyte))
 
 
+def _bias(bias, B, Hq, S):
+    """additive_bias (Section 3.1): [Bb, Hb, S, S] with Bb in {1, B}, Hb in {1, Hq}, or None."""
+    if bias is None:
+        return None, 1, 1
+    a = _f64(bias)
+    assert a.ndim == 4 and a.shape[2:] == (S, S) and a.shape[0] in (1, B) and a.shape[1] in (1, Hq)
+    return a, a.shape[0], a.shape[1]
+
+
 def fwd(q, k, v, *, theta: float = 10000.0, rotary_dim: int = 0, pos_offset: int = 0,
         causal: bool = True, window: int = -1, slopes=None, scale: Optional[float] = None,
-        rows: Optional[Sequence[int]] = None, blocks=None, block_size: int = 128):
+        rows: Optional[Sequence[int]] = None, blocks=None, block_size: int = 128, bias=None,
+        normaliser: str = "softmax"):
     """O and L = m + ln(l) of the composed variant.  `rows`: optional subset of query
     rows (same for every head); then O is [B,Hq,len(rows),D].  `blocks`: optional [nb, nb] matrix of
-    active blocks (Section 4.6): pairs in inactive blocks are dropped on top of the element mask."""
+    active blocks (Section 4.3): pairs in inactive blocks are dropped on top of the element mask.
+    `bias`: additive_bias of Section 3.1.  normaliser "relu": relu_attention of Section 3.1 (L is None)."""
+    assert normaliser in ("softmax", "relu")
     q, k, v = _f64(q), _f64(k), _f64(v)
     B, Hq, Hkv, S, D = _check(q, k, v)
     scale = float(scale) if scale is not None else 1.0 / np.sqrt(D)
@@ -99,16 +115,19 @@ def fwd(q, k, v, *, theta: float = 10000.0, rotary_dim: int = 0, pos_offset: int
     o = np.empty((B, Hq, nr, D), dtype=np.float64)
     lse = np.empty((B, Hq, nr), dtype=np.float64)
     ba, bptr = _blocks(blocks, block_size, S)
-    _load().af_oracle_fwd_blocks(_p(q), _p(k), _p(v), B, Hq, Hkv, S, D, float(theta), int(rotary_dim),
-                                 int(pos_offset), int(bool(causal)), int(window), _p(sl), scale,
-                                 bptr, int(block_size), rp, nr, _p(o), _p(lse))
-    return o, lse
+    bi, bi_b, bi_h = _bias(bias, B, Hq, S)
+    relu = normaliser == "relu"
+    _load().af_oracle_fwd_variant(_p(q), _p(k), _p(v), B, Hq, Hkv, S, D, float(theta), int(rotary_dim),
+                                  int(pos_offset), int(bool(causal)), int(window), _p(sl), scale,
+                                  bptr, int(block_size), _p(bi), bi_b, bi_h, int(relu), rp, nr, _p(o), _p(lse))
+    return o, (None if relu else lse)
 
 
 def bwd(q, k, v, d_o, *, theta: float = 10000.0, rotary_dim: int = 0, pos_offset: int = 0,
         causal: bool = True, window: int = -1, slopes=None, scale: Optional[float] = None,
-        blocks=None, block_size: int = 128):
-    """dQ, dK, dV for upstream dO (Section 4.4 algebra, rotation transposed back)."""
+        blocks=None, block_size: int = 128, bias=None, normaliser: str = "softmax"):
+    """dQ, dK, dV for upstream dO (Section 4.4 algebra, rotation transposed back).  The bias gets no gradient."""
+    assert normaliser in ("softmax", "relu")
     q, k, v, d_o = _f64(q), _f64(k), _f64(v), _f64(d_o)
     B, Hq, Hkv, S, D = _check(q, k, v)
     assert d_o.shape == q.shape
@@ -118,9 +137,11 @@ def bwd(q, k, v, d_o, *, theta: float = 10000.0, rotary_dim: int = 0, pos_offset
     dk = np.empty_like(k)
     dv = np.empty_like(v)
     ba, bptr = _blocks(blocks, block_size, S)
-    _load().af_oracle_bwd_blocks(_p(q), _p(k), _p(v), _p(d_o), B, Hq, Hkv, S, D, float(theta), int(rotary_dim),
-                                 int(pos_offset), int(bool(causal)), int(window), _p(sl), scale,
-                                 bptr, int(block_size), _p(dq), _p(dk), _p(dv))
+    bi, bi_b, bi_h = _bias(bias, B, Hq, S)
+    _load().af_oracle_bwd_variant(_p(q), _p(k), _p(v), _p(d_o), B, Hq, Hkv, S, D, float(theta), int(rotary_dim),
+                                  int(pos_offset), int(bool(causal)), int(window), _p(sl), scale,
+                                  bptr, int(block_size), _p(bi), bi_b, bi_h, int(normaliser == "relu"),
+                                  _p(dq), _p(dk), _p(dv))
     return dq, dk, dv
 
 

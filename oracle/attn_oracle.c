@@ -16,12 +16,20 @@
  *  - Sliding window with causal: keep 0 <= i-j <= W (W+1 keys); without causal |i-j| <= W.
  *  - ALiBi: slope_h * (j - i) added after the softmax scale is applied.
  *  - Saved statistic (Section 4.4): L_i = m_i + ln(l_i), natural log.
- *  - Block-sparse attention (Section 4.6): the active-block lists only restrict the kept set: a pair
+ *  - Block-sparse attention (Section 4.3): the active-block lists only restrict the kept set: a pair
  *    (i, j) is kept iff the element mask keeps it AND block (i / bs, j / bs) is active.  Here the lists
  *    arrive as a dense nb x nb byte matrix (nb = ceil(S / bs)); a row with no kept pair gives O = 0,
  *    L = -inf and zero gradients.
  *  - Backward (Section 4.4, FlashAttention-2 algebra) with the chain rule through the
  *    rotation: gradients w.r.t. rotated rows are rotated back by the transpose.
+ *  - additive_bias (Section 3.1 names the combinator only): a dense tensor bias[bb, hh, i, j] added to the
+ *    scaled score after the softmax scale, like the ALiBi term; its batch and head extents are 1
+ *    (broadcast) or B / Hq.  A bias of -inf drops the pair like a mask.  The bias gets no gradient.
+ *  - relu_attention (Section 3.1 names the combinator only): the normaliser softmax is replaced by
+ *    P_ij = max(s_ij, 0) / n_i over the kept pairs, n_i = number of kept pairs of row i (the sequence
+ *    length when nothing is masked, which is the published ReLU-attention scaling); O_i = sum_j P_ij v_j.
+ *    There is no row statistic L for it.  Gradient: dS_ij = [s_ij > 0] <dO_i, v_j> / n_i.
+ *  - full (Section 3.1): no mask, i.e. causal = 0 and window < 0.
  */
 #include <math.h>
 #include <stdlib.h>
@@ -54,7 +62,7 @@ void af_oracle_rope(const double* x, double* y, int B, int H, int S, int D,
     }
 }
 
-/* Section 4.6: active-block matrix (NULL = every block active). */
+/* Section 4.3: active-block matrix (NULL = every block active). */
 typedef struct { const unsigned char* active; int bs, nb; } block_mask;
 
 static int kept(int i, int j, int causal, int window, const block_mask* bm)
@@ -74,12 +82,22 @@ static int kept(int i, int j, int causal, int window, const block_mask* bm)
  * Otherwise only the n_rows listed query rows (same list for every head):
  * o is [B,Hq,n_rows,D], lse [B,Hq,n_rows].  slopes: Hq doubles or NULL.
  */
-void af_oracle_fwd_blocks(const double* q, const double* k, const double* v,
-                          int B, int Hq, int Hkv, int S, int D,
-                          double theta, int R, int p0, int causal, int window,
-                          const double* slopes, double scale,
-                          const unsigned char* blocks, int block_size,
-                          const int* rows, int n_rows, double* o, double* lse)
+/* bias[bb, hh, i, j], bb = b or 0, hh = h or 0 (extents 1 broadcast); NULL = none */
+static double bias_at(const double* bias, int bias_B, int bias_H, int S, int b, int h, int i, int j)
+{
+    if (!bias) return 0.0;
+    long bb = bias_B == 1 ? 0 : b, hh = bias_H == 1 ? 0 : h;
+    return bias[((bb * bias_H + hh) * S + i) * (long)S + j];
+}
+
+/* Section 3.1, all combinators: relu != 0 selects the relu_attention normaliser (lse is then not written). */
+void af_oracle_fwd_variant(const double* q, const double* k, const double* v,
+                           int B, int Hq, int Hkv, int S, int D,
+                           double theta, int R, int p0, int causal, int window,
+                           const double* slopes, double scale,
+                           const unsigned char* blocks, int block_size,
+                           const double* bias, int bias_B, int bias_H, int relu,
+                           const int* rows, int n_rows, double* o, double* lse)
 {
     block_mask bmv = { blocks, block_size, block_size > 0 ? (S + block_size - 1) / block_size : 0 };
     const block_mask* bm = blocks ? &bmv : NULL;
@@ -105,12 +123,25 @@ void af_oracle_fwd_blocks(const double* q, const double* k, const double* v,
                 for (int d = 0; d < D; ++d) dot += qr[d] * kr[(long)j * D + d];
                 double s = scale * dot;
                 if (slopes) s += slopes[h] * (double)(j - i);
+                s += bias_at(bias, bias_B, bias_H, S, b, h, i, j);
                 sc[j] = s;
                 if (s > m) m = s;
             }
             double* orow = o + (((long)b * Hq + h) * nr + t) * D;
             for (int d = 0; d < D; ++d) orow[d] = 0.0;
             double l = 0.0;
+            if (relu) {
+                /* relu_attention: P_ij = max(s_ij, 0) / n_i over the kept pairs */
+                long n_kept = 0;
+                for (int j = 0; j < S; ++j) if (sc[j] != -INFINITY) ++n_kept;
+                if (n_kept == 0) continue;
+                for (int j = 0; j < S; ++j) {
+                    if (sc[j] == -INFINITY || sc[j] <= 0.0) continue;
+                    double p = sc[j] / (double)n_kept;
+                    for (int d = 0; d < D; ++d) orow[d] += p * vh[(long)j * D + d];
+                }
+                continue;
+            }
             if (m == -INFINITY) { lse[((long)b * Hq + h) * nr + t] = -INFINITY; continue; }
             for (int j = 0; j < S; ++j) {
                 if (sc[j] == -INFINITY) continue;
@@ -123,6 +154,17 @@ void af_oracle_fwd_blocks(const double* q, const double* k, const double* v,
         }
         free(kr); free(qr); free(sc);
     }
+}
+
+void af_oracle_fwd_blocks(const double* q, const double* k, const double* v,
+                          int B, int Hq, int Hkv, int S, int D,
+                          double theta, int R, int p0, int causal, int window,
+                          const double* slopes, double scale,
+                          const unsigned char* blocks, int block_size,
+                          const int* rows, int n_rows, double* o, double* lse)
+{
+    af_oracle_fwd_variant(q, k, v, B, Hq, Hkv, S, D, theta, R, p0, causal, window, slopes, scale, blocks, block_size,
+                          NULL, 1, 1, 0, rows, n_rows, o, lse);
 }
 
 void af_oracle_fwd(const double* q, const double* k, const double* v,
@@ -139,12 +181,13 @@ void af_oracle_fwd(const double* q, const double* k, const double* v,
  * Backward, given upstream dO [B,Hq,S,D].  Recomputes P from the definition.
  * dq [B,Hq,S,D], dk, dv [B,Hkv,S,D]; dk and dv of a kv head sum over its g query heads.
  */
-void af_oracle_bwd_blocks(const double* q, const double* k, const double* v, const double* d_o,
-                          int B, int Hq, int Hkv, int S, int D,
-                          double theta, int R, int p0, int causal, int window,
-                          const double* slopes, double scale,
-                          const unsigned char* blocks, int block_size,
-                          double* dq, double* dk, double* dv)
+void af_oracle_bwd_variant(const double* q, const double* k, const double* v, const double* d_o,
+                           int B, int Hq, int Hkv, int S, int D,
+                           double theta, int R, int p0, int causal, int window,
+                           const double* slopes, double scale,
+                           const unsigned char* blocks, int block_size,
+                           const double* bias, int bias_B, int bias_H, int relu,
+                           double* dq, double* dk, double* dv)
 {
     block_mask bmv = { blocks, block_size, block_size > 0 ? (S + block_size - 1) / block_size : 0 };
     const block_mask* bm = blocks ? &bmv : NULL;
@@ -178,11 +221,31 @@ void af_oracle_bwd_blocks(const double* q, const double* k, const double* v, con
                     for (int d = 0; d < D; ++d) dot += qr[d] * kr[(long)j * D + d];
                     double s = scale * dot;
                     if (slopes) s += slopes[h] * (double)(j - i);
+                    s += bias_at(bias, bias_B, bias_H, S, b, h, i, j);
                     pr[j] = s;
                     if (s > m) m = s;
                 }
                 for (int d = 0; d < D; ++d) { dqr[d] = 0.0; orow[d] = 0.0; }
                 if (m == -INFINITY) { for (int d = 0; d < D; ++d) dqh[(long)i * D + d] = 0.0; continue; }
+                if (relu) {
+                    /* relu_attention: P_ij = max(s_ij, 0) / n_i; dV_j += P_ij dO_i; dS_ij = [s_ij > 0] <dO_i, v_j> / n_i */
+                    long n_kept = 0;
+                    for (int j = 0; j < S; ++j) if (pr[j] != -INFINITY) ++n_kept;
+                    for (int j = 0; j < S; ++j) {
+                        if (pr[j] == -INFINITY || pr[j] <= 0.0) continue;
+                        double p = pr[j] / (double)n_kept;
+                        double dp = 0.0;
+                        for (int d = 0; d < D; ++d) dp += doi[d] * vh[(long)j * D + d];
+                        double ds = dp / (double)n_kept;
+                        for (int d = 0; d < D; ++d) {
+                            dvh[(long)j * D + d] += p * doi[d];
+                            dqr[d] += scale * ds * kr[(long)j * D + d];
+                            dkr[(long)j * D + d] += scale * ds * qr[d];
+                        }
+                    }
+                    rope_row(dqr, dqh + (long)i * D, D, R, theta, (long)p0 + i, -1);
+                    continue;
+                }
                 double l = 0.0;
                 for (int j = 0; j < S; ++j) {
                     if (pr[j] == -INFINITY) { pr[j] = 0.0; continue; }
@@ -215,6 +278,17 @@ void af_oracle_bwd_blocks(const double* q, const double* k, const double* v, con
         for (int j = 0; j < S; ++j) rope_row(dkr + (long)j * D, dkh + (long)j * D, D, R, theta, (long)p0 + j, -1);
         free(kr); free(dkr); free(qr); free(dqr); free(orow); free(pr);
     }
+}
+
+void af_oracle_bwd_blocks(const double* q, const double* k, const double* v, const double* d_o,
+                          int B, int Hq, int Hkv, int S, int D,
+                          double theta, int R, int p0, int causal, int window,
+                          const double* slopes, double scale,
+                          const unsigned char* blocks, int block_size,
+                          double* dq, double* dk, double* dv)
+{
+    af_oracle_bwd_variant(q, k, v, d_o, B, Hq, Hkv, S, D, theta, R, p0, causal, window, slopes, scale, blocks,
+                          block_size, NULL, 1, 1, 0, dq, dk, dv);
 }
 
 void af_oracle_bwd(const double* q, const double* k, const double* v, const double* d_o,

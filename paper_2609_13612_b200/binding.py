@@ -73,8 +73,16 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_version.restype = i
         L.attnfuse_strerror.restype = ctypes.c_char_p
         L.attnfuse_strerror.argtypes = [i]
+        L.attnfuse_set_option.restype = i
+        L.attnfuse_set_option.argtypes = [i, i]
+        L.attnfuse_get_option.restype = i
+        L.attnfuse_get_option.argtypes = [i]
         L.attnfuse_device_status.restype = i
         L.attnfuse_device_status.argtypes = [P(ctypes.c_uint)]
+        L.attnfuse_stream_status.restype = i
+        L.attnfuse_stream_status.argtypes = [vp, P(ctypes.c_uint)]
+        L.attnfuse_selftest_wait_timeout.restype = i
+        L.attnfuse_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp]
         L.attnfuse_rope_table_bytes.restype = sz
         L.attnfuse_rope_table_bytes.argtypes = [i, i]
         L.attnfuse_rope_table.restype = i
@@ -126,6 +134,34 @@ def version() -> int:
     return lib().attnfuse_version()
 
 
+# af_option values (include/attnfuse.h)
+OPT_FWD_QTILES, OPT_FWD_PAIR_HEADS, OPT_FWD_KEYS_BF16, OPT_FWD_CTA_PAIR, OPT_BS_ROWPAIR = range(5)
+
+
+def set_option(option: int, value: int) -> None:
+    _check(lib().attnfuse_set_option(option, value))
+
+
+def get_option(option: int) -> int:
+    return lib().attnfuse_get_option(option)
+
+
+class option:
+    """Context manager: a tuning option set for the duration of a block, then restored."""
+
+    def __init__(self, opt: int, value: int):
+        self.opt, self.value = opt, value
+
+    def __enter__(self):
+        self.old = get_option(self.opt)
+        set_option(self.opt, self.value)
+        return self
+
+    def __exit__(self, *exc):
+        set_option(self.opt, self.old)
+        return False
+
+
 def device_status() -> Tuple[int, int]:
     d = ctypes.c_uint(0)
     code = lib().attnfuse_device_status(ctypes.byref(d))
@@ -134,6 +170,18 @@ def device_status() -> Tuple[int, int]:
 
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
+
+
+def stream_status() -> Tuple[int, int]:
+    """Status word read in order on the current stream (synchronises that stream only)."""
+    d = ctypes.c_uint(0)
+    code = lib().attnfuse_stream_status(_stream(), ctypes.byref(d))
+    return code, d.value
+
+
+def selftest_wait_timeout(limit_cycles: int = 2_000_000) -> None:
+    """Launch the self-test CTA whose bounded wait runs out after `limit_cycles` SM clocks."""
+    _check(lib().attnfuse_selftest_wait_timeout(limit_cycles, _stream()))
 
 
 def _need_cuda(*ts):
@@ -244,7 +292,7 @@ def fwd_hybrid(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: Rop
 
 
 class BlockMask:
-    """Active 128 x 128 blocks of a block-sparse mask (Section 4.6) as device index lists: CSR by query row
+    """Active 128 x 128 blocks of a block-sparse mask (Section 4.3) as device index lists: CSR by query row
     block and CSC by key block.  Built once from a boolean [nb, nb] matrix (nb = ceil(S / 128))."""
 
     def __init__(self, active, device="cuda"):

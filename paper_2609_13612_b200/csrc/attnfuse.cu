@@ -12,6 +12,7 @@
 #include "../../include/attnfuse.h"
 #include "fwd_kernel.cuh"
 #include "bwd_kernel.cuh"
+#include "bwd_first_rows.cuh"
 #include "decode_kernels.cuh"
 #include "fwd2_kernel.cuh"
 #include "rope_kernels.cuh"
@@ -75,18 +76,52 @@ af_status make_tmap_table(CUtensorMap* tm, const void* table, int S, int R) {
     return r == CUDA_SUCCESS ? AF_OK : AF_ERR_CUDA;
 }
 
-int env_int(const char* name, int dflt) {
-    const char* v = getenv(name);
-    return v ? atoi(v) : dflt;
+// Tuning options (attnfuse_set_option / attnfuse_get_option): a process-wide table of atomics.  Each entry
+// takes its initial value from the environment variable of the same name once, when the table is first
+// touched; launches read the table, never the environment.
+struct OptionDef { const char* env; int dflt; };
+constexpr OptionDef kOptionDefs[AF_OPT_COUNT_] = {
+    {"AF_FWD_NQ", 2},           // AF_OPT_FWD_QTILES
+    {"AF_FWD_PAIR", 1},         // AF_OPT_FWD_PAIR_HEADS
+    {"AF_FWD_KEYS_BF16", 0},    // AF_OPT_FWD_KEYS_BF16
+    {"AF_FWD_2CTA", 0},         // AF_OPT_FWD_CTA_PAIR
+    {"AF_BS_ROWPAIR", 1},       // AF_OPT_BS_ROWPAIR
+};
+std::atomic<int> g_options[AF_OPT_COUNT_];
+std::once_flag g_options_once;
+void init_options() {
+    std::call_once(g_options_once, [] {
+        for (int i = 0; i < AF_OPT_COUNT_; ++i) {
+            const char* v = getenv(kOptionDefs[i].env);
+            g_options[i].store(v ? atoi(v) : kOptionDefs[i].dflt, std::memory_order_relaxed);
+        }
+    });
+}
+int opt(af_option o) {
+    init_options();
+    return g_options[o].load(std::memory_order_relaxed);
 }
 
-// AF_FWD_KEYS_BF16=1 (forward only, rotary widths 16, 32, 64, 128): key tiles are rotated in packed bf16
+// AF_OPT_FWD_KEYS_BF16 (forward only, rotary widths 16, 32, 64, 128): key tiles are rotated in packed bf16
 // arithmetic from the table's bf16 copy instead of fp32 arithmetic from the fp32 rows.  Faster (the rotation
 // competes with the softmax for issue slots), but a rotated key then carries about three bf16 roundings instead
 // of one; the backward pass always rotates in fp32, so a log-sum-exp produced in this mode is slightly
 // inconsistent with the scores the backward pass recomputes.  Off by default.
 bool keys_rotate_in_bf16(int R) {
-    return (R == 16 || R == 32 || R == 64 || R == 128) && env_int("AF_FWD_KEYS_BF16", 0);
+    return (R == 16 || R == 32 || R == 64 || R == 128) && opt(AF_OPT_FWD_KEYS_BF16);
+}
+
+// Number of SMs of the current device (cached per device ordinal).
+int sm_count() {
+    static std::atomic<int> cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    int n = cached[dev & 63].load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 0;
+        cached[dev & 63].store(n, std::memory_order_relaxed);
+    }
+    return n;
 }
 
 // Opt a kernel in to its dynamic shared-memory size once per device (the attribute is per device and per
@@ -197,7 +232,7 @@ af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const
     static std::atomic<unsigned long long> configured{0};
     if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
     // an even GQA group lets the two query tiles of a CTA be two heads of one kv head (same key range)
-    p.pair_heads = (NQ == 2 && (p.group % 2) == 0 && env_int("AF_FWD_PAIR", 1)) ? 1 : 0;
+    p.pair_heads = (NQ == 2 && (p.group % 2) == 0 && opt(AF_OPT_FWD_PAIR_HEADS)) ? 1 : 0;
     const int rows_per_cta = p.pair_heads ? BM : BM * NQ;
     p.n_row_blocks = (p.S + rows_per_cta - 1) / rows_per_cta;
     dim3 grid(p.pair_heads ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
@@ -237,7 +272,7 @@ af_status launch_fwd2_variant(const CUtensorMap& tq, const CUtensorMap& tk2, con
     return cudaLaunchKernelEx(&cfg, kern, tq, tk2, tv, p) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
-// Block-sparse variant (Section 4.6): the grid is (heads or head pairs, 128-row blocks); every CTA walks the
+// Block-sparse variant (Section 4.3): the grid is (heads or head pairs, 128-row blocks); every CTA walks the
 // list of active key blocks of its row block.  An even GQA group pairs two heads per CTA, otherwise one head.
 template <int D, int NQ, bool ROPE>
 af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
@@ -269,7 +304,7 @@ af_status launch_fwd_blocks(const CUtensorMap& tq, const CUtensorMap& tk, const 
 template <int D>
 af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const CUtensorMap& tt, const FwdParams& p,
                      cudaStream_t stream) {
-    const int nq = env_int("AF_FWD_NQ", 2);
+    const int nq = opt(AF_OPT_FWD_QTILES);
     if (nq == 1) {
         return p.R > 0 ? launch_fwd_variant<D, 1, true, 2, 2>(tq, tk, tv, to, tt, p, stream)
                        : launch_fwd_variant<D, 1, false, 2, 2>(tq, tk, tv, to, tt, p, stream);
@@ -316,12 +351,42 @@ af_status launch_rope(const void* x_in, const af_strides& st, void* x_out, int B
 // delta, then the two gradient kernels.  tkp / tqp: tensor maps over the rotated-K and rotated-Q caches in
 // the workspace, or nullptr when the workspace has no room for them (see bwd_kernel.cuh for the three set-ups).
 // k / stkv / kcache: the caller's K, its strides and the K' cache, for the RoPE pass of the two-cache set-up.
+// The first query rows of every head in fp32, after the MMA kernels of the sequence (see bwd_first_rows.cuh).
+template <int D>
+af_status launch_first_rows(const FirstRowsParams& fp, cudaStream_t stream) {
+    using L = FirstRowsSmem<D>;
+    auto kern = bwd_first_rows_kernel<D>;
+    static std::atomic<unsigned long long> configured{0};
+    if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
+    return launch_kernel(kern, dim3(fp.B * fp.Hkv, 1, 1), dim3(256, 1, 1), L::BYTES, stream, true, fp);
+}
+
+template <int D>
+af_status launch_bwd_mma(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                         const CUtensorMap& tdo, const CUtensorMap* tkp, const CUtensorMap* tqp, const void* k,
+                         const af_strides& stkv, void* kcache, const void* o, const void* d_o, BwdParams p, void* dq,
+                         int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, const af_blocks* blocks,
+                         cudaStream_t stream);
+
 template <int D>
 af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                      const CUtensorMap& tdo, const CUtensorMap* tkp, const CUtensorMap* tqp, const void* k,
                      const af_strides& stkv, void* kcache, const void* o, const void* d_o, BwdParams p, void* dq,
                      int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, const af_blocks* blocks,
-                     cudaStream_t stream) {
+                     cudaStream_t stream, const FirstRowsParams& fp) {
+    p.skip_rows = fp.rows;
+    af_status st = launch_bwd_mma<D>(sh, tq, tk, tv, tdo, tkp, tqp, k, stkv, kcache, o, d_o, p, dq, dq_f32, dk, dv, dkv_f32,
+                                     delta, blocks, stream);
+    if (st != AF_OK || fp.rows == 0) return st;
+    return launch_first_rows<D>(fp, stream);
+}
+
+template <int D>
+af_status launch_bwd_mma(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                         const CUtensorMap& tdo, const CUtensorMap* tkp, const CUtensorMap* tqp, const void* k,
+                         const af_strides& stkv, void* kcache, const void* o, const void* d_o, BwdParams p, void* dq,
+                         int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, const af_blocks* blocks,
+                         cudaStream_t stream) {
     // block lists by stationary block: by key block for the dK/dV role, by query block for the dQ role
     auto role_lists = [&](bool dkv_role) {
         p.bs_ptr = blocks ? (dkv_role ? blocks->col_ptr : blocks->row_ptr) : nullptr;
@@ -336,7 +401,12 @@ af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMa
     p.delta = delta;
     const unsigned tiles = static_cast<unsigned>((sh->S + 127) / 128);
     af_status st;
-    const int only = env_int("AF_BWD_ONLY", 0);   // tuning aid: 1 = dK/dV kernel only, 2 = dQ kernel only
+#ifdef AF_TRACE
+    // tracing builds only: 1 = dK/dV kernel only, 2 = dQ kernel only (the skipped outputs stay unwritten)
+    const int only = getenv("AF_BWD_ONLY") ? atoi(getenv("AF_BWD_ONLY")) : 0;
+#else
+    constexpr int only = 0;
+#endif
     dim3 gkv(sh->B * sh->Hkv, tiles, 1), gq(sh->B * sh->Hq, tiles, 1);
     if (p.R > 0 && tkp && tqp && only == 0) {
         // both caches: K' by the RoPE pass, Q' by the dQ kernel, no on-chip rotation in the dK/dV loop
@@ -396,6 +466,33 @@ const char* attnfuse_strerror(af_status st) {
     return "unknown status";
 }
 
+af_status attnfuse_set_option(af_option option, int value) {
+    if (option < 0 || option >= AF_OPT_COUNT_) return AF_ERR_SPEC;
+    init_options();
+    g_options[option].store(value, std::memory_order_relaxed);
+    return AF_OK;
+}
+
+int attnfuse_get_option(af_option option) {
+    if (option < 0 || option >= AF_OPT_COUNT_) return -1;
+    return opt(option);
+}
+
+af_status attnfuse_stream_status(void* cuda_stream, unsigned int* detail) {
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    unsigned int w = 0, zero = 0;
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, af::g_device_status) != cudaSuccess) return AF_ERR_CUDA;
+    if (cudaMemcpyAsync(&w, addr, sizeof(w), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return AF_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return AF_ERR_CUDA;
+    if (w) {
+        if (cudaMemcpyAsync(addr, &zero, sizeof(zero), cudaMemcpyHostToDevice, stream) != cudaSuccess) return AF_ERR_CUDA;
+        if (cudaStreamSynchronize(stream) != cudaSuccess) return AF_ERR_CUDA;
+    }
+    if (detail) *detail = w;
+    return w ? AF_ERR_DEVICE_TIMEOUT : AF_OK;
+}
+
 af_status attnfuse_device_status(unsigned int* detail) {
     unsigned int w = 0, zero = 0;
     if (cudaDeviceSynchronize() != cudaSuccess) return AF_ERR_CUDA;
@@ -403,6 +500,14 @@ af_status attnfuse_device_status(unsigned int* detail) {
     if (w && cudaMemcpyToSymbol(af::g_device_status, &zero, sizeof(zero)) != cudaSuccess) return AF_ERR_CUDA;
     if (detail) *detail = w;
     return w ? AF_ERR_DEVICE_TIMEOUT : AF_OK;
+}
+
+af_status attnfuse_selftest_wait_timeout(unsigned int limit_cycles, void* cuda_stream) {
+    if (limit_cycles < 1000u || limit_cycles > 100000000u) return AF_ERR_SPEC;
+    af_status st = check_arch();
+    if (st != AF_OK) return st;
+    wait_timeout_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(cuda_stream)>>>(static_cast<long long>(limit_cycles));
+    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
 size_t attnfuse_rope_table_bytes(int S, int rotary_dim) {
@@ -506,7 +611,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     p.bs_col_idx = bs_col_idx;
     p.bs_order = bs_order;
     p.bs_rowpair = 0;
-    if (blocks && (gqa_group % 2) == 1 && blocks->pair_ptr && blocks->pair_idx && env_int("AF_BS_ROWPAIR", 1)) {
+    if (blocks && (gqa_group % 2) == 1 && blocks->pair_ptr && blocks->pair_idx && opt(AF_OPT_BS_ROWPAIR)) {
         // odd GQA group: no two heads share K and V, so a CTA takes two row blocks of one head instead
         p.bs_row_ptr = blocks->pair_ptr;
         p.bs_col_idx = blocks->pair_idx;
@@ -524,7 +629,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
         return shape->D == 128 ? launch_fwd_blocks<128>(tq, tk, tv, to, tt, p, stream) : launch_fwd_blocks<64>(tq, tk, tv, to, tt, p, stream);
     const int R = rope->rotary_dim;
     const bool pair_ok = shape->D == 128 && (gqa_group % 4) == 0 && (R == 0 || R == 16 || R == 32 || R == 64 || R == 128);
-    if (pair_ok && !k_prerotated && env_int("AF_FWD_2CTA", 0)) {
+    if (pair_ok && !k_prerotated && opt(AF_OPT_FWD_CTA_PAIR)) {
         CUtensorMap tk2;
         if ((st = make_tmap(&tk2, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, 64)) != AF_OK) return st;
         return R > 0 ? launch_fwd2_variant<true>(tq, tk2, tv, p, stream) : launch_fwd2_variant<false>(tq, tk2, tv, p, stream);
@@ -622,6 +727,25 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
     std::lock_guard<std::mutex> lock(g_pipe_mutex);
     HostPipe* pipe = get_pipe();
     if (!pipe) return AF_ERR_CUDA;
+    // Whatever happens below, work may already sit on the internal streams when the call returns: on every exit
+    // path the caller's stream is made to wait for it, so that reusing `staging` or the host buffers afterwards
+    // (in stream order) cannot race with copies or kernels still in flight.
+    struct JoinOnExit {
+        HostPipe* pipe;
+        cudaStream_t stream;
+        bool done = false;
+        af_status join() {
+            done = true;
+            cudaEvent_t a = pipe->ev[pipe->next];
+            pipe->next = (pipe->next + 1) % HostPipe::kEvents;
+            cudaEvent_t b = pipe->ev[pipe->next];
+            pipe->next = (pipe->next + 1) % HostPipe::kEvents;
+            bool ok = cudaEventRecord(a, pipe->compute) == cudaSuccess && cudaStreamWaitEvent(stream, a, 0) == cudaSuccess;
+            ok = cudaEventRecord(b, pipe->d2h) == cudaSuccess && cudaStreamWaitEvent(stream, b, 0) == cudaSuccess && ok;
+            return ok ? AF_OK : AF_ERR_CUDA;
+        }
+        ~JoinOnExit() { if (!done) join(); }
+    } joiner{pipe, stream};
     auto next_event = [&]() {
         cudaEvent_t e = pipe->ev[pipe->next];
         pipe->next = (pipe->next + 1) % HostPipe::kEvents;
@@ -679,18 +803,17 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
     const size_t ln = static_cast<size_t>(shape->B) * shape->Hq * shape->S * 4;
     if (lse_host && cudaMemcpyAsync(lse_host, dl, ln, cudaMemcpyDeviceToHost, pipe->d2h) != cudaSuccess) return AF_ERR_CUDA;
     // the caller's stream continues once the last results are on the host
-    cudaEvent_t e_done = next_event();
-    if (cudaEventRecord(e_done, pipe->d2h) != cudaSuccess || cudaStreamWaitEvent(stream, e_done, 0) != cudaSuccess)
-        return AF_ERR_CUDA;
-    return AF_OK;
+    return joiner.join();
 }
 
 int attnfuse_decode_splits(const af_shape* shape) {
     if (!shape || shape->B < 1 || shape->Hkv < 1 || shape->S < 1) return 0;
     // one CTA per SM fits (its stages take most of the shared memory): as many splits as give at most one
-    // CTA per SM (148 SMs) in a single wave, at least 128 keys (one tile per warp) per split
+    // CTA per SM of the current device in a single wave, at least 128 keys (one tile per warp) per split
     const int ctas_per_split = shape->B * shape->Hkv;
-    const int want = 148 / ctas_per_split;
+    int sms = sm_count();
+    if (sms < 1) sms = 148;   // no device to ask (host-only callers sizing a workspace): the B200 count
+    const int want = sms / ctas_per_split;
     const int most = (shape->S + 127) / 128;
     return want < 1 ? 1 : (want > most ? most : want);
 }
@@ -793,7 +916,7 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     p.table = static_cast<const float2*>(rope_table);
     p.lse = lse;
     p.delta = nullptr; p.out1 = nullptr; p.out2 = nullptr; p.out_f32 = 0; p.store_x = 0;
-    p.bs_ptr = nullptr; p.bs_idx = nullptr; p.bs_order = nullptr;
+    p.bs_ptr = nullptr; p.bs_idx = nullptr; p.bs_order = nullptr; p.skip_rows = 0;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     float* delta = static_cast<float*>(workspace);
     // rotated-K and rotated-Q caches: used when there is a rotation and the workspace has room behind delta
@@ -811,11 +934,24 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
         void* qc = static_cast<uint8_t*>(workspace) + off_q;
         if ((st = make_tmap(&tqp, qc, shape->B, shape->Hq, shape->S, shape->D, stc, 128)) != AF_OK) return st;
     }
+    // Under a causal mask (dense, not over block lists) the first query rows of every head are computed in fp32 by a
+    // small kernel of their own and dropped from the MMA kernels: see bwd_first_rows.cuh.
+    FirstRowsParams fp = {};
+    fp.B = shape->B; fp.Hq = shape->Hq; fp.Hkv = shape->Hkv; fp.S = shape->S; fp.group = gqa_group;
+    fp.R = p.R; fp.window = p.window;
+    fp.rows = (p.causal && !blocks) ? (shape->S < kFirstRows ? shape->S : kFirstRows) : 0;
+    fp.scale = softmax_scale;
+    fp.slopes = p.slopes; fp.table = p.table;
+    fp.q = static_cast<const __nv_bfloat16*>(q); fp.k = static_cast<const __nv_bfloat16*>(k);
+    fp.v = static_cast<const __nv_bfloat16*>(v); fp.d_o = static_cast<const __nv_bfloat16*>(d_o);
+    fp.qb = stq.b; fp.qh = stq.h; fp.qs = stq.s; fp.kb = stkv.b; fp.kh = stkv.h; fp.ks = stkv.s;
+    fp.dq = dq; fp.dk = dk; fp.dv = dv;
+    fp.dq_f32 = dq_dtype == AF_F32; fp.dkv_f32 = dkv_dtype == AF_F32;
     return shape->D == 128
                ? launch_bwd<128>(shape, tq, tk, tv, tdo, have_k ? &tkp : nullptr, have_q ? &tqp : nullptr, k, stkv, kc, o,
-                                 d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream)
+                                 d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream, fp)
                : launch_bwd<64>(shape, tq, tk, tv, tdo, have_k ? &tkp : nullptr, have_q ? &tqp : nullptr, k, stkv, kc, o,
-                                d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream);
+                                d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream, fp);
 }
 }  // namespace
 
@@ -867,6 +1003,7 @@ extern "C" af_status attnfuse_bwd_static(const af_shape* shape, const void* q, c
     if (shape->B < 1 || shape->Hq < 1 || shape->S < 1) return AF_ERR_SHAPE;
     const long long rows = static_cast<long long>(shape->B) * shape->Hq * shape->S;
     if (rows > AF_BWD_STATIC_MAX_ROWS) return AF_ERR_STATIC_LIMIT;
+    static_assert(sizeof(g_bwd_static_scratch) >= AF_BWD_STATIC_MAX_ROWS * sizeof(float) + 256, "scratch holds delta");
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return AF_ERR_CUDA;
     if (dev < 0 || dev >= kMaxDevices) return AF_ERR_CUDA;
@@ -881,6 +1018,8 @@ extern "C" af_status attnfuse_bwd_static(const af_shape* shape, const void* q, c
         }
         scratch = g_bwd_static_ptr[dev];
     }
+    // the size passed is delta's alone, so that the call always takes the delta-only set-up whatever the problem
+    // size (with more room attnfuse_bwd would also place its rotated-K / rotated-Q caches in the array)
     return attnfuse_bwd(shape, q, k, v, o, lse, d_o, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, dq,
-                        dq_dtype, dk, dv, dkv_dtype, scratch, sizeof(g_bwd_static_scratch), cuda_stream);
+                        dq_dtype, dk, dv, dkv_dtype, scratch, bwd_delta_bytes(shape), cuda_stream);
 }

@@ -37,12 +37,13 @@ struct BwdParams {
     void* out2;           // DKV: dK   DQ: unused
     int out_f32;
     int store_x;          // write the rotated X tile through tm_s
-    // Block-sparse attention (Section 4.6), BS kernels only: index lists of the active 128 x 128 blocks by
+    // Block-sparse attention (Section 4.3), BS kernels only: index lists of the active 128 x 128 blocks by
     // stationary block - for the dK/dV role by key block (the query blocks that see it), for the dQ role by
     // query block (its key blocks): ptr [ceil(S/128) + 1], idx [ptr[last]] (device).
     const int* bs_ptr;
     const int* bs_idx;
     const int* bs_order;   // optional launch order of the stationary blocks (longest lists first), or nullptr
+    int skip_rows;         // query rows i < skip_rows are left to bwd_first_rows_kernel (0: none)
 };
 
 // delta[row] = <dO[row], O[row]>; one 16-byte chunk per thread, D/8 threads per row.
@@ -275,7 +276,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::OFF_MISC + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const MaskSpec ms{p.S, p.causal, p.window};
+    const MaskSpec ms{p.S, p.causal, p.window, p.skip_rows};
     // stationary tile: DKV -> key tile of kv head (b, hk); DQ -> query tile of head (b, h)
     const int xh_count = DKV ? p.Hkv : p.Hq;
     const int b = blockIdx.x / xh_count, xh = blockIdx.x - b * xh_count;

@@ -14,6 +14,8 @@ struct MaskSpec {
     int S;
     int causal;
     int window;  // < 0: none; host clamps to S
+    int skip_rows = 0;  // backward only: query rows below this are computed by the first-rows kernel, so the
+                        // MMA kernels drop every pair (i, j) with i < skip_rows
 };
 
 // Key-tile range [jlo, jhi] that a query tile starting at row i0 can see (Section 5: fully masked
@@ -38,6 +40,7 @@ __device__ __forceinline__ void qtile_range(const MaskSpec& m, int j0, int& ilo,
 // True if some (i, j) of the tile pair is masked out, so per-element mask logic is needed.
 __device__ __forceinline__ bool tile_needs_mask(const MaskSpec& m, int i0, int j0) {
     if (j0 + BN > m.S) return true;
+    if (i0 < m.skip_rows) return true;
     if (m.causal && j0 + BN - 1 > i0) return true;
     if (m.window >= 0) {
         if (i0 + BM - 1 - j0 > m.window) return true;
@@ -71,12 +74,12 @@ __device__ __forceinline__ void kept_keys_of_query(const MaskSpec& m, int i, int
         lo = max(lo, d - m.window);
         if (!m.causal) hi = min(hi, d + m.window);
     }
-    n = hi >= lo ? static_cast<uint32_t>(hi - lo + 1) : 0u;
+    n = (hi >= lo && i >= m.skip_rows) ? static_cast<uint32_t>(hi - lo + 1) : 0u;
 }
 __device__ __forceinline__ void kept_queries_of_key(const MaskSpec& m, int j, int i0, int& lo, uint32_t& n) {
     const int d = j - i0;
     int hi = BM - 1;
-    lo = 0;
+    lo = max(0, m.skip_rows - i0);
     if (m.causal) lo = max(lo, d);
     if (m.window >= 0) {
         hi = min(hi, d + m.window);

@@ -1,4 +1,4 @@
-// Flash Decoding (Section 4.5 of the paper): one query position per head against a long KV cache.
+// Flash Decoding (Section 4.2 of the paper): one query position per head against a long KV cache.
 //
 // Phase 1 (decode_split_kernel): the cache is cut into splits; a CTA takes one split of one kv head
 // and computes, for the g query heads of that kv head, a partial (m, l, acc) triple with the online

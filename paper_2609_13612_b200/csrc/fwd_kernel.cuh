@@ -23,7 +23,7 @@ struct FwdParams {
     float* lse;         // nullable
     int n_row_blocks;   // ceil(S / (128 * NQ)), or ceil(S / 128) with pair_heads
     int pair_heads;     // NQ = 2 only: the two query tiles are the same 128 rows of two heads of one kv group
-    // Block-sparse attention (Section 4.6), BS kernels only: CSR lists of the active 128 x 128 blocks, row_ptr
+    // Block-sparse attention (Section 4.3), BS kernels only: CSR lists of the active 128 x 128 blocks, row_ptr
     // [ceil(S/128) + 1] and col_idx [row_ptr[last]] (device).  The key loop walks a row block's list instead of
     // a contiguous tile range; the element mask (causal, window) still applies inside the listed tiles.
     const int* bs_row_ptr;

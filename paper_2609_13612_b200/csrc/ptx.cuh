@@ -49,7 +49,7 @@ constexpr long long kWaitLimitCycles = 2000000000LL;
 // Bounded wait.  Returns false if it gave up (limit reached, or another thread already aborted).
 // `abort_flag` lives in shared memory; `code` identifies the wait site.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t code) {
+                                          uint32_t code, long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     long long t0 = clock64();
     uint32_t spins = 0;
@@ -57,7 +57,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1u;
                 atomicCAS(&g_device_status, 0u, (code << 16) | (blockIdx.x & 0xffffu));
                 return false;
@@ -70,8 +70,27 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 // warp-collective tcgen05.ld/st): all 32 lanes wait, and all of them give up if any of them did.
 // (Letting only lane 0 poll was measured slower: the warp woke up later.)
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                               uint32_t code) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, code));
+                                               uint32_t code, long long limit_cycles = kWaitLimitCycles) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, code, limit_cycles));
+}
+
+// Self-test of the time-out path: one CTA, one barrier that nothing ever arrives on.  Warp 1 waits on it with
+// the given (short) limit, gives up, records wait-site code kSelfTestWaitCode and raises the abort flag; warp 0
+// waits on the same barrier with the full limit and must be released by the flag.  The kernel then returns
+// normally: no trap, no fault, the context stays usable.
+constexpr uint32_t kSelfTestWaitCode = 0x7e;
+__global__ void wait_timeout_selftest_kernel(long long limit_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ volatile uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x >= 32) mbar_wait_warp(&bar, 0, &abort_flag, kSelfTestWaitCode, limit_cycles);
+    else mbar_wait_warp(&bar, 0, &abort_flag, kSelfTestWaitCode + 1);
+    __syncthreads();
 }
 
 // ---------------------------------------------------------------- proxies and fences

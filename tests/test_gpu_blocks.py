@@ -1,4 +1,4 @@
-"""GPU parity of block-sparse attention (Section 4.6): the kernels walk index lists of active 128 x 128
+"""GPU parity of block-sparse attention (Section 4.3): the kernels walk index lists of active 128 x 128
 blocks; the oracle applies the same block matrix on top of the element mask."""
 import numpy as np
 import pytest
@@ -87,10 +87,10 @@ def test_block_sparse_row_pairs_of_one_head():
 
 
 @pytest.mark.parametrize("w,pattern", [FWD_CASES[4], FWD_CASES[5]], ids=lambda x: x.name if hasattr(x, "name") else "")
-def test_block_sparse_forward_one_row_block_per_cta(w, pattern, monkeypatch):
+def test_block_sparse_forward_one_row_block_per_cta(w, pattern):
     """The same odd-group cases without the pair lists (one query tile per CTA)."""
-    monkeypatch.setenv("AF_BS_ROWPAIR", "0")
-    run_fwd(w, pattern((w.S + 127) // 128))
+    with af.option(af.OPT_BS_ROWPAIR, 0):
+        run_fwd(w, pattern((w.S + 127) // 128))
 
 
 def test_block_sparse_all_active_equals_the_dense_kernel():

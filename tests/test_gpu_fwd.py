@@ -34,7 +34,7 @@ SMALL = [
 ]
 
 
-def run_case(w, out_dtype=torch.bfloat16, nq=None, monkeypatch=None, lse_tol=pu.LSE_TOL):
+def run_case(w, out_dtype=torch.bfloat16, lse_tol=pu.LSE_TOL):
     t = synth.draw_all(w)
     dev = {k: pu.to_dev(v) for k, v in t.items()}
     # poison outputs: a kernel that skips rows leaves NaNs behind
@@ -59,19 +59,27 @@ def test_forward_small(w):
 
 @pytest.mark.parametrize("w", [SMALL[i] for i in (2, 3, 4, 5, 6, 7, 9, 10, 11, 12, 14, 16, 17)] + [synth.CONFIGS[1]],
                          ids=lambda w: w.name)
-def test_forward_keys_rotated_in_packed_bf16(w, monkeypatch):
+def test_forward_keys_rotated_in_packed_bf16(w):
     """Optional forward mode: key tiles rotated in packed bf16 arithmetic from TMA-fed tiles of the table's bf16
     copy.  The outputs are held to the same bounds; L gets the output bound, because a row with a single kept
     key has L equal to its one scaled score, which here carries about three bf16 roundings per key element
     (1.1e-2 was measured on such rows at D = 64)."""
-    monkeypatch.setenv("AF_FWD_KEYS_BF16", "1")
-    run_case(w, lse_tol=2e-2)
+    with af.option(af.OPT_FWD_KEYS_BF16, 1):
+        run_case(w, lse_tol=2e-2)
 
 
 @pytest.mark.parametrize("w", SMALL[3:8], ids=lambda w: w.name)
-def test_forward_small_one_query_tile_per_cta(w, monkeypatch):
-    monkeypatch.setenv("AF_FWD_NQ", "1")
-    run_case(w)
+def test_forward_small_one_query_tile_per_cta(w):
+    with af.option(af.OPT_FWD_QTILES, 1):
+        run_case(w)
+
+
+@pytest.mark.parametrize("w", [SMALL[i] for i in (1, 3, 4, 6, 9, 12)], ids=lambda w: w.name)
+def test_forward_small_row_block_pairs(w):
+    """Even GQA groups with head pairing switched off: the two query tiles of a work item are consecutive row
+    blocks of one head, with different key ranges."""
+    with af.option(af.OPT_FWD_PAIR_HEADS, 0):
+        run_case(w)
 
 
 @pytest.mark.parametrize("w", [SMALL[i] for i in (1, 3, 4, 6, 7, 9, 12, 14, 15, 17)] + [synth.CONFIGS[1]],
@@ -247,19 +255,17 @@ def test_config1_tiny_and_config2_full():
         run_case(w)
 
 
-def test_config3_composed_variant_sampled_heads():
-    """Config 3 at full size (window 1024 + ALiBi): all rows of sampled heads (steepest and flattest slope)."""
+def test_config3_composed_variant_full():
+    """Config 3 at full size (window 1024 + ALiBi): every row of every head against the oracle."""
     w = synth.CONFIGS[2]
     t = synth.draw_all(w)
     dev = {k: pu.to_dev(v) for k, v in t.items()}
     o, lse = pu.gpu_fwd(w, dev)
-    sl = w.alibi_slopes()
-    for b, h in ((0, 0), (1, 7), (1, 15)):
-        sub = {k: v[b:b + 1, h:h + 1] for k, v in t.items()}
-        want_o, want_l = oracle.fwd(sub["q"], sub["k"], sub["v"], theta=w.theta, rotary_dim=w.R, window=w.window,
-                                    slopes=sl[h:h + 1], scale=w.scale)
-        pu.assert_close("c3 O head %d" % h, pu.to_np(o[b:b + 1, h:h + 1]), want_o)
-        assert np.abs(pu.to_np(lse[b:b + 1, h:h + 1]) - want_l).max() <= pu.LSE_TOL
+    want_o, want_l = oracle.run_workload(w, t)
+    got_o, got_l = pu.to_np(o), pu.to_np(lse)
+    for h in range(w.Hq):   # per head, so that a failure names the slope it belongs to
+        pu.assert_close("c3 O head %d" % h, got_o[:, h], want_o[:, h])
+    assert np.abs(got_l - want_l).max() <= pu.LSE_TOL
 
 
 def test_config4_long_context_sampled_rows():
@@ -289,12 +295,12 @@ PAIR_CASES = [
 
 
 @pytest.mark.parametrize("w", PAIR_CASES, ids=lambda w: w.name)
-def test_forward_cta_pair_kernel(w, monkeypatch):
+def test_forward_cta_pair_kernel(w):
     """The CTA-pair variant (two SMs share the K/V tiles of a GQA quad; cta_group::2 MMAs)."""
-    monkeypatch.setenv("AF_FWD_2CTA", "1")
-    run_case(w)
+    with af.option(af.OPT_FWD_CTA_PAIR, 1):
+        run_case(w)
 
 
-def test_forward_cta_pair_kernel_config2(monkeypatch):
-    monkeypatch.setenv("AF_FWD_2CTA", "1")
-    run_case(synth.CONFIGS[1])
+def test_forward_cta_pair_kernel_config2():
+    with af.option(af.OPT_FWD_CTA_PAIR, 1):
+        run_case(synth.CONFIGS[1])

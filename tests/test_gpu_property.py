@@ -1,0 +1,127 @@
+"""Property-based parity (Section 6.6 of the paper checks its kernels with generated examples across forward and
+backward): shapes, GQA groups, rotary widths, position offsets, masks, ALiBi, block lists and workspace sizes are
+drawn by hypothesis from a fixed (derandomised) stream, and every example is compared element by element with
+the fp64 oracle on the same seeded inputs, at the tolerances of the other parity tests.
+
+The kernels branch on many of these parameters - ragged last tiles, head pairs on even groups and row pairs on
+odd ones, the rotary widths with a fast path against the generic one, window edges that fall on tile borders,
+three workspace set-ups of the backward - and the hand-picked cases elsewhere cannot cover their product."""
+import numpy as np
+import pytest
+import torch
+from hypothesis import HealthCheck, given, settings, strategies as st
+
+import oracle
+import paper_2609_13612_b200 as af
+from paper_2609_13612_b200 import synth
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+COMMON = dict(derandomize=True, deadline=None, database=None,
+              suppress_health_check=[HealthCheck.too_slow, HealthCheck.data_too_large])
+
+
+@st.composite
+def workloads(draw, backward):
+    D = draw(st.sampled_from([64, 128]))
+    g = draw(st.sampled_from([1, 2, 3, 4, 8]))
+    Hkv = draw(st.integers(1, 2))
+    B = draw(st.integers(1, 2))
+    # lengths around tile borders, short ones, and ragged ones up to a few tiles
+    S = draw(st.one_of(st.sampled_from([1, 127, 128, 129, 255, 256, 257, 384, 512, 640]), st.integers(2, 700)))
+    R = draw(st.sampled_from([0, 16, 32, 48, 64, 96, 128]).filter(lambda r: r <= D))
+    causal = draw(st.booleans())
+    window = draw(st.one_of(st.just(-1), st.sampled_from([0, 1, 127, 128, 129, 256]), st.integers(0, 700)))
+    alibi = draw(st.booleans())
+    p0 = draw(st.sampled_from([0, 0, 1, 1000, 32768 - 700]))
+    theta = draw(st.sampled_from([1.0e4, 5.0e5]))
+    sigma = draw(st.sampled_from([0.5, 1.0]))
+    seed = draw(st.integers(1000, 1 << 20))
+    return synth.Workload("hyp", B, Hkv * g, Hkv, S, D, theta=theta, rotary_dim=R, pos_offset=p0, causal=causal,
+                          window=window, alibi=alibi, sigma=sigma, seed_id=seed, backward=backward)
+
+
+@settings(max_examples=50, **COMMON)
+@given(w=workloads(backward=False), f32_out=st.booleans(), hybrid=st.booleans())
+def test_forward_examples(w, f32_out, hybrid):
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S) if w.R > 0 else None
+    call = af.fwd_hybrid if hybrid else af.fwd
+    o, lse = call(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale,
+                  out_dtype=torch.float32 if f32_out else torch.bfloat16)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    want_o, want_l = oracle.run_workload(w, t)
+    pu.assert_close("%r O" % (w,), pu.to_np(o), want_o)
+    assert np.abs(pu.to_np(lse) - want_l).max() <= pu.LSE_TOL, w
+
+
+@settings(max_examples=30, **COMMON)
+@given(w=workloads(backward=True), tier=st.integers(0, 2), dq_f32=st.booleans())
+def test_backward_examples(w, tier, dq_f32):
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S) if w.R > 0 else None
+    o, lse = af.fwd(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale)
+    # workspace set-ups: delta alone / + rotated-K cache / + rotated-Q cache as well
+    n_delta = (w.B * w.Hq * w.S * 4 + 255) // 256 * 256
+    n_k = w.B * w.Hkv * w.S * w.D * 2
+    n_q = w.B * w.Hq * w.S * w.D * 2
+    ws = torch.empty(n_delta + (n_k if tier >= 1 else 0) + (n_q if tier >= 2 else 0), dtype=torch.uint8, device="cuda")
+    dq, dk, dv = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale,
+                        dq_dtype=torch.float32 if dq_f32 else torch.bfloat16, dkv_dtype=torch.float32, workspace=ws)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    wq, wk, wv = oracle.run_workload(w, t, backward=True)
+    pu.assert_close("%r dQ" % (w,), pu.to_np(dq), wq)
+    pu.assert_close("%r dK" % (w,), pu.to_np(dk), wk)
+    pu.assert_close("%r dV" % (w,), pu.to_np(dv), wv)
+
+
+@st.composite
+def block_patterns(draw, nb):
+    """A random set of active 128 x 128 blocks, sometimes with empty row blocks."""
+    density = draw(st.sampled_from([0.15, 0.4, 0.8]))
+    bits = draw(st.lists(st.floats(0, 1), min_size=nb * nb, max_size=nb * nb))
+    a = (np.array(bits).reshape(nb, nb) < density)
+    if draw(st.booleans()):
+        a |= np.eye(nb, dtype=bool)        # keep the diagonal: no empty rows under a causal mask
+    return a
+
+
+@settings(max_examples=20, **COMMON)
+@given(data=st.data())
+def test_block_sparse_examples(data):
+    D = data.draw(st.sampled_from([64, 128]))
+    g = data.draw(st.sampled_from([1, 2, 3, 4]))
+    S = data.draw(st.sampled_from([128, 200, 384, 515, 640]))
+    causal = data.draw(st.booleans())
+    R = data.draw(st.sampled_from([0, 32, 64]))
+    seed = data.draw(st.integers(2000, 1 << 20))
+    nb = (S + 127) // 128
+    active = data.draw(block_patterns(nb))
+    w = synth.Workload("hypbs", 1, 2 * g, 2, S, D, theta=1.0e4, rotary_dim=R, causal=causal, seed_id=seed, backward=True)
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S) if w.R > 0 else None
+    bm = af.BlockMask(active)
+    o, lse = af.fwd_blocks(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale, bm)
+    dq, dk, dv = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale, blocks=bm)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    kw = dict(theta=w.theta, rotary_dim=w.R, pos_offset=0, causal=causal, window=-1, slopes=None, scale=w.scale)
+    want_o, want_l = oracle.fwd(t["q"], t["k"], t["v"], blocks=active, block_size=128, **kw)
+    pu.assert_close("bs O", pu.to_np(o), want_o)
+    got_l = pu.to_np(lse)
+    fin = np.isfinite(want_l)
+    assert np.array_equal(np.isneginf(got_l), np.isneginf(want_l))
+    assert np.abs(got_l[fin] - want_l[fin]).max(initial=0.0) <= pu.LSE_TOL
+    wq, wk, wv = oracle.bwd(t["q"], t["k"], t["v"], t["do"], blocks=active, block_size=128, **kw)
+    pu.assert_close("bs dQ", pu.to_np(dq), wq)
+    pu.assert_close("bs dK", pu.to_np(dk), wk)
+    pu.assert_close("bs dV", pu.to_np(dv), wv)

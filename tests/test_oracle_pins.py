@@ -313,7 +313,7 @@ def test_backward_structural_properties():
     assert not np.allclose(dk3, dk, atol=1e-6)
 
 
-# ---------------------------------------------------------------- block-sparse attention (Section 4.6)
+# ---------------------------------------------------------------- block-sparse attention (Section 4.3)
 
 def test_blocks_all_active_is_the_dense_result():
     q, k, v, do = rnd((1, 4, 24, 8), 60), rnd((1, 2, 24, 8), 61), rnd((1, 2, 24, 8), 62), rnd((1, 4, 24, 8), 63)
