@@ -363,3 +363,126 @@ def test_blocks_brute_force_and_autograd_tiny():
     assert np.allclose(dq, tq.grad.numpy(), atol=1e-11) and np.allclose(dk, tk.grad.numpy(), atol=1e-11)
     assert np.allclose(dv, tv.grad.numpy(), atol=1e-11)
     assert np.all(dq[:, :, 3:6] == 0.0)
+
+
+# ---------------------------------------------------------------- additive_bias, relu_attention, full (Section 3.1)
+
+def _naive(q, k, v, keep, bias, scale, relu):
+    """Explicit torch graph in fp64: scores, bias, mask, normaliser, P V (GQA by repeat_interleave)."""
+    g = q.shape[1] // k.shape[1]
+    s = scale * q @ k.repeat_interleave(g, dim=1).transpose(-1, -2)
+    if bias is not None:
+        s = s + bias
+    if relu:
+        n = keep.sum(-1, keepdim=True).clamp(min=1)
+        p = torch.where(keep, torch.relu(s), torch.zeros_like(s)) / n
+    else:
+        p = torch.nan_to_num(torch.softmax(s.masked_fill(~keep, float("-inf")), -1), nan=0.0)
+    return p @ v.repeat_interleave(g, dim=1)
+
+
+def test_bias_filled_with_the_alibi_term_is_alibi():
+    """additive_bias carrying slope_h * (j - i) gives what the ALiBi combinator gives, forward and backward."""
+    S, D = 20, 8
+    q, k, v, do = rnd((2, 4, S, D), 80), rnd((2, 2, S, D), 81), rnd((2, 2, S, D), 82), rnd((2, 4, S, D), 83)
+    slopes = np.array([0.5, 0.25, 0.125, 0.0625])
+    ji = (np.arange(S)[None, :] - np.arange(S)[:, None]).astype(np.float64)
+    bias = slopes[None, :, None, None] * ji[None, None]
+    kw = dict(theta=100.0, rotary_dim=8, pos_offset=2, causal=True, window=11, scale=0.3)
+    a, b = oracle.fwd(q, k, v, slopes=slopes, **kw), oracle.fwd(q, k, v, bias=bias, **kw)
+    assert np.allclose(a[0], b[0], atol=1e-13) and np.allclose(a[1], b[1], atol=1e-13)
+    ga, gb = oracle.bwd(q, k, v, do, slopes=slopes, **kw), oracle.bwd(q, k, v, do, bias=bias, **kw)
+    assert all(np.allclose(x, y, atol=1e-12) for x, y in zip(ga, gb))
+    # a sign or transposition slip in the bias index would show: the transposed bias is a different result
+    c = oracle.fwd(q, k, v, bias=np.swapaxes(bias, 2, 3), **kw)
+    assert not np.allclose(a[0], c[0], atol=1e-6)
+
+
+def test_bias_of_minus_infinity_is_a_mask_and_broadcasts():
+    S, D = 14, 4
+    q, k, v, do = rnd((2, 2, S, D), 84), rnd((2, 2, S, D), 85), rnd((2, 2, S, D), 86), rnd((2, 2, S, D), 87)
+    causal_bias = np.where(np.arange(S)[None, :] <= np.arange(S)[:, None], 0.0, -np.inf)[None, None]
+    kw = dict(rotary_dim=4, theta=50.0, scale=0.5)
+    a = oracle.fwd(q, k, v, causal=True, **kw)
+    b = oracle.fwd(q, k, v, causal=False, bias=causal_bias, **kw)                      # [1, 1, S, S] broadcast
+    c = oracle.fwd(q, k, v, causal=False, bias=np.broadcast_to(causal_bias, (2, 2, S, S)).copy(), **kw)
+    assert np.allclose(a[0], b[0], atol=1e-13) and np.allclose(a[1], b[1], atol=1e-13)
+    assert np.array_equal(b[0], c[0]) and np.array_equal(b[1], c[1])
+    ga = oracle.bwd(q, k, v, do, causal=True, **kw)
+    gb = oracle.bwd(q, k, v, do, causal=False, bias=causal_bias, **kw)
+    assert all(np.allclose(x, y, atol=1e-12) for x, y in zip(ga, gb))
+    # `full` (no mask at all) is causal=False without a window: every pair kept
+    full = oracle.fwd(q, k, v, causal=False, window=-1, **kw)
+    assert not np.allclose(full[0], a[0], atol=1e-6)
+
+
+def test_bias_per_batch_and_head_against_autograd():
+    S, D, Hq, Hkv = 11, 4, 4, 2
+    q, k, v, do = rnd((2, Hq, S, D), 88), rnd((2, Hkv, S, D), 89), rnd((2, Hkv, S, D), 90), rnd((2, Hq, S, D), 91)
+    bias = rnd((2, Hq, S, S), 92)
+    keep = torch.from_numpy(np.arange(S)[None, :] <= np.arange(S)[:, None])
+    tq, tk, tv = (torch.from_numpy(x).requires_grad_(True) for x in (q, k, v))
+    out = _naive(tq, tk, tv, keep, torch.from_numpy(bias), 0.7, relu=False)
+    out.backward(torch.from_numpy(do))
+    o, _ = oracle.fwd(q, k, v, rotary_dim=0, causal=True, scale=0.7, bias=bias)
+    assert np.allclose(o, out.detach().numpy(), atol=1e-12)
+    dq, dk, dv = oracle.bwd(q, k, v, do, rotary_dim=0, causal=True, scale=0.7, bias=bias)
+    assert np.allclose(dq, tq.grad.numpy(), atol=1e-11) and np.allclose(dk, tk.grad.numpy(), atol=1e-11)
+    assert np.allclose(dv, tv.grad.numpy(), atol=1e-11)
+    # the head extent of the bias follows the QUERY head: permuting heads of q and bias together permutes O
+    perm = [1, 0, 3, 2]
+    o2, _ = oracle.fwd(q[:, perm], k, v, rotary_dim=0, causal=True, scale=0.7, bias=bias[:, perm])
+    assert np.allclose(o2, o[:, perm], atol=1e-13)
+
+
+def test_relu_attention_closed_forms_fix_the_normalisation():
+    """With Q = 0 every score equals its bias.  A constant bias c > 0 gives O_i = c * mean of the kept values
+    (relu(c) / n_i each): with the row's kept count n_i, not the sequence length, under a mask.  A negative
+    constant gives O = 0."""
+    S, D = 9, 3
+    k, v = rnd((1, 1, S, D), 93), rnd((1, 1, S, D), 94)
+    q = np.zeros((1, 2, S, D))
+    c = 1.75
+    o, l = oracle.fwd(q, k, v, rotary_dim=0, causal=True, scale=1.0, bias=np.full((1, 1, S, S), c), normaliser="relu")
+    assert l is None
+    for i in range(S):
+        assert np.allclose(o[0, :, i], c * v[0, 0, :i + 1].mean(0), atol=1e-13)
+    o, _ = oracle.fwd(q, k, v, rotary_dim=0, causal=True, window=2, scale=1.0, bias=np.full((1, 1, S, S), c), normaliser="relu")
+    for i in range(S):
+        assert np.allclose(o[0, :, i], c * v[0, 0, max(0, i - 2):i + 1].mean(0), atol=1e-13)
+    o, _ = oracle.fwd(q, k, v, rotary_dim=0, causal=False, scale=1.0, bias=np.full((1, 1, S, S), c), normaliser="relu")
+    assert np.allclose(o[0, 0], np.broadcast_to(c * v[0, 0].mean(0), (S, D)), atol=1e-13)   # full: n_i = S
+    o, _ = oracle.fwd(q, k, v, rotary_dim=0, causal=True, scale=1.0, bias=np.full((1, 1, S, S), -c), normaliser="relu")
+    assert not o.any()
+
+
+def test_relu_attention_against_autograd_and_finite_differences():
+    S, D, Hq, Hkv = 10, 4, 4, 2
+    q, k, v, do = rnd((2, Hq, S, D), 95), rnd((2, Hkv, S, D), 96), rnd((2, Hkv, S, D), 97), rnd((2, Hq, S, D), 98)
+    bias = 0.3 * rnd((1, Hq, S, S), 99)
+    keep_np = (np.arange(S)[None, :] <= np.arange(S)[:, None]) & (np.arange(S)[:, None] - np.arange(S)[None, :] <= 6)
+    tq, tk, tv = (torch.from_numpy(x).requires_grad_(True) for x in (q, k, v))
+    out = _naive(tq, tk, tv, torch.from_numpy(keep_np), torch.from_numpy(bias), 0.6, relu=True)
+    out.backward(torch.from_numpy(do))
+    kw = dict(rotary_dim=0, causal=True, window=6, scale=0.6, bias=bias, normaliser="relu")
+    o, _ = oracle.fwd(q, k, v, **kw)
+    assert np.allclose(o, out.detach().numpy(), atol=1e-12)
+    dq, dk, dv = oracle.bwd(q, k, v, do, **kw)
+    assert np.allclose(dq, tq.grad.numpy(), atol=1e-11) and np.allclose(dk, tk.grad.numpy(), atol=1e-11)
+    assert np.allclose(dv, tv.grad.numpy(), atol=1e-11)
+    # with RoPE in front: central differences of sum(O * dO) (the kinks of relu have measure zero)
+    kw = dict(theta=30.0, rotary_dim=4, pos_offset=1, causal=True, scale=0.6, normaliser="relu")
+    dq, dk, dv = oracle.bwd(q, k, v, do, **kw)
+    f = lambda a, b, c: float((oracle.fwd(a, b, c, **kw)[0] * do).sum())
+    h = 1e-6
+    r = np.random.default_rng(5)
+    for (name, x, gx) in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        for _ in range(6):
+            idx = tuple(r.integers(0, n) for n in x.shape)
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += h
+            xm[idx] -= h
+            args_p = {"q": (xp, k, v), "k": (q, xp, v), "v": (q, k, xp)}[name]
+            args_m = {"q": (xm, k, v), "k": (q, xm, v), "v": (q, k, xm)}[name]
+            num = (f(*args_p) - f(*args_m)) / (2 * h)
+            assert abs(num - gx[idx]) <= 1e-6 * max(1.0, abs(num)), (name, idx, num, gx[idx])
