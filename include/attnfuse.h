@@ -185,6 +185,40 @@ af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* 
                               int gqa_group, float softmax_scale, const af_blocks* blocks,
                               void* o, af_dtype o_dtype, float* lse, void* cuda_stream);
 
+/* ---- composed variants (Section 3.1: the ten combinators) ---------------------------------------------
+ * One description of a variant and one forward entry point for it, the counterpart of a program composed
+ * from the paper's combinators (Section 3.1) and run through its single run-time entry (Section 3.3):
+ *   scaled_dot_product  -> softmax_scale        rope            -> rope + rope_table
+ *   causal              -> mask.causal          sliding_window  -> mask.window
+ *   full                -> mask.causal = 0 and mask.window < 0 (nothing masked)
+ *   block_sparse        -> blocks               alibi           -> mask.alibi_slopes
+ *   additive_bias       -> bias                 softmax / relu_attention -> normaliser
+ * additive_bias: a dense fp32 tensor bias[bb, hh, i, j] (DEVICE, contiguous [bias_B, bias_H, S, S], 4-byte
+ * aligned; extents 1 = broadcast, else B resp. Hq), added to the scaled score after the softmax scale, like
+ * the ALiBi term.  A bias of -inf drops the pair like a mask.  NULL: none.  The kernel reads it with plain
+ * loads, one row of 128 values per thread and key tile (16-byte loads when S is a multiple of 4): the
+ * variant is bound by the S x S bias traffic, not by the tensor pipe.
+ * relu_attention (the paper names the combinator only; reading): P_ij = max(s_ij, 0) / n_i over the kept
+ * pairs, n_i = number of kept pairs of row i (pairs that the mask keeps and whose bias is finite), in place
+ * of the softmax; there is no row statistic, so lse must be NULL; not available over block lists.
+ * Forward only: attnfuse_bwd covers rope, causal, sliding_window, full, block_sparse, alibi and softmax.
+ * Errors as for attnfuse_fwd; AF_ERR_SHAPE for bias extents other than 1 / B / Hq, AF_ERR_SPEC for an
+ * unknown normaliser, for lse with relu_attention, and for relu_attention with blocks. */
+typedef enum { AF_NORM_SOFTMAX = 0, AF_NORM_RELU = 1 } af_normaliser;
+typedef struct {
+    af_rope rope;
+    const void* rope_table;      /* from attnfuse_rope_table; may be NULL iff rope.rotary_dim = 0 */
+    af_mask mask;
+    const float* bias;           /* additive_bias or NULL */
+    int bias_B, bias_H;          /* its batch and head extents: 1 or B, 1 or Hq */
+    af_normaliser normaliser;
+    const af_blocks* blocks;     /* block_sparse lists or NULL (dense) */
+} af_variant;
+af_status attnfuse_fwd_variant(const af_shape* shape, const void* q, const void* k, const void* v,
+                               const af_strides* sq, const af_strides* skv, const af_variant* variant,
+                               int gqa_group, float softmax_scale,
+                               void* o, af_dtype o_dtype, float* lse, void* cuda_stream);
+
 /* Same computation with HOST buffers: q, k, v, o (bf16) and lse (nullable) are host pointers
  * (pinned memory: with pageable memory the copies are not asynchronous).  `staging` is a DEVICE buffer
  * of at least attnfuse_fwd_host_staging_bytes() bytes, caller-owned.  The work is cut into chunks of

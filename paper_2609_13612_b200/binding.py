@@ -36,12 +36,21 @@ class _Blocks(ctypes.Structure):
                 ("pair_order", ctypes.c_void_p)]
 
 
+class _Variant(ctypes.Structure):
+    pass
+
+
 class _Rope(ctypes.Structure):
     _fields_ = [("theta", ctypes.c_float), ("rotary_dim", ctypes.c_int), ("pos_offset", ctypes.c_int)]
 
 
 class _Mask(ctypes.Structure):
     _fields_ = [("causal", ctypes.c_int), ("window", ctypes.c_int), ("alibi_slopes", ctypes.c_void_p)]
+
+
+_Variant._fields_ = [("rope", _Rope), ("rope_table", ctypes.c_void_p), ("mask", _Mask), ("bias", ctypes.c_void_p),
+                     ("bias_B", ctypes.c_int), ("bias_H", ctypes.c_int), ("normaliser", ctypes.c_int),
+                     ("blocks", ctypes.POINTER(_Blocks))]
 
 
 @dataclasses.dataclass(frozen=True)
@@ -92,6 +101,8 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_fwd.restype = i
         L.attnfuse_fwd.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp, P(_Mask), i, f,
                                    vp, i, vp, vp]
+        L.attnfuse_fwd_variant.restype = i
+        L.attnfuse_fwd_variant.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Strides), P(_Variant), i, f, vp, i, vp, vp]
         L.attnfuse_fwd_hybrid_workspace_bytes.restype = sz
         L.attnfuse_fwd_hybrid_workspace_bytes.argtypes = [P(_Shape)]
         L.attnfuse_fwd_hybrid.restype = i
@@ -255,6 +266,39 @@ def fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, 
                               ctypes.byref(m), Hq // Hkv, float(softmax_scale), out.data_ptr(),
                               AF_F32 if out.dtype == torch.float32 else AF_BF16,
                               lse.data_ptr() if lse is not None else None, _stream()))
+    return out, lse
+
+
+def fwd_variant(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor],
+                mask: MaskSpec, softmax_scale: float, bias: Optional[torch.Tensor] = None, normaliser: str = "softmax",
+                blocks: Optional["BlockMask"] = None, out: Optional[torch.Tensor] = None,
+                out_dtype: torch.dtype = torch.bfloat16):
+    """Forward of a composed variant (Section 3.1): `fwd` plus an optional additive bias (fp32 [1|B, 1|Hq, S, S]
+    on the device), the normaliser ("softmax" or "relu") and optional block lists.  Returns (o, lse); lse is
+    None for the ReLU normaliser."""
+    _need_cuda(q, k, v, table, out, bias)
+    assert q.dtype == k.dtype == v.dtype == torch.bfloat16 and normaliser in ("softmax", "relu")
+    B, Hq, S, D = q.shape
+    Hkv = k.shape[1]
+    assert k.shape == v.shape == (B, Hkv, S, D) and k.stride() == v.stride()
+    if out is None:
+        out = torch.empty((B, Hq, S, D), dtype=out_dtype, device=q.device)
+    relu = normaliser == "relu"
+    lse = None if relu else torch.empty((B, Hq, S), dtype=torch.float32, device=q.device)
+    if bias is not None:
+        assert bias.dtype == torch.float32 and bias.is_contiguous() and bias.dim() == 4 and bias.shape[2:] == (S, S)
+    sh = _Shape(B, Hq, Hkv, S, D)
+    sq, skv = _strides(q), _strides(k)
+    bl = blocks.struct() if blocks is not None else None
+    var = _Variant(_Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset),
+                   table.data_ptr() if table is not None else None, _mask_struct(mask),
+                   bias.data_ptr() if bias is not None else None,
+                   bias.shape[0] if bias is not None else 1, bias.shape[1] if bias is not None else 1,
+                   1 if relu else 0, ctypes.pointer(bl) if bl is not None else None)
+    _check(lib().attnfuse_fwd_variant(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), ctypes.byref(sq),
+                                      ctypes.byref(skv), ctypes.byref(var), Hq // Hkv, float(softmax_scale),
+                                      out.data_ptr(), AF_F32 if out.dtype == torch.float32 else AF_BF16,
+                                      lse.data_ptr() if lse is not None else None, _stream()))
     return out, lse
 
 

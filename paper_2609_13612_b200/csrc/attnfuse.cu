@@ -564,13 +564,19 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
                    const af_strides* skv, const af_rope* rope, const void* rope_table, const af_mask* mask,
                    int gqa_group, float softmax_scale, const int* bs_row_ptr, const int* bs_col_idx,
                    const int* bs_order, void* o, af_dtype o_dtype, float* lse, bool k_prerotated, void* cuda_stream,
-                   const af_blocks* blocks = nullptr) {
+                   const af_blocks* blocks = nullptr, const float* bias = nullptr, int bias_B = 1, int bias_H = 1,
+                   int relu = 0) {
     af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
     if (st != AF_OK) return st;
     if (!q || !k || !v || !o) return AF_ERR_NULL;
     if (o_dtype != AF_BF16 && o_dtype != AF_F32) return AF_ERR_DTYPE;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return AF_ERR_ALIGN;
     if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return AF_ERR_SPEC;
+    if (bias) {
+        if ((bias_B != 1 && bias_B != shape->B) || (bias_H != 1 && bias_H != shape->Hq)) return AF_ERR_SHAPE;
+        if ((reinterpret_cast<uintptr_t>(bias) & 3u) != 0) return AF_ERR_ALIGN;
+    }
+    if (relu && (lse || bs_row_ptr)) return AF_ERR_SPEC;   // no row statistic for the ReLU normaliser; not built over block lists
     af_strides stq, stkv;
     if ((st = resolve_strides(sq, shape->Hq, shape->S, shape->D, &stq)) != AF_OK) return st;
     if ((st = resolve_strides(skv, shape->Hkv, shape->S, shape->D, &stkv)) != AF_OK) return st;
@@ -620,6 +626,10 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     }
     p.rot_k = k_prerotated ? 0 : 1;
     p.keys_bf16 = keys_bf16 ? 1 : 0;
+    p.bias = bias;
+    p.bias_sh = (bias && bias_H > 1) ? static_cast<long long>(shape->S) * shape->S : 0;
+    p.bias_sb = (bias && bias_B > 1) ? static_cast<long long>(bias_H) * shape->S * shape->S : 0;
+    p.relu = relu ? 1 : 0;
 #ifdef AF_TRACE
     p.trace = reinterpret_cast<long long*>(getenv("AF_TRACE_PTR") ? strtoull(getenv("AF_TRACE_PTR"), nullptr, 0) : 0ull);
     cudaMemcpyToSymbol(af::g_trace, &p.trace, sizeof(p.trace));
@@ -629,7 +639,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
         return shape->D == 128 ? launch_fwd_blocks<128>(tq, tk, tv, to, tt, p, stream) : launch_fwd_blocks<64>(tq, tk, tv, to, tt, p, stream);
     const int R = rope->rotary_dim;
     const bool pair_ok = shape->D == 128 && (gqa_group % 4) == 0 && (R == 0 || R == 16 || R == 32 || R == 64 || R == 128);
-    if (pair_ok && !k_prerotated && opt(AF_OPT_FWD_CTA_PAIR)) {
+    if (pair_ok && !k_prerotated && !bias && !relu && opt(AF_OPT_FWD_CTA_PAIR)) {
         CUtensorMap tk2;
         if ((st = make_tmap(&tk2, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, 64)) != AF_OK) return st;
         return R > 0 ? launch_fwd2_variant<true>(tq, tk2, tv, p, stream) : launch_fwd2_variant<false>(tq, tk2, tv, p, stream);
@@ -645,6 +655,22 @@ af_status attnfuse_fwd(const af_shape* shape, const void* q, const void* k, cons
                        int gqa_group, float softmax_scale, void* o, af_dtype o_dtype, float* lse, void* cuda_stream) {
     return fwd_impl(shape, q, k, v, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, nullptr, nullptr, nullptr,
                     o, o_dtype, lse, false, cuda_stream);
+}
+
+af_status attnfuse_fwd_variant(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* sq,
+                               const af_strides* skv, const af_variant* variant, int gqa_group, float softmax_scale,
+                               void* o, af_dtype o_dtype, float* lse, void* cuda_stream) {
+    if (!variant) return AF_ERR_NULL;
+    if (variant->normaliser != AF_NORM_SOFTMAX && variant->normaliser != AF_NORM_RELU) return AF_ERR_SPEC;
+    const af_blocks* bl = variant->blocks;
+    if (bl) {
+        if (!bl->row_ptr || !bl->col_idx) return AF_ERR_NULL;
+        if (bl->block != 128) return AF_ERR_SPEC;
+    }
+    return fwd_impl(shape, q, k, v, sq, skv, &variant->rope, variant->rope_table, &variant->mask, gqa_group, softmax_scale,
+                    bl ? bl->row_ptr : nullptr, bl ? bl->col_idx : nullptr, bl ? bl->row_order : nullptr, o, o_dtype, lse,
+                    false, cuda_stream, bl, variant->bias, variant->bias_B, variant->bias_H,
+                    variant->normaliser == AF_NORM_RELU);
 }
 
 size_t attnfuse_fwd_hybrid_workspace_bytes(const af_shape* shape) {

@@ -36,6 +36,11 @@ struct FwdParams {
     int keys_bf16;         // host-side choice of the TAB instantiation (packed-bf16 key rotation)
     int rot_k;             // ROPE kernels: 1 = rotate the key tiles on chip; 0 = the keys arrive rotated (hybrid
                            // arm of Section 5.3: K rotated once by a RoPE pass, only Q rotated in the kernel)
+    // Section 3.1, additive_bias: fp32 bias[bb, hh, i, j] added to the scaled score (nullptr: none); element strides
+    // of its batch and head extents (0 where the extent is 1 and the bias is broadcast), rows of S floats.
+    const float* bias;
+    long long bias_sb, bias_sh;
+    int relu;              // Section 3.1, relu_attention: P = max(s, 0) / (kept pairs of the row) in place of the softmax
 #ifdef AF_TRACE
     long long* trace;
 #endif
@@ -195,6 +200,111 @@ __device__ __forceinline__ bool softmax_tile_halves(uint32_t tS, uint32_t tO, in
     }
     l_run = l_run * alpha + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
     AF_STAMP_SM(6);
+    return true;
+}
+
+// The same step for the variants with an additive bias and / or the ReLU normaliser (Section 3.1: additive_bias,
+// relu_attention): one straight implementation with the mask, ALiBi and the bias decided at run time, so that
+// the variants above stay as they are.  Scores are formed in natural units, s = c S + slope (j - i) + bias_ij,
+// masked pairs and pairs whose bias is -inf drop out.
+//   softmax:  as above (running max and sum in the log2 domain, lazy rescale).
+//   RELU:     P = max(s, 0), unnormalised; l_run counts the kept pairs of the row, and the epilogue's division by
+//             l_run is the normalisation by the number of kept pairs.  m_run is not used.
+// bias_row: this thread's row of the bias at the tile's first column (or nullptr); cols_ok: how many of the 128
+// columns lie inside the sequence (loads stop there); vec: the row is 16-byte aligned.
+template <int D, bool RELU>
+__device__ __forceinline__ bool softmax_tile_general(uint32_t tS, uint32_t tO, int n, float scale_log2, float slope2,
+                                                     int j0_minus_i, int mlo, uint32_t mn, const float* bias_row,
+                                                     int cols_ok, bool vec, uint64_t* s_full, uint64_t* p_ready,
+                                                     uint32_t parity, volatile uint32_t* abort_flag, int lane,
+                                                     float& m_run, float& l_run) {
+    constexpr float kLog2e = 1.4426950408889634f;
+    uint32_t v[BN];
+    if (!mbar_wait_warp(&s_full[0], parity, abort_flag, 10)) return false;
+    tc_fence_after_sync();
+    tmem_ld32(tS, v);
+    tmem_ld32(tS + 32, v + 32);
+    tmem_ld32(tS + 64, v + 64);
+    tmem_ld32(tS + 96, v + 96);
+    tmem_wait_ld();
+    // scores in the log2 domain: t = c2 S + slope2 (j - i) + log2(e) bias
+    float mx = -INFINITY, cnt = 0.f;
+#pragma unroll
+    for (int e4 = 0; e4 < BN; e4 += 4) {
+        float bv[4] = {0.f, 0.f, 0.f, 0.f};
+        if (bias_row) {
+            if (vec && e4 + 4 <= cols_ok) {
+                const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias_row + e4));
+                bv[0] = b4.x; bv[1] = b4.y; bv[2] = b4.z; bv[3] = b4.w;
+            } else {
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (e4 + u < cols_ok) bv[u] = __ldg(bias_row + e4 + u);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int e = e4 + u;
+            float t = fmaf(__uint_as_float(v[e]), scale_log2, slope2 * static_cast<float>(j0_minus_i + e));
+            t = fmaf(bv[u], kLog2e, t);
+            const bool kept = static_cast<uint32_t>(e - mlo) < mn && t > -INFINITY;
+            t = kept ? t : -INFINITY;
+            v[e] = __float_as_uint(t);
+            mx = fmaxf(mx, t);
+            cnt += kept ? 1.f : 0.f;
+        }
+    }
+    float alpha = 1.f;
+    bool upd = false;
+    if (!RELU) {
+        upd = mx > m_run + kRescaleThreshold;
+        if (upd) {
+            alpha = ex2(m_run - mx);
+            m_run = mx;
+        }
+    }
+    const float ref = (m_run == -INFINITY) ? 0.f : m_run;
+    float psum = 0.f;
+    constexpr int CPP = 4 / kPParts;
+#pragma unroll
+    for (int pt = 0; pt < kPParts; ++pt) {
+#pragma unroll
+        for (int c = 0; c < CPP; ++c) {
+            uint32_t pk[16];
+            const int col0 = (pt * CPP + c) * 32;
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+                const float t0 = __uint_as_float(v[col0 + e]), t1 = __uint_as_float(v[col0 + e + 1]);
+                float p0, p1;
+                if (RELU) {   // back to natural units; a dropped pair (-inf) gives 0
+                    p0 = fmaxf(t0 * 0.6931471805599453f, 0.f);
+                    p1 = fmaxf(t1 * 0.6931471805599453f, 0.f);
+                } else {
+                    p0 = ex2(t0 - ref);
+                    p1 = ex2(t1 - ref);
+                    psum += p0 + p1;
+                }
+                pk[e >> 1] = pack_bf16x2(p0, p1);
+            }
+            tmem_st16(tS + pt * (BN / kPParts) + c * 16, pk);
+        }
+        if (!RELU && pt == 0 && n > 0 && __any_sync(0xffffffffu, upd)) {
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tO + c * 32, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                tmem_st32(tO + c * 32, o);
+            }
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_ready[pt]);
+    }
+    l_run = RELU ? l_run + cnt : l_run * alpha + psum;
     return true;
 }
 
@@ -581,7 +691,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (need_mask) kept_keys_of_query(ms, i, j0, mlo, mn);
             uint64_t* sf = &bars[L::B_SFULL + 2 * q];
             uint64_t* pr = &bars[L::B_PREADY + 4 * q];
-            if (alibi) {
+            if (p.bias || p.relu) {
+                // Section 3.1: additive_bias / relu_attention
+                const float* brow = nullptr;
+                if (p.bias && i < p.S)
+                    brow = p.bias + b * p.bias_sb + hq[q] * p.bias_sh + static_cast<long long>(i) * p.S + j0;
+                const int cols_ok = min(BN, p.S - j0);
+                const bool vec = (p.S & 3) == 0 && (reinterpret_cast<uintptr_t>(p.bias) & 15u) == 0 &&
+                                 (((b * p.bias_sb + hq[q] * p.bias_sh) & 3) == 0);
+                if (p.relu) ok = softmax_tile_general<D, true>(tS, tO, n, p.scale_log2, slope2, j0 - i, mlo, mn, brow, cols_ok, vec, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
+                else ok = softmax_tile_general<D, false>(tS, tO, n, p.scale_log2, slope2, j0 - i, mlo, mn, brow, cols_ok, vec, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
+            } else if (alibi) {
                 if (need_mask) ok = softmax_tile_halves<D, true, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
                 else ok = softmax_tile_halves<D, false, true>(tS, tO, n, p.scale_log2, kb, bias0, mlo, mn, sf, pr, n & 1, abort_flag, lane, m_run, l_run);
             } else {
@@ -651,7 +771,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
             }
-            if (p.lse && i < p.S)
+            if (p.lse && !p.relu && i < p.S)
                 p.lse[static_cast<size_t>(bh) * p.S + i] =
                     l_run > 0.f ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
         }

@@ -12,7 +12,13 @@ from paper_2609_13612_b200 import synth
 # Tolerance of the bf16-in / fp32-accumulate path against the fp64 oracle.
 MAX_ABS_TOL = 2e-2
 MEAN_ABS_TOL = 2e-3
-LSE_TOL = 1e-2
+# L = ln sum_j exp(s_ij) moves by at most max_j |ds_ij|, and a score carries the bf16 roundings of the rotated q'
+# and k' (relative 2^-9 each, independent over the D products): ds has a standard deviation of about
+# c * 2^-9 * sqrt(2/3) * |q' * k'|_2, i.e. 1.6e-3 for unit-variance rows at D = 128, c = 1/sqrt(D).  A row that one
+# key dominates (steep ALiBi slopes, the first rows of a causal mask) has L = that score, so over the 2.6e5 rows of
+# the composed-variant configuration the largest deviation sits near six standard deviations, 1e-2 (measured:
+# 1.06e-2).  L is therefore held to the bound of the outputs, 2e-2 (about twelve standard deviations).
+LSE_TOL = 2e-2
 
 
 def to_dev(x: np.ndarray) -> torch.Tensor:
@@ -65,3 +71,20 @@ def assert_close(name, got, want, max_tol=MAX_ABS_TOL, mean_tol=MEAN_ABS_TOL):
     assert mx <= max_tol and mean <= mean_tol, "%s: max abs %.4g (tol %g), mean abs %.4g (tol %g)" % (
         name, mx, max_tol, mean, mean_tol)
     return mx, mean
+
+
+# Generated examples reach corners where a gradient row is a sum of very many same-sized terms (non-causal ALiBi sends
+# every query to the last key, whose dV row then adds up P * dO over all rows and heads of the group and reaches
+# magnitudes of 10 and more).  Each term carries one bf16 rounding (P and dS go to the tensor cores in bf16), so
+# the error of the sum scales with its size: the absolute bound is kept and a relative share of one bf16 ulp
+# (2^-8 of the exact value) is allowed on top.  The fixed configurations are held to the absolute bound alone.
+BF16_ULP = 2.0 ** -8
+
+
+def assert_close_scaled(name, got, want, max_tol=MAX_ABS_TOL, mean_tol=MEAN_ABS_TOL, rel=BF16_ULP):
+    assert np.isfinite(got).all(), "%s has non-finite values" % name
+    d = np.abs(got - want)
+    excess = d - rel * np.abs(want)
+    assert excess.max() <= max_tol and d.mean() <= mean_tol + rel * np.abs(want).mean(), \
+        "%s: max abs %.4g, beyond the relative share %.4g (tol %g), mean abs %.4g (tol %g)" % (
+            name, d.max(), excess.max(), max_tol, d.mean(), mean_tol)
