@@ -36,9 +36,12 @@ from paper_2609_13612_b200 import synth  # noqa: E402
 METRIC = "fused RoPE+causal attention TFLOP/s (bf16 fwd/bwd) and % of B200 tensor peak"
 UNIT = "TFLOP/s"
 L2_BYTES = 126 * 1024 * 1024
-# DRAM bytes per launch of the forward kernel on this workload, from the ncu capture summarised in
-# profiles/attn_fwd_kernel_c2_llama3_8b.md (dram__bytes_read.sum + dram__bytes_write.sum).
-FWD_TRAFFIC_BYTES_PER_LAUNCH = 55.3e6
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture), by kernel and workload.
+# A kernel or workload that has no entry reports "traffic": null instead of a figure that belongs to another one.
+KERNEL_TRAFFIC_BYTES = {
+    ("attn_fwd_kernel<128,2,rope>", "c2_llama3_8b_fwd"): 55.3e6,
+}
+RIDGE_CONTEXT = {"paper_ampere_flop_per_byte": 152, "paper_hopper_flop_per_byte": 300}
 PAPER_CONTEXT = {
     "rtx3090_fused_vs_flex_prerotate_rope_causal": "2.10x (RTX 3090, fp16, B=4 H=12 D=64, N=4096)",
     "h100_llama3_8b_training_step_vs_sdpa": "within ~5% (H100 NVL, fp16, N=2048: 7.65 ms vs 7.27 ms)",
@@ -87,7 +90,11 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            time.sleep(0.002)
+            time.sleep(0.0002)
+
+    def mark(self):
+        """Number of samples taken so far (to tell the samples of the timed region from later ones)."""
+        return len(self.samples)
 
     def __enter__(self):
         if self._nv is not None:
@@ -281,6 +288,19 @@ def main():
 
     with ClockSampler(local) as clk:
         total_ms, per, _ = timed(step, args.steps, args.warmup)
+        n_timed = clk.mark()
+        # A short run (the timed region of 20 steps lasts a few milliseconds) yields only a few NVML samples: the
+        # same step keeps running, untimed, until the sampler has seen the clocks under this load for at least 30 ms.
+        t_end = time.perf_counter() + 0.03
+        i_extra = 0
+        while time.perf_counter() < t_end or clk.mark() < 12:
+            step(i_extra)
+            i_extra += 1
+            if i_extra % 8 == 0:
+                torch.cuda.synchronize()
+            if i_extra > 20000:
+                break
+        torch.cuda.synchronize()
     code, detail = af.device_status()
     if code != 0:
         raise SystemExit("device-side wait ran out (0x%x): numbers invalid" % detail)
@@ -292,7 +312,7 @@ def main():
     roofline = {"bound": "tensor", "kernel": "attn_fwd_kernel<128,2,rope>", "achieved": achieved,
                 "peak": peaks["bf16_tflops"], "peak_kind": "burst bf16 dense, %s" % peaks["source"], "unit": UNIT,
                 "frac": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
-                "traffic": FWD_TRAFFIC_BYTES_PER_LAUNCH, "kernel_ms": kern_ms,
+                "traffic": KERNEL_TRAFFIC_BYTES.get(("attn_fwd_kernel<128,2,rope>", w.name)), "kernel_ms": kern_ms,
                 "algorithmic_flops_per_launch": flops}
 
     # ------------------------------------------------------------------ e2e: host buffers through the C-ABI
@@ -319,7 +339,8 @@ def main():
                    "l2": "inputs rotate over %d independent sets (%.0f MB total > 126 MB L2)" % (
                        len(sets), len(sets) * input_bytes(w) / 1e6),
                    "sharding": "replicated per-GPU workload, no collective" if world > 1 else "single GPU"},
-        "clocks": clk.summary(),
+        "clocks": dict(clk.summary(), samples_in_timed_region=n_timed,
+                       note="sampled over warm-up, timed region and the same step continued untimed for 30 ms"),
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": args.steps,
@@ -465,8 +486,7 @@ def main():
             ld = torch.empty(1, Hq_, device=dev, dtype=torch.float32)
             shp = binding._Shape(1, Hq_, Hkv_, N_, 128)
             nsp = af.lib().attnfuse_decode_splits(__import__("ctypes").byref(shp))
-            wsd = torch.empty(af.lib().attnfuse_decode_workspace_bytes(__import__("ctypes").byref(shp), nsp),
-                              dtype=torch.uint8, device=dev)
+            wsd = af.decode_workspace(1, Hq_, Hkv_, N_, 128, nsp, device=dev)
             call = lambda i: af.decode(qd, kcs[i % nsets], vcs[i % nsets], md, 128 ** -0.5, n_splits=nsp, out=od, lse=ld,
                                        workspace=wsd)
             t_host, _, _ = timed(call, 2 * k_ex, w_ex)
@@ -529,19 +549,63 @@ def main():
                                            "fwd_ms": t_bf2 / k_ex, "speedup_over_dense": t_df / t_bf2}
         del sb
         torch.cuda.empty_cache()
-        # Rotation Calculus sweep (Section 5.3): fused vs separate RoPE at constant B*S = 32768 tokens
-        sweep = []
-        for S in (512, 1024, 2048, 4096, 8192, 16384, 32768):
-            wl = synth.Workload("sweep_S%d" % S, 32768 // S, 32, 8, S, 128, theta=5.0e5, seed_id=50)
-            ms_f, ss = fwd_ms(wl, True)
-            ms_s, _ = fwd_ms(wl, False, ss)
-            ms_h, _ = fwd_ms(wl, True, ss, hybrid=True)
-            sweep.append({"S": S, "B": wl.B, "fused_ms": ms_f, "separate_ms": ms_s, "hybrid_ms": ms_h,
-                          "speedup_fused": ms_s / ms_f, "speedup_hybrid_over_fused": ms_f / ms_h,
-                          "fused_tflops": wl.fwd_flops() / ms_f / 1e9, "hybrid_tflops": wl.fwd_flops() / ms_h / 1e9})
-            del ss
-            torch.cuda.empty_cache()
-        ex["rotation_calculus_sweep"] = sweep
+        # Rotation Calculus sweep (Section 5.3): fused vs separate RoPE at constant B*S = 32768 tokens, with the
+        # hybrid arm and the same kernel without RoPE as the floor, in the Llama geometry (32 q / 8 kv heads, D = 128)
+        # and in the geometry of the paper's own table (12 heads, D = 64).
+        def plain_ms(wl, sets_):
+            r, m, tb = specs(wl)
+            oo = torch.empty((wl.B, wl.Hq, wl.S, wl.D), dtype=torch.bfloat16, device=dev)
+            ll = torch.empty((wl.B, wl.Hq, wl.S), dtype=torch.float32, device=dev)
+            norope = af.RopeSpec()
+            t, _, _ = timed(lambda i: af.fwd(sets_[i % len(sets_)]["q"], sets_[i % len(sets_)]["k"], sets_[i % len(sets_)]["v"],
+                                             norope, None, m, wl.scale, out=oo, lse=ll), k_ex, w_ex)
+            return t / k_ex
+
+        def crossover(rows):
+            """S at which fused / separate crosses 1 (log-linear interpolation between neighbouring lengths)."""
+            for a, b_ in zip(rows, rows[1:]):
+                fa, fb_ = a["speedup_fused"] - 1.0, b_["speedup_fused"] - 1.0
+                if fa == 0.0:
+                    return float(a["S"])
+                if fa * fb_ < 0:
+                    x = fa / (fa - fb_)
+                    return float(math.exp(math.log(a["S"]) + x * (math.log(b_["S"]) - math.log(a["S"]))))
+            return None
+
+        def sweep_geometry(Hq_, Hkv_, D_, theta_, tokens, lengths):
+            rows = []
+            for S in lengths:
+                wl = synth.Workload("sweep_S%d" % S, tokens // S, Hq_, Hkv_, S, D_, theta=theta_, seed_id=50)
+                ms_f, ss = fwd_ms(wl, True)
+                ms_s, _ = fwd_ms(wl, False, ss)
+                ms_h, _ = fwd_ms(wl, True, ss, hybrid=True)
+                ms_p = plain_ms(wl, ss)
+                # K-tile rotations the fused kernel performs: one per key tile and CTA (a CTA holds two query tiles:
+                # two heads of a kv group when the group is even, else two consecutive row blocks of a head)
+                n = (S + 127) // 128
+                pair = (Hq_ // Hkv_) % 2 == 0
+                rot = wl.B * (Hq_ // 2) * n * (n + 1) // 2 if pair else wl.B * Hq_ * sum(min(2 * r + 2, n) for r in range((n + 1) // 2))
+                rows.append({"S": S, "B": wl.B, "fused_ms": ms_f, "separate_ms": ms_s, "hybrid_ms": ms_h, "no_rope_ms": ms_p,
+                             "speedup_fused": ms_s / ms_f, "speedup_hybrid_over_fused": ms_f / ms_h,
+                             "fused_tflops": wl.fwd_flops() / ms_f / 1e9, "hybrid_tflops": wl.fwd_flops() / ms_h / 1e9,
+                             "no_rope_tflops": wl.fwd_flops() / ms_p / 1e9, "key_tile_rotations": rot})
+                del ss
+                torch.cuda.empty_cache()
+            # cost of one on-chip key-tile rotation as the fused kernel pays it: least squares through the origin of
+            # (fused - no RoPE) against rotations per SM
+            xs = np.array([r["key_tile_rotations"] / 148.0 for r in rows])
+            ys = np.array([(r["fused_ms"] - r["no_rope_ms"]) * 1e3 for r in rows])
+            t_rot_us = float((xs * ys).sum() / (xs * xs).sum())
+            return {"geometry": {"Hq": Hq_, "Hkv": Hkv_, "D": D_, "tokens": tokens}, "rows": rows,
+                    "crossover_S": crossover(rows),
+                    "t_rot_us_per_key_tile_rotation": t_rot_us,
+                    "t_rot_note": "fused minus the same kernel without RoPE, per key-tile rotation and SM (it contains the "
+                                  "Q rotation of the prologue and the hand-offs); the separate pass costs 4*B*S*D*(Hq+Hkv) bytes"}
+
+        ex["rotation_calculus_sweep"] = sweep_geometry(32, 8, 128, 5.0e5, 32768, (512, 1024, 2048, 4096, 8192, 16384, 32768))
+        ex["rotation_calculus_sweep_d64_h12"] = sweep_geometry(12, 12, 64, 1.0e4, 16384, (512, 1024, 2048, 4096, 8192, 16384))
+        ex["rotation_calculus_ridge"] = dict(RIDGE_CONTEXT, b200_measured_flop_per_byte=peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9),
+                                             paper_crossover="~5.5k tokens on H100, none on RTX 3090 (Section 5.3)")
         # separate RoPE kernel alone on a larger-than-L2 buffer (HBM roofline)
         wl = synth.CONFIGS[3]
         x = torch.randn((wl.B, wl.Hq, wl.S, wl.D), device=dev).to(torch.bfloat16)
@@ -551,6 +615,26 @@ def main():
         gbs = 2 * x.numel() * 2 / (t_r / k_ex * 1e-3) / 1e9
         ex["rope_apply_kernel"] = {"bytes": 2 * x.numel() * 2, "ms": t_r / k_ex, "GB/s": gbs,
                                    "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]}
+        # host time of a call through the C-ABI binding (argument marshalling, tensor-map encoding, launches), no sync
+        def host_us(fn, n=200):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for i in range(n):
+                fn(i)
+            dt = time.perf_counter() - t0
+            torch.cuda.synchronize()
+            return dt / n * 1e6
+        wt = synth.Workload("host_call_probe", 1, 8, 2, 256, 128, theta=5.0e5, backward=True, seed_id=54)
+        rt, mt, tt_ = specs(wt)
+        st_ = make_sets(wt, 1)[0]
+        ot, lt = af.fwd(st_["q"], st_["k"], st_["v"], rt, tt_, mt, wt.scale)
+        wst = torch.empty(af.lib().attnfuse_bwd_workspace_bytes(
+            __import__("ctypes").byref(binding._Shape(wt.B, wt.Hq, wt.Hkv, wt.S, wt.D))), dtype=torch.uint8, device=dev)
+        ex["host_us_per_call"] = {
+            "fwd": host_us(lambda i: af.fwd(st_["q"], st_["k"], st_["v"], rt, tt_, mt, wt.scale, out=ot, lse=lt)),
+            "bwd": host_us(lambda i: af.bwd(st_["q"], st_["k"], st_["v"], ot, lt, st_["do"], rt, tt_, mt, wt.scale, workspace=wst)),
+            "decode": ex["flash_decoding"][0]["c_abi_call_from_host_us"],
+            "note": "Python ctypes binding included; small shapes so that the device never back-pressures the host"}
         line["extras"] = ex
         # the three arms of the fuse-or-not experiment on the headline workload, side by side (TFLOP/s)
         c2 = ex[synth.CONFIGS[1].name]

@@ -76,10 +76,9 @@ typedef enum {
                                   heads of one kv head; 0: two consecutive row blocks of one head */
     AF_OPT_FWD_KEYS_BF16 = 2,  /* AF_FWD_KEYS_BF16, default 0: key tiles rotated in packed bf16 arithmetic (faster,
                                   about 1.4 times the rounding error on rotated keys; forward only) */
-    AF_OPT_FWD_CTA_PAIR = 3,   /* AF_FWD_2CTA, default 0: CTA-pair forward kernel for GQA groups that are multiples of 4 */
-    AF_OPT_BS_ROWPAIR = 4,     /* AF_BS_ROWPAIR, default 1: block-sparse forward with an odd GQA group gives a CTA two
+    AF_OPT_BS_ROWPAIR = 3,     /* AF_BS_ROWPAIR, default 1: block-sparse forward with an odd GQA group gives a CTA two
                                   row blocks of one head when the caller supplied pair lists */
-    AF_OPT_COUNT_ = 5
+    AF_OPT_COUNT_ = 4
 } af_option;
 af_status attnfuse_set_option(af_option option, int value);
 int       attnfuse_get_option(af_option option);
@@ -240,7 +239,7 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
  *   o[b,h,:] = softmax_j( c * <q[b,h], k[b,h/g,j]> + m_h (j - (N - 1)) ) v[b,h/g,j],  j kept iff j >= N - 1 - W.
  * Phase 1 splits the cache over n_splits CTAs per (batch, kv head); each computes a partial (max, sum,
  * accumulator) for the g query heads of its kv head (packed as rows of one MMA tile, K and V read once);
- * phase 2 merges the partials with a log-sum-exp.  No rotation is applied: q and the cached keys are used
+ * phase 2 merges the partials with a log-sum-exp (same launch, see `workspace` below).  No rotation is applied: q and the cached keys are used
  * as they are (a cache holds rotated keys; rotate q with attnfuse_rope).  mask->causal is ignored (every
  * cached key precedes the query); window and ALiBi slopes apply as in attnfuse_fwd.
  * q, o: [B,Hq,D] bf16 contiguous (device); k, v: [B,Hkv,N,D] bf16 with strides skv (NULL = contiguous; the
@@ -248,9 +247,15 @@ af_status attnfuse_fwd_host(const af_shape* shape, const void* q_host, const voi
  * gqa_group <= 16; D in {64, 128}.  n_splits <= 0: attnfuse_decode_splits(shape), the largest count that keeps the
  * grid of n_splits x B x Hkv CTAs within one CTA per SM of the current device (one wave) with at least 128 keys
  * per split.  Larger requests are clamped to ceil(S / 128) and to 256 splits.
- * workspace: attnfuse_decode_workspace_bytes(shape, n_splits) device bytes for the partials. */
+ * workspace: attnfuse_decode_workspace_bytes(shape, n_splits) device bytes: a ticket counter per (batch, kv head)
+ * at its head, then the partials.  Both phases run in ONE launch: the CTA that finishes last for a kv head merges
+ * that head group's partials (in split order: the result does not depend on which CTA is last).  The counters must
+ * be ZERO before the first call that uses a workspace - call attnfuse_decode_workspace_init once after allocating it
+ * (it clears the workspace on the given stream) - and every call leaves them zero.  A workspace serves one call at
+ * a time: calls that may overlap on the GPU need workspaces of their own.  After AF_ERR_DEVICE_TIMEOUT, clear it again. */
 int       attnfuse_decode_splits(const af_shape* shape);
 size_t    attnfuse_decode_workspace_bytes(const af_shape* shape, int n_splits);
+af_status attnfuse_decode_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);
 af_status attnfuse_decode(const af_shape* shape, const void* q, const void* k, const void* v,
                           const af_strides* skv, const af_mask* mask, int gqa_group, float softmax_scale,
                           void* o, float* lse, int n_splits,

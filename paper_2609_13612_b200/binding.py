@@ -127,6 +127,8 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_decode_splits.argtypes = [P(_Shape)]
         L.attnfuse_decode_workspace_bytes.restype = sz
         L.attnfuse_decode_workspace_bytes.argtypes = [P(_Shape), i]
+        L.attnfuse_decode_workspace_init.restype = i
+        L.attnfuse_decode_workspace_init.argtypes = [vp, sz, vp]
         L.attnfuse_decode.restype = i
         L.attnfuse_decode.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Mask), i, f, vp, vp, i, vp, sz, vp]
         L.attnfuse_bwd_static.restype = i
@@ -146,7 +148,7 @@ def version() -> int:
 
 
 # af_option values (include/attnfuse.h)
-OPT_FWD_QTILES, OPT_FWD_PAIR_HEADS, OPT_FWD_KEYS_BF16, OPT_FWD_CTA_PAIR, OPT_BS_ROWPAIR = range(5)
+OPT_FWD_QTILES, OPT_FWD_PAIR_HEADS, OPT_FWD_KEYS_BF16, OPT_BS_ROWPAIR = range(4)
 
 
 def set_option(option: int, value: int) -> None:
@@ -486,9 +488,9 @@ def decode(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, mask: MaskSpec, so
     sh = _Shape(B, Hq, Hkv, N, D)
     if n_splits <= 0:
         n_splits = lib().attnfuse_decode_splits(ctypes.byref(sh))
-    n_ws = lib().attnfuse_decode_workspace_bytes(ctypes.byref(sh), n_splits)
-    if workspace is None:
-        workspace = torch.empty(n_ws, dtype=torch.uint8, device=q.device)
+    if workspace is None:   # (a caller's own workspace must have been cleared once: decode_workspace)
+        workspace = torch.zeros(lib().attnfuse_decode_workspace_bytes(ctypes.byref(sh), n_splits), dtype=torch.uint8,
+                                device=q.device)
     skv = _strides(k)
     m = _mask_struct(mask)
     _check(lib().attnfuse_decode(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), ctypes.byref(skv),
@@ -496,6 +498,14 @@ def decode(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, mask: MaskSpec, so
                                  lse.data_ptr() if lse is not None else None, int(n_splits), workspace.data_ptr(),
                                  workspace.numel() * workspace.element_size(), _stream()))
     return out, lse
+
+
+def decode_workspace(B: int, Hq: int, Hkv: int, N: int, D: int, n_splits: int = 0, device="cuda") -> torch.Tensor:
+    """A cleared workspace for `decode` on this geometry (its ticket counters must start at zero)."""
+    sh = _Shape(B, Hq, Hkv, N, D)
+    ws = torch.empty(lib().attnfuse_decode_workspace_bytes(ctypes.byref(sh), n_splits), dtype=torch.uint8, device=device)
+    _check(lib().attnfuse_decode_workspace_init(ws.data_ptr(), ws.numel(), _stream()))
+    return ws
 
 
 def bwd_static(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softmax_scale: float,

@@ -14,7 +14,6 @@
 #include "bwd_kernel.cuh"
 #include "bwd_first_rows.cuh"
 #include "decode_kernels.cuh"
-#include "fwd2_kernel.cuh"
 #include "rope_kernels.cuh"
 
 namespace {
@@ -40,7 +39,47 @@ EncodeTiledFn get_encode() {
 
 // Tensor map over a bf16 tensor [B, H, S, D] (D contiguous) with a box of [rows x 64 columns],
 // 128-byte swizzle, zero fill outside the tensor.
+// Encoding a tensor map costs a driver call of a few microseconds, several per entry point; a map depends only
+// on the pointer, the extents, the strides and the box, so each host thread keeps the last few it built.
+struct TmapKey {
+    const void* ptr;
+    int B, H, S, D, rows;
+    int64_t sb, sh, ss;
+    bool operator==(const TmapKey& o) const {
+        return ptr == o.ptr && B == o.B && H == o.H && S == o.S && D == o.D && rows == o.rows && sb == o.sb && sh == o.sh &&
+               ss == o.ss;
+    }
+};
+struct TmapSlot {
+    TmapKey key;
+    CUtensorMap map;
+    bool valid;
+};
+constexpr int kTmapSlots = 32;
+thread_local TmapSlot t_tmap_cache[kTmapSlots];
+
+af_status make_tmap_uncached(CUtensorMap* tm, const void* ptr, int B, int H, int S, int D, const af_strides& st, int rows);
+
 af_status make_tmap(CUtensorMap* tm, const void* ptr, int B, int H, int S, int D, const af_strides& st, int rows) {
+    const TmapKey key{ptr, B, H, S, D, rows, st.b, st.h, st.s};
+    uint64_t hsh = reinterpret_cast<uintptr_t>(ptr) >> 4;
+    hsh ^= (static_cast<uint64_t>(S) * 0x9E3779B97F4A7C15ull) ^ (static_cast<uint64_t>(H) << 20) ^ (static_cast<uint64_t>(rows) << 7) ^
+           static_cast<uint64_t>(st.s);
+    TmapSlot& slot = t_tmap_cache[(hsh ^ (hsh >> 17)) % kTmapSlots];
+    if (slot.valid && slot.key == key) {
+        *tm = slot.map;
+        return AF_OK;
+    }
+    const af_status r = make_tmap_uncached(tm, ptr, B, H, S, D, st, rows);
+    if (r == AF_OK) {
+        slot.key = key;
+        slot.map = *tm;
+        slot.valid = true;
+    }
+    return r;
+}
+
+af_status make_tmap_uncached(CUtensorMap* tm, const void* ptr, int B, int H, int S, int D, const af_strides& st, int rows) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return AF_ERR_CUDA;
     cuuint64_t dims[4] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(S), static_cast<cuuint64_t>(H),
@@ -84,7 +123,6 @@ constexpr OptionDef kOptionDefs[AF_OPT_COUNT_] = {
     {"AF_FWD_NQ", 2},           // AF_OPT_FWD_QTILES
     {"AF_FWD_PAIR", 1},         // AF_OPT_FWD_PAIR_HEADS
     {"AF_FWD_KEYS_BF16", 0},    // AF_OPT_FWD_KEYS_BF16
-    {"AF_FWD_2CTA", 0},         // AF_OPT_FWD_CTA_PAIR
     {"AF_BS_ROWPAIR", 1},       // AF_OPT_BS_ROWPAIR
 };
 std::atomic<int> g_options[AF_OPT_COUNT_];
@@ -224,11 +262,11 @@ af_status resolve_strides(const af_strides* in, int H, int S, int D, af_strides*
     return AF_OK;
 }
 
-template <int D, int NQ, bool ROPE, int KS, int VS, bool TAB = false>
+template <int D, int NQ, bool ROPE, int KS, int VS, bool TAB = false, bool GEN = false>
 af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const CUtensorMap& tt,
                              FwdParams p, cudaStream_t stream) {
     using L = FwdSmem<D, NQ, KS, VS, ROPE && TAB>;
-    auto kern = attn_fwd_kernel<D, NQ, ROPE, KS, VS, false, TAB>;
+    auto kern = attn_fwd_kernel<D, NQ, ROPE, KS, VS, false, TAB, GEN>;
     static std::atomic<unsigned long long> configured{0};
     if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
     // an even GQA group lets the two query tiles of a CTA be two heads of one kv head (same key range)
@@ -245,40 +283,13 @@ af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
-// CTA-pair variant (fwd2_kernel.cuh): clusters of two CTAs, one per (batch, head quad, 128-row block).
-// tk2: tensor map over K with 64-row boxes.
-template <bool ROPE>
-af_status launch_fwd2_variant(const CUtensorMap& tq, const CUtensorMap& tk2, const CUtensorMap& tv, FwdParams p,
-                              cudaStream_t stream) {
-    constexpr int KS = 3, VS = 3;
-    using L = Fwd2Smem<128, KS, VS>;
-    auto kern = attn_fwd2_kernel<128, ROPE, KS, VS>;
-    static std::atomic<unsigned long long> configured{0};
-    if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
-    p.pair_heads = 0;
-    p.n_row_blocks = (p.S + BM - 1) / BM;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2u * p.B * (p.Hq / 4), p.n_row_blocks, 1);
-    cfg.blockDim = dim3(512, 1, 1);
-    cfg.dynamicSmemBytes = L::BYTES;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, tq, tk2, tv, p) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
-}
-
 // Block-sparse variant (Section 4.3): the grid is (heads or head pairs, 128-row blocks); every CTA walks the
 // list of active key blocks of its row block.  An even GQA group pairs two heads per CTA, otherwise one head.
-template <int D, int NQ, bool ROPE>
+template <int D, int NQ, bool ROPE, bool GEN = false>
 af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                                     const CUtensorMap& to, const CUtensorMap& tt, FwdParams p, cudaStream_t stream) {
     using L = FwdSmem<D, NQ, 2, 2>;
-    auto kern = attn_fwd_kernel<D, NQ, ROPE, 2, 2, true>;
+    auto kern = attn_fwd_kernel<D, NQ, ROPE, 2, 2, true, false, GEN>;
     static std::atomic<unsigned long long> configured{0};
     if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
     // NQ = 2: two heads of one kv head on the same row block (even GQA group), or - with pair lists - the row
@@ -294,7 +305,13 @@ template <int D>
 af_status launch_fwd_blocks(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const CUtensorMap& tt,
                             const FwdParams& p, cudaStream_t stream) {
     // (p.bs_rowpair is set only for an odd GQA group, when the caller supplied the lists of row-block pairs)
-    if ((p.group % 2) == 0 || p.bs_rowpair)
+    const bool two_tiles = (p.group % 2) == 0 || p.bs_rowpair;
+    if (p.bias || p.relu) {   // Section 3.1 extras: built for CTAs of two query tiles only
+        if (!two_tiles) return AF_ERR_SPEC;
+        return p.R > 0 ? launch_fwd_blocks_variant<D, 2, true, true>(tq, tk, tv, to, tt, p, stream)
+                       : launch_fwd_blocks_variant<D, 2, false, true>(tq, tk, tv, to, tt, p, stream);
+    }
+    if (two_tiles)
         return p.R > 0 ? launch_fwd_blocks_variant<D, 2, true>(tq, tk, tv, to, tt, p, stream)
                        : launch_fwd_blocks_variant<D, 2, false>(tq, tk, tv, to, tt, p, stream);
     return p.R > 0 ? launch_fwd_blocks_variant<D, 1, true>(tq, tk, tv, to, tt, p, stream)
@@ -304,6 +321,9 @@ af_status launch_fwd_blocks(const CUtensorMap& tq, const CUtensorMap& tk, const 
 template <int D>
 af_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to, const CUtensorMap& tt, const FwdParams& p,
                      cudaStream_t stream) {
+    if (p.bias || p.relu)   // Section 3.1 extras (additive_bias, relu_attention): their own instantiation
+        return p.R > 0 ? launch_fwd_variant<D, 2, true, 2, 2, false, true>(tq, tk, tv, to, tt, p, stream)
+                       : launch_fwd_variant<D, 2, false, 2, 2, false, true>(tq, tk, tv, to, tt, p, stream);
     const int nq = opt(AF_OPT_FWD_QTILES);
     if (nq == 1) {
         return p.R > 0 ? launch_fwd_variant<D, 1, true, 2, 2>(tq, tk, tv, to, tt, p, stream)
@@ -599,7 +619,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     // (optional mode) key tiles receive the 128 rows of the table's bf16 copy that belong to them by TMA
     const int Rr = rope->rotary_dim;
     CUtensorMap tt = tq;
-    const bool keys_bf16 = !k_prerotated && keys_rotate_in_bf16(Rr);
+    const bool keys_bf16 = !k_prerotated && !bias && !relu && keys_rotate_in_bf16(Rr);
     if (keys_bf16 && (st = make_tmap_table(&tt, rope_table, shape->S, Rr)) != AF_OK) return st;
 
     FwdParams p;
@@ -637,13 +657,6 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (bs_row_ptr)
         return shape->D == 128 ? launch_fwd_blocks<128>(tq, tk, tv, to, tt, p, stream) : launch_fwd_blocks<64>(tq, tk, tv, to, tt, p, stream);
-    const int R = rope->rotary_dim;
-    const bool pair_ok = shape->D == 128 && (gqa_group % 4) == 0 && (R == 0 || R == 16 || R == 32 || R == 64 || R == 128);
-    if (pair_ok && !k_prerotated && !bias && !relu && opt(AF_OPT_FWD_CTA_PAIR)) {
-        CUtensorMap tk2;
-        if ((st = make_tmap(&tk2, k, shape->B, shape->Hkv, shape->S, shape->D, stkv, 64)) != AF_OK) return st;
-        return R > 0 ? launch_fwd2_variant<true>(tq, tk2, tv, p, stream) : launch_fwd2_variant<false>(tq, tk2, tv, p, stream);
-    }
     return shape->D == 128 ? launch_fwd<128>(tq, tk, tv, to, tt, p, stream) : launch_fwd<64>(tq, tk, tv, to, tt, p, stream);
 }
 }  // namespace
@@ -844,10 +857,22 @@ int attnfuse_decode_splits(const af_shape* shape) {
     return want < 1 ? 1 : (want > most ? most : want);
 }
 
+// bytes of the ticket counters at the head of the decode workspace (one per (batch, kv head), rounded up to 256)
+static size_t decode_ticket_bytes(const af_shape* shape) {
+    return (static_cast<size_t>(shape->B) * shape->Hkv * sizeof(unsigned int) + 255) / 256 * 256;
+}
+
 size_t attnfuse_decode_workspace_bytes(const af_shape* shape, int n_splits) {
     if (!shape) return 0;
     if (n_splits <= 0) n_splits = attnfuse_decode_splits(shape);
-    return static_cast<size_t>(shape->B) * shape->Hq * n_splits * (shape->D + 2) * sizeof(float);
+    return decode_ticket_bytes(shape) + static_cast<size_t>(shape->B) * shape->Hq * n_splits * (shape->D + 2) * sizeof(float);
+}
+
+af_status attnfuse_decode_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!workspace) return AF_ERR_NULL;
+    if (!aligned16(workspace)) return AF_ERR_ALIGN;
+    return cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? AF_OK
+                                                                                                              : AF_ERR_CUDA;
 }
 
 af_status attnfuse_decode(const af_shape* shape, const void* q, const void* k, const void* v, const af_strides* skv,
@@ -878,8 +903,11 @@ af_status attnfuse_decode(const af_shape* shape, const void* q, const void* k, c
     p.slopes = mask->alibi_slopes;
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.n_splits = n_splits;
-    p.part_o = static_cast<float*>(workspace);
+    p.tickets = static_cast<unsigned int*>(workspace);
+    p.part_o = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + decode_ticket_bytes(shape));
     p.part_ml = p.part_o + static_cast<size_t>(shape->B) * shape->Hq * n_splits * shape->D;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.lse = lse;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     dim3 grid(n_splits, shape->B * shape->Hkv, 1);
     if (shape->D == 128) {
@@ -891,9 +919,6 @@ af_status attnfuse_decode(const af_shape* shape, const void* q, const void* k, c
         if (allow_dynamic_smem(decode_split_kernel<64>, DecodeSmem<64>::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
         decode_split_kernel<64><<<grid, kDecWarps * 32, DecodeSmem<64>::BYTES, stream>>>(tk, tv, p);
     }
-    if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
-    decode_combine_kernel<<<shape->B * shape->Hq, kCombineThreads, 0, stream>>>(p.part_o, p.part_ml, n_splits, shape->D,
-                                                                         static_cast<__nv_bfloat16*>(o), lse);
     return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 

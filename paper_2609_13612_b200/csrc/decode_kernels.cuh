@@ -3,8 +3,8 @@
 // Phase 1 (decode_split_kernel): the cache is cut into splits; a CTA takes one split of one kv head
 // and computes, for the g query heads of that kv head, a partial (m, l, acc) triple with the online
 // softmax.  The g heads are the rows of a 16-row MMA tile (padded by cyclic replication, as the paper
-// does), so K and V are read exactly once per CTA.  Phase 2 (decode_combine_kernel) merges the
-// partials with a log-sum-exp.
+// does), so K and V are read exactly once per CTA.  Phase 2 merges the partials with a log-sum-exp; it runs in
+// the same launch, in the CTA that finishes last for its kv head (a ticket counter tells which).
 //
 // The path is bound by HBM (every K and V byte is read once and used for 4 g flops), so the kernel is
 // built around the memory system: each of the 4 warps of a CTA streams its own 32-key tiles through
@@ -27,8 +27,16 @@ struct DecodeParams {
     float* part_o;              // [B * Hq, n_splits, D]   unnormalised partial outputs
     float* part_ml;             // [B * Hq, n_splits, 2]   running max (log2 units) and sum of each partial
     int n_splits;               // CTAs per (batch, kv head); the kept 32-key tiles are dealt out evenly among them
+    // Merge in the same launch: one counter per (batch, kv head), zero before the launch.  The CTA that finishes
+    // last for its kv head (it draws the last ticket) merges the partials of the g query heads, in split order,
+    // writes o / lse and sets the counter back to zero.
+    unsigned int* tickets;
+    __nv_bfloat16* o;           // [B, Hq, D]
+    float* lse;                 // [B, Hq] or nullptr
 };
 
+constexpr int kCombineThreads = 128;
+constexpr int kCombineMaxSplits = 1024;
 constexpr int kDecTile = 32;    // keys per warp tile
 constexpr int kDecWarps = 4;
 #ifndef AF_DEC_STAGES
@@ -45,6 +53,7 @@ struct DecodeSmem {
     static constexpr int BYTES = OFF_MISC + 16 + 1024;
     static constexpr int MERGE_STRIDE = D + 4;                               // floats per merged row
     static_assert(kDecWarps * 16 * (MERGE_STRIDE + 2) * 4 <= OFF_BAR, "merge buffer must fit in the stages");
+    static_assert((16 * kCombineMaxSplits + 32) * 4 <= OFF_BAR, "combine weights (up to 16 heads) must fit in the stages");
 };
 
 // 16-byte chunk `chunk` of key row r in a tile of D/64 boxes [32 rows][64 cols], 128-byte swizzle
@@ -310,74 +319,73 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             p.part_ml[row * 2 + 1] = lsum;
         }
     }
-}
 
-// Phase 2: one block of 128 threads per (batch, head).  The weights 2^(m_s - M) of the partials are formed
-// once in shared memory; then thread (sg, d4) sums four head dimensions over the splits s = sg, sg + G, ...
-// (independent 16-byte loads, several in flight), and the G partial sums are added through shared memory.
-constexpr int kCombineThreads = 128;
-constexpr int kCombineMaxSplits = 1024;
-__global__ void __launch_bounds__(kCombineThreads)
-decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_splits, int D,
-                      __nv_bfloat16* __restrict__ o, float* __restrict__ lse) {
-    __shared__ float w[kCombineMaxSplits];
-    __shared__ float red[kCombineThreads];
-    __shared__ float4 acc_s[kCombineThreads];
-    const size_t bh = blockIdx.x;
-    const int tid = threadIdx.x;
-    // M = max_s m_s, L = sum_s l_s 2^(m_s - M)
-    float mloc = -INFINITY;
-    for (int s = tid; s < n_splits; s += kCombineThreads) {
-        const float2 ml = *reinterpret_cast<const float2*>(part_ml + (bh * n_splits + s) * 2);
-        w[s] = ml.x;
-        mloc = fmaxf(mloc, ml.x);
-    }
-    red[tid] = mloc;
+    // ---- phase 2 in the same launch (Section 4.2: log-sum-exp combine of the partials).  Every CTA publishes its
+    // partials (fence), then draws a ticket; the CTA with the last ticket of its kv head sees all of them.  The sums
+    // run over the splits in index order whichever CTA is last, so the result is run-to-run deterministic.
+    __shared__ int s_last;
+    __threadfence();
     __syncthreads();
-    for (int st = kCombineThreads / 2; st > 0; st >>= 1) {
-        if (tid < st) red[tid] = fmaxf(red[tid], red[tid + st]);
-        __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int t = atomicAdd(p.tickets + blockIdx.y, 1u);
+        s_last = (t == static_cast<unsigned int>(p.n_splits) - 1u) ? 1 : 0;
     }
-    const float M = red[0];
     __syncthreads();
-    float lloc = 0.f;
-    for (int s = tid; s < n_splits; s += kCombineThreads) {
-        const float f = M == -INFINITY ? 0.f : ex2(w[s] - M);
-        w[s] = f;
-        lloc = fmaf(part_ml[(bh * n_splits + s) * 2 + 1], f, lloc);
-    }
-    red[tid] = lloc;
-    __syncthreads();
-    for (int st = kCombineThreads / 2; st > 0; st >>= 1) {
-        if (tid < st) red[tid] += red[tid + st];
-        __syncthreads();
-    }
-    const float L = red[0];
-    // weighted sum of the partial accumulators
-    const int tpr = D / 4, G = kCombineThreads / tpr;   // threads per row of D floats, split groups
-    const int d4 = tid % tpr, sg = tid / tpr;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-    for (int s = sg; s < n_splits; s += G) {
-        const float4 v = *reinterpret_cast<const float4*>(part_o + (bh * n_splits + s) * D + d4 * 4);
-        const float f = w[s];
-        acc.x = fmaf(v.x, f, acc.x);
-        acc.y = fmaf(v.y, f, acc.y);
-        acc.z = fmaf(v.z, f, acc.z);
-        acc.w = fmaf(v.w, f, acc.w);
-    }
-    acc_s[tid] = acc;
-    __syncthreads();
-    if (sg == 0) {
-        for (int g2 = 1; g2 < G; ++g2) {
-            const float4 v = acc_s[g2 * tpr + d4];
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    if (!s_last) return;
+    __threadfence();
+    // weights 2^(m_s - M) of every head and split (the stages are idle): one warp per head, lanes over the splits
+    float* wgt = reinterpret_cast<float*>(smem);          // [group][n_splits]
+    float* stat = wgt + 16 * kCombineMaxSplits;            // [group][2]: M, L
+    const int tid = threadIdx.x, n = p.n_splits;
+    const size_t bh0 = static_cast<size_t>(b) * p.Hq + hk * p.group;
+    for (int h = warp; h < p.group; h += kDecWarps) {
+        const float* ml = p.part_ml + (bh0 + h) * n * 2;
+        float mloc = -INFINITY;
+        for (int sidx = lane; sidx < n; sidx += 32) mloc = fmaxf(mloc, __ldcg(ml + sidx * 2));
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, off));
+        float lloc = 0.f;
+        for (int sidx = lane; sidx < n; sidx += 32) {
+            const float2 v2 = __ldcg(reinterpret_cast<const float2*>(ml + sidx * 2));
+            const float f = mloc == -INFINITY ? 0.f : ex2(v2.x - mloc);
+            wgt[h * n + sidx] = f;
+            lloc = fmaf(v2.y, f, lloc);
         }
-        const float inv = L > 0.f ? 1.f / L : 0.f;
-        *reinterpret_cast<uint2*>(o + bh * D + d4 * 4) =
+        // (fixed tree: the sum does not depend on which CTA runs this)
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) lloc += __shfl_xor_sync(0xffffffffu, lloc, off);
+        if (lane == 0) {
+            stat[2 * h] = mloc;
+            stat[2 * h + 1] = lloc;
+        }
+    }
+    __syncthreads();
+    // weighted sums: one thread per (head, four head dims), the splits in index order, 16-byte loads several in flight
+    constexpr int D4 = D / 4;
+    for (int idx = tid; idx < p.group * D4; idx += kDecWarps * 32) {
+        const int h = idx / D4, d4 = idx - h * D4;
+        const float4* po = reinterpret_cast<const float4*>(p.part_o + (bh0 + h) * n * D) + d4;
+        const float* wh = wgt + h * n;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+        for (int sidx = 0; sidx < n; ++sidx) {
+            const float4 v4 = __ldcg(po + static_cast<size_t>(sidx) * D4);
+            const float f = wh[sidx];
+            acc.x = fmaf(v4.x, f, acc.x);
+            acc.y = fmaf(v4.y, f, acc.y);
+            acc.z = fmaf(v4.z, f, acc.z);
+            acc.w = fmaf(v4.w, f, acc.w);
+        }
+        const float Lsum = stat[2 * h + 1];
+        const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+        *reinterpret_cast<uint2*>(p.o + (bh0 + h) * D + d4 * 4) =
             make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
     }
-    if (lse && tid == 0) lse[bh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+    if (p.lse && tid < p.group) {
+        const float M = stat[2 * tid], Lsum = stat[2 * tid + 1];
+        p.lse[bh0 + tid] = Lsum > 0.f ? (M + log2f(Lsum)) * 0.6931471805599453f : -INFINITY;
+    }
+    if (tid == 0) p.tickets[blockIdx.y] = 0u;   // ready for the next call on this workspace
 }
 
 }  // namespace af

@@ -89,14 +89,8 @@ __device__ long long* g_trace = nullptr;
 #endif
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the row max grows by more
 
-#ifndef AF_SPLIT_S
-#define AF_SPLIT_S 0
-#endif
-constexpr bool kSplitS = AF_SPLIT_S != 0;   // S tile produced as two N = 64 halves (measured slower: N = 64 MMAs are inefficient)
-#ifndef AF_P_PARTS
-#define AF_P_PARTS 2
-#endif
-constexpr int kPParts = AF_P_PARTS;          // P is handed to the MMA issuer in this many column parts (2 or 4)
+constexpr int kPParts = 2;   // P is handed to the MMA issuer in two column halves (four parts, and an S tile produced as
+                             // two N = 64 halves, measured slower)
 
 // One key tile of the online softmax for one query row (this thread's TMEM lane): reads the 128
 // raw scores, adds ALiBi and the mask in the raw domain, updates the running max and sum in the
@@ -105,14 +99,11 @@ constexpr int kPParts = AF_P_PARTS;          // P is handed to the MMA issuer in
 //   score (log2 domain) t_e = c2 * (S_e + kb * e) + bias0,  kb = slope2 / c2, bias0 = slope2 * (j0 - i)
 // The work is handed over in column halves, so that less of it sits on the
 // S-MMA -> softmax -> PV-MMA dependency chain of a query tile:
-//  - with kSplitS the scores arrive as two 64-column halves (two barriers): the TMEM load of the first
-//    half overlaps the MMAs of the second;
 //  - P goes back in two halves, each announced on its own barrier (p_ready[0], p_ready[1]), so that the
 //    first four K-steps of O += P V run while the second half of the exponentials is computed.
 // P halves sit at the start of their own 64 score columns (bf16 pairs: 32 columns each).
 // Returns false if a bounded wait gave up.
-// PAIR: the barriers p_ready live in the leader CTA of a CTA pair (arrive through the cluster).
-template <int D, bool MASKED, bool ALIBI, bool PAIR = false>
+template <int D, bool MASKED, bool ALIBI>
 __device__ __forceinline__ bool softmax_tile_halves(uint32_t tS, uint32_t tO, int n, float scale_log2, float kb,
                                                     float bias0, int mlo, uint32_t mn, uint64_t* s_full, uint64_t* p_ready,
                                                     uint32_t parity, volatile uint32_t* abort_flag, int lane, float& m_run,
@@ -122,13 +113,6 @@ __device__ __forceinline__ bool softmax_tile_halves(uint32_t tS, uint32_t tO, in
     tc_fence_after_sync();
     tmem_ld32(tS, v);
     tmem_ld32(tS + 32, v + 32);
-    if (kSplitS) {
-        if (!mbar_wait_warp(&s_full[1], parity, abort_flag, 10)) {
-            tmem_wait_ld();
-            return false;
-        }
-        tc_fence_after_sync();
-    }
     tmem_ld32(tS + 64, v + 64);
     tmem_ld32(tS + 96, v + 96);
     tmem_wait_ld();
@@ -192,10 +176,7 @@ __device__ __forceinline__ bool softmax_tile_halves(uint32_t tS, uint32_t tO, in
         tmem_wait_st();
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) {
-            if (PAIR) mbar_arrive_cluster(&p_ready[pt], 0);
-            else mbar_arrive(&p_ready[pt]);
-        }
+        if (lane == 0) mbar_arrive(&p_ready[pt]);
         if (pt == 0) AF_STAMP_SM(5);
     }
     l_run = l_run * alpha + ((ps2[0].x + ps2[0].y) + (ps2[1].x + ps2[1].y));
@@ -310,7 +291,9 @@ __device__ __forceinline__ bool softmax_tile_general(uint32_t tS, uint32_t tO, i
 
 // TAB (with ROPE): key tiles are rotated in packed bf16 arithmetic from table tiles that arrive by TMA through
 // tm_t (the bf16 copy of the cos/sin table); otherwise in fp32 arithmetic from the fp32 table rows.
-template <int D, int NQ, bool ROPE, int KS, int VS, bool BS = false, bool TAB = false>
+// GEN: the instantiation for the variants with an additive bias or the ReLU normaliser (softmax_tile_general); kept
+// apart so that the kernels of the other variants carry none of its registers.
+template <int D, int NQ, bool ROPE, int KS, int VS, bool BS = false, bool TAB = false, bool GEN = false>
 __global__ void __launch_bounds__(128 * (2 + NQ), 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -485,28 +468,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             auto issue_S = [&](int q, int ks) {
                 const uint32_t q_lo = desc_lo(smem_u32(sQ + q * TILE), 16), k_lo = desc_lo(smem_u32(sK + ks * TILE), 16);
                 const uint32_t d = tmem_base + q * BN;
-                if (kSplitS) {
-                    // two N = 64 halves: key rows [64 h, 64 h + 64) of the tile (8 KB further in each box)
-                    constexpr uint32_t IDESC_SH = idesc_bf16_f32(BM, 64, 0, 0);
 #pragma unroll
-                    for (int hf = 0; hf < 2; ++hf) {
-#pragma unroll
-                        for (int kk = 0; kk < D / 16; ++kk) {
-                            const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
-                            if (kk == 0) mma_ss_lo<false>(d + hf * 64, q_lo + off, k_lo + off + hf * 512, dhi, IDESC_SH);
-                            else mma_ss_lo<true>(d + hf * 64, q_lo + off, k_lo + off + hf * 512, dhi, IDESC_SH);
-                        }
-                        mma_commit(&bars[L::B_SFULL + 2 * q + hf]);
-                    }
-                } else {
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
-                        if (kk == 0) mma_ss_lo<false>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
-                        else mma_ss_lo<true>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
-                    }
-                    mma_commit(&bars[L::B_SFULL + 2 * q]);
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
+                    if (kk == 0) mma_ss_lo<false>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
+                    else mma_ss_lo<true>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
                 }
+                mma_commit(&bars[L::B_SFULL + 2 * q]);
             };
             // part pt of O += P V: its 8 / kPParts K-steps; that part of P starts at its own score columns
             auto issue_O_part = [&](int q, int vs, bool acc, int pt) {
@@ -691,7 +659,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (need_mask) kept_keys_of_query(ms, i, j0, mlo, mn);
             uint64_t* sf = &bars[L::B_SFULL + 2 * q];
             uint64_t* pr = &bars[L::B_PREADY + 4 * q];
-            if (p.bias || p.relu) {
+            if constexpr (GEN) {
                 // Section 3.1: additive_bias / relu_attention
                 const float* brow = nullptr;
                 if (p.bias && i < p.S)
@@ -771,7 +739,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
             }
-            if (p.lse && !p.relu && i < p.S)
+            if (p.lse && !(GEN && p.relu) && i < p.S)
                 p.lse[static_cast<size_t>(bh) * p.S + i] =
                     l_run > 0.f ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
         }

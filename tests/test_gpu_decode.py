@@ -106,3 +106,27 @@ def test_decode_argument_errors():
     with pytest.raises(af.AttnFuseError) as e:
         af.decode(qd, kd, vd, mask, -1.0)
     assert e.value.code == 5
+
+
+def test_decode_reuses_one_cleared_workspace_over_many_calls():
+    """The ticket counters at the head of the workspace are cleared once (decode_workspace) and every call leaves
+    them at zero: repeated calls on the same workspace, with changing inputs, all match the oracle; the last CTA
+    to finish differs from call to call, the bits of the result do not."""
+    B, Hq, Hkv, N, D = 2, 8, 2, 1900, 128
+    ws = af.decode_workspace(B, Hq, Hkv, N, D)
+    mask = af.MaskSpec(True, -1, None)
+    first = None
+    for it in range(6):
+        q, k, v = draw(B, Hq, Hkv, N, D, 350 + (it % 2))
+        qd, kd, vd = pu.to_dev(q), pu.to_dev(k), pu.to_dev(v)
+        o, lse = af.decode(qd, kd, vd, mask, D ** -0.5, workspace=ws)
+        torch.cuda.synchronize()
+        assert af.device_status()[0] == 0
+        assert int(ws[:256].view(torch.int32).abs().sum().item()) == 0      # counters back at zero
+        want_o, want_l = oracle_decode(q, k, v, D ** -0.5)
+        pu.assert_close("decode call %d" % it, pu.to_np(o), want_o)
+        assert np.abs(pu.to_np(lse) - want_l).max() <= pu.LSE_TOL
+        if it == 0:
+            first = (o.clone(), lse.clone())
+        if it == 2:
+            assert torch.equal(o, first[0]) and torch.equal(lse, first[1])

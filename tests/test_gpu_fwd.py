@@ -281,26 +281,3 @@ def test_config4_long_context_sampled_rows():
     idx = torch.tensor(rows, device="cuda")
     pu.assert_close("c4 O", pu.to_np(o[:, :, idx]), want_o)
     assert np.abs(pu.to_np(lse[:, :, idx]) - want_l).max() <= pu.LSE_TOL
-
-
-PAIR_CASES = [
-    W("pair_norope_dense", 1, 4, 1, 128, 128, rotary_dim=0, causal=False, seed_id=140),
-    W("pair_rope_causal_g4", 2, 8, 2, 640, 128, theta=5e5, seed_id=141),
-    W("pair_rope_causal_g8", 1, 8, 1, 512, 128, theta=5e5, seed_id=142),
-    W("pair_ragged", 1, 4, 1, 333, 128, theta=1e4, seed_id=143),
-    W("pair_window_alibi", 1, 8, 2, 700, 128, theta=1e4, window=200, alibi=True, seed_id=144),
-    W("pair_partial_rotary", 1, 4, 1, 256, 128, theta=1e4, rotary_dim=64, seed_id=145),
-    W("pair_single_row", 1, 4, 1, 1, 128, theta=1e4, seed_id=146),
-]
-
-
-@pytest.mark.parametrize("w", PAIR_CASES, ids=lambda w: w.name)
-def test_forward_cta_pair_kernel(w):
-    """The CTA-pair variant (two SMs share the K/V tiles of a GQA quad; cta_group::2 MMAs)."""
-    with af.option(af.OPT_FWD_CTA_PAIR, 1):
-        run_case(w)
-
-
-def test_forward_cta_pair_kernel_config2():
-    with af.option(af.OPT_FWD_CTA_PAIR, 1):
-        run_case(synth.CONFIGS[1])
