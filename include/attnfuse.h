@@ -78,7 +78,11 @@ typedef enum {
                                   about 1.4 times the rounding error on rotated keys; forward only) */
     AF_OPT_BS_ROWPAIR = 3,     /* AF_BS_ROWPAIR, default 1: block-sparse forward with an odd GQA group gives a CTA two
                                   row blocks of one head when the caller supplied pair lists */
-    AF_OPT_COUNT_ = 4
+    AF_OPT_BWD_ONEPASS = 4,    /* AF_BWD_ONEPASS, default 1: where the one-pass sequence of attnfuse_bwd applies (D = 128, dense,
+                                  workspace of attnfuse_bwd_onepass_workspace_bytes) it is taken when rows are short (at most
+                                  12 kept key tiles per query tile on average), where it measured faster; 2: whenever it
+                                  applies; 0: never - always the two-kernel sequence, whose dQ is bit-reproducible */
+    AF_OPT_COUNT_ = 5
 } af_option;
 af_status attnfuse_set_option(af_option option, int value);
 int       attnfuse_get_option(af_option option);
@@ -274,8 +278,18 @@ af_status attnfuse_decode(const af_shape* shape, const void* q, const void* k, c
  * loop.  A smaller workspace is accepted: with delta + K cache the dK/dV kernel runs first, rotates K once
  * per key tile and every Q tile it streams, and the dQ kernel streams the cached K; with delta alone both
  * kernels rotate everything they touch on chip.  Results of the three set-ups agree up to the bf16
- * rounding of a few rotated elements. */
+ * rounding of a few rotated elements.  These three are deterministic: no atomics, every accumulator has one
+ * owner and a fixed order of additions.
+ * One-pass sequence (D = 128, dense masks): with a workspace of attnfuse_bwd_onepass_workspace_bytes(shape) -
+ * the three pieces above followed by an fp32 accumulator of dQ (B*Hq*S*D*4 bytes) - and where option
+ * AF_OPT_BWD_ONEPASS selects it, RoPE passes write both caches and ONE kernel per key tile forms dK, dV and its
+ * share of dQ (five tile products per kept tile pair instead of seven; S and dP are not recomputed a second
+ * time).  The shares of dQ from different key tiles are added into the accumulator with fp32 reductions in
+ * global memory, in an order that depends on CTA scheduling: dQ may differ in its last bits from run to run
+ * (within the same bounds against the exact result); dK and dV stay reproducible.  A last pass scales the
+ * accumulator, rotates it back and writes dq.  The accumulator needs no initialisation by the caller. */
 size_t    attnfuse_bwd_workspace_bytes(const af_shape* shape);
+size_t    attnfuse_bwd_onepass_workspace_bytes(const af_shape* shape);
 af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, const void* v,
                        const void* o, const float* lse, const void* d_o,
                        const af_strides* sq, const af_strides* skv,

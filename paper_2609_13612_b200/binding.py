@@ -114,6 +114,8 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_fwd_host.argtypes = [P(_Shape), vp, vp, vp, P(_Rope), vp, P(_Mask), i, f, vp, vp, vp, sz, vp]
         L.attnfuse_bwd_workspace_bytes.restype = sz
         L.attnfuse_bwd_workspace_bytes.argtypes = [P(_Shape)]
+        L.attnfuse_bwd_onepass_workspace_bytes.restype = sz
+        L.attnfuse_bwd_onepass_workspace_bytes.argtypes = [P(_Shape)]
         L.attnfuse_bwd.restype = i
         L.attnfuse_bwd.argtypes = [P(_Shape), vp, vp, vp, vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp,
                                    P(_Mask), i, f, vp, i, vp, vp, i, vp, sz, vp]
@@ -148,7 +150,7 @@ def version() -> int:
 
 
 # af_option values (include/attnfuse.h)
-OPT_FWD_QTILES, OPT_FWD_PAIR_HEADS, OPT_FWD_KEYS_BF16, OPT_BS_ROWPAIR = range(4)
+OPT_FWD_QTILES, OPT_FWD_PAIR_HEADS, OPT_FWD_KEYS_BF16, OPT_BS_ROWPAIR, OPT_BWD_ONEPASS = range(5)
 
 
 def set_option(option: int, value: int) -> None:
@@ -430,19 +432,29 @@ def fwd_host_staging_bytes(B: int, Hq: int, Hkv: int, S: int, D: int) -> int:
     return lib().attnfuse_fwd_host_staging_bytes(ctypes.byref(sh))
 
 
+def bwd_workspace_bytes(B: int, Hq: int, Hkv: int, S: int, D: int, onepass: bool = True) -> int:
+    """Workspace size of the backward: with `onepass` the size that admits the one-pass sequence (delta, both
+    rotated caches and the fp32 dQ accumulator; D = 128), otherwise delta and the two caches."""
+    sh = _Shape(B, Hq, Hkv, S, D)
+    if onepass and D == 128:
+        return lib().attnfuse_bwd_onepass_workspace_bytes(ctypes.byref(sh))
+    return lib().attnfuse_bwd_workspace_bytes(ctypes.byref(sh))
+
+
 def bwd(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softmax_scale: float,
         dq_dtype: torch.dtype = torch.bfloat16, dkv_dtype: torch.dtype = torch.float32, workspace=None,
         blocks: Optional[BlockMask] = None):
-    """Fused backward (over the active blocks of `blocks`, if given).  Returns (dq, dk, dv)."""
+    """Fused backward (over the active blocks of `blocks`, if given).  Returns (dq, dk, dv).
+    Without a workspace of the caller's, one of the largest useful size is allocated (`bwd_workspace_bytes`)."""
     _need_cuda(q, k, v, o, lse, d_o, table, workspace)
     B, Hq, S, D = q.shape
     Hkv = k.shape[1]
     assert o.is_contiguous() and d_o.is_contiguous() and lse.is_contiguous()
     assert o.dtype == d_o.dtype == torch.bfloat16 and lse.dtype == torch.float32
     sh = _Shape(B, Hq, Hkv, S, D)
-    n_ws = lib().attnfuse_bwd_workspace_bytes(ctypes.byref(sh))
     if workspace is None:
-        workspace = torch.empty(n_ws, dtype=torch.uint8, device=q.device)
+        workspace = torch.empty(bwd_workspace_bytes(B, Hq, Hkv, S, D, onepass=blocks is None), dtype=torch.uint8,
+                                device=q.device)
     dq = torch.empty((B, Hq, S, D), dtype=dq_dtype, device=q.device)
     dk = torch.empty((B, Hkv, S, D), dtype=dkv_dtype, device=q.device)
     dv = torch.empty((B, Hkv, S, D), dtype=dkv_dtype, device=q.device)

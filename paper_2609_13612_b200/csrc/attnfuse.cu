@@ -1,6 +1,7 @@
 // Host side of the C-ABI declared in include/attnfuse.h: argument validation, tensor-map
 // encoding, variant selection and launches.  All arithmetic of the path runs in the kernels.
 #include <cuda.h>
+#include <algorithm>
 #include <atomic>
 #include <utility>
 #include <cuda_runtime.h>
@@ -13,6 +14,7 @@
 #include "fwd_kernel.cuh"
 #include "bwd_kernel.cuh"
 #include "bwd_first_rows.cuh"
+#include "bwd_fused_kernel.cuh"
 #include "decode_kernels.cuh"
 #include "rope_kernels.cuh"
 
@@ -124,6 +126,7 @@ constexpr OptionDef kOptionDefs[AF_OPT_COUNT_] = {
     {"AF_FWD_PAIR", 1},         // AF_OPT_FWD_PAIR_HEADS
     {"AF_FWD_KEYS_BF16", 0},    // AF_OPT_FWD_KEYS_BF16
     {"AF_BS_ROWPAIR", 1},       // AF_OPT_BS_ROWPAIR
+    {"AF_BWD_ONEPASS", 1},      // AF_OPT_BWD_ONEPASS
 };
 std::atomic<int> g_options[AF_OPT_COUNT_];
 std::once_flag g_options_once;
@@ -388,17 +391,75 @@ af_status launch_bwd_mma(const af_shape* sh, const CUtensorMap& tq, const CUtens
                          int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, const af_blocks* blocks,
                          cudaStream_t stream);
 
+struct OnePassArgs;
+af_status launch_bwd_onepass(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                             const CUtensorMap& tdo, const CUtensorMap& tkp, const CUtensorMap& tqp, const void* k,
+                             const af_strides& stkv, void* kcache, const void* o, const void* d_o, BwdParams p, void* dq,
+                             int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, const OnePassArgs& a,
+                             cudaStream_t stream);
+
 template <int D>
 af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                      const CUtensorMap& tdo, const CUtensorMap* tkp, const CUtensorMap* tqp, const void* k,
                      const af_strides& stkv, void* kcache, const void* o, const void* d_o, BwdParams p, void* dq,
                      int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, const af_blocks* blocks,
-                     cudaStream_t stream, const FirstRowsParams& fp) {
+                     cudaStream_t stream, const FirstRowsParams& fp, const OnePassArgs* onepass) {
     p.skip_rows = fp.rows;
-    af_status st = launch_bwd_mma<D>(sh, tq, tk, tv, tdo, tkp, tqp, k, stkv, kcache, o, d_o, p, dq, dq_f32, dk, dv, dkv_f32,
-                                     delta, blocks, stream);
+    af_status st;
+    if constexpr (D == 128) {
+        st = onepass ? launch_bwd_onepass(sh, tq, tk, tv, tdo, tkp ? *tkp : tk, tqp ? *tqp : tq, k, stkv, kcache, o, d_o, p, dq, dq_f32, dk, dv,
+                                          dkv_f32, delta, *onepass, stream)
+                     : launch_bwd_mma<D>(sh, tq, tk, tv, tdo, tkp, tqp, k, stkv, kcache, o, d_o, p, dq, dq_f32, dk, dv,
+                                         dkv_f32, delta, blocks, stream);
+    } else {
+        st = launch_bwd_mma<D>(sh, tq, tk, tv, tdo, tkp, tqp, k, stkv, kcache, o, d_o, p, dq, dq_f32, dk, dv, dkv_f32,
+                               delta, blocks, stream);
+    }
     if (st != AF_OK || fp.rows == 0) return st;
     return launch_first_rows<D>(fp, stream);
+}
+
+// One-pass sequence (bwd_fused_kernel.cuh): zero the fp32 dQ' accumulator, delta, RoPE passes on K and Q into the
+// caches, the one-pass kernel (dK, dV, dQ' partials), then scale / rotate back / convert dQ.
+struct OnePassArgs {
+    const void* q;
+    af_strides stq;
+    void* qcache;
+    float* dq_acc;
+    size_t dq_acc_bytes;
+};
+af_status launch_bwd_onepass(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                             const CUtensorMap& tdo, const CUtensorMap& tkp, const CUtensorMap& tqp, const void* k,
+                             const af_strides& stkv, void* kcache, const void* o, const void* d_o, BwdParams p, void* dq,
+                             int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, const OnePassArgs& a,
+                             cudaStream_t stream) {
+    constexpr int D = 128;
+    using L = BwdFusedSmem<D>;
+    if (cudaMemsetAsync(a.dq_acc, 0, a.dq_acc_bytes, stream) != cudaSuccess) return AF_ERR_CUDA;
+    const long long rows = static_cast<long long>(sh->B) * sh->Hq * sh->S;
+    const long long threads = rows * (D / 8);
+    bwd_delta_kernel<D><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
+        static_cast<const uint4*>(o), static_cast<const uint4*>(d_o), delta, rows);
+    if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
+    af_status st;
+    if (p.R > 0) {
+        if ((st = launch_rope(k, stkv, kcache, sh->B, sh->Hkv, sh->S, D, p.R, p.table, 0, stream, true)) != AF_OK) return st;
+        if ((st = launch_rope(a.q, a.stq, a.qcache, sh->B, sh->Hq, sh->S, D, p.R, p.table, 0, stream, true)) != AF_OK) return st;
+    }
+    p.delta = delta;
+    p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32; p.store_x = 0;
+    p.dq_acc = a.dq_acc;
+    auto kern = attn_bwd_fused_kernel<D>;
+    static std::atomic<unsigned long long> configured{0};
+    if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
+    const unsigned tiles = static_cast<unsigned>((sh->S + 127) / 128);
+    dim3 grid(sh->B * sh->Hkv, tiles, 1);
+    st = p.R > 0 ? launch_kernel(kern, grid, dim3(512, 1, 1), L::BYTES, stream, true, tkp, tv, tqp, tdo, p)
+                 : launch_kernel(kern, grid, dim3(512, 1, 1), L::BYTES, stream, true, tk, tv, tq, tdo, p);
+    if (st != AF_OK) return st;
+    const long long fthreads = rows * (D / 4);
+    return launch_kernel(bwd_dq_finish_kernel<D>, dim3(static_cast<unsigned>((fthreads + 255) / 256), 1, 1), dim3(256, 1, 1), 0,
+                         stream, true, static_cast<const float*>(a.dq_acc), dq, dq_f32, p.table, sh->S, p.R, p.scale, rows);
 }
 
 template <int D>
@@ -460,6 +521,9 @@ size_t bwd_kcache_bytes(const af_shape* sh) {
 }
 size_t bwd_qcache_bytes(const af_shape* sh) {
     return static_cast<size_t>(sh->B) * sh->Hq * sh->S * sh->D * 2;
+}
+size_t bwd_dqacc_bytes(const af_shape* sh) {
+    return static_cast<size_t>(sh->B) * sh->Hq * sh->S * sh->D * sizeof(float);
 }
 
 }  // namespace
@@ -927,6 +991,11 @@ size_t attnfuse_bwd_workspace_bytes(const af_shape* shape) {
     return bwd_delta_bytes(shape) + bwd_kcache_bytes(shape) + bwd_qcache_bytes(shape);   // delta + rotated-K and -Q caches
 }
 
+size_t attnfuse_bwd_onepass_workspace_bytes(const af_shape* shape) {
+    if (!shape) return 0;
+    return attnfuse_bwd_workspace_bytes(shape) + bwd_dqacc_bytes(shape);   // ... + the fp32 accumulator of dQ'
+}
+
 }  // extern "C"
 
 namespace {
@@ -973,16 +1042,28 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     // rotated-K and rotated-Q caches: used when there is a rotation and the workspace has room behind delta
     CUtensorMap tkp, tqp;
     const size_t off_k = bwd_delta_bytes(shape), off_q = off_k + bwd_kcache_bytes(shape);
+    const size_t off_acc = off_q + bwd_qcache_bytes(shape);
+    // One-pass sequence: D = 128, dense, room for both caches and the fp32 dQ' accumulator, and not switched off.
+    // Left to itself (option value 1) the choice goes by the average number of kept key tiles per query tile: the
+    // one-pass kernel costs more per tile pair than the two roles of the two-kernel sequence together, but the dQ
+    // role pays a fixed set-up and epilogue per query tile, which dominates while rows are short (measured: ahead at
+    // 8.5 and 9.5 tiles per query tile, behind at 16.5).
+    const int mode = opt(AF_OPT_BWD_ONEPASS);
+    const double n_tiles = (shape->S + 127) / 128;
+    double avg_tiles = p.causal ? 0.5 * (n_tiles + 1) : n_tiles;
+    if (p.window >= 0) avg_tiles = std::min(avg_tiles, (p.causal ? 1.0 : 2.0) * p.window / 128.0 + 1.5);
+    const bool onepass = shape->D == 128 && !blocks && workspace_bytes >= off_acc + bwd_dqacc_bytes(shape) &&
+                         (mode >= 2 || (mode == 1 && avg_tiles <= 12.0));
     const bool have_k = p.R > 0 && workspace_bytes >= off_q;
-    const bool have_q = have_k && workspace_bytes >= off_q + bwd_qcache_bytes(shape);
+    const bool have_q = have_k && workspace_bytes >= off_acc;
     void* kc = static_cast<uint8_t*>(workspace) + off_k;
+    void* qc = static_cast<uint8_t*>(workspace) + off_q;
     if (have_k) {
         af_strides stk;
         resolve_strides(nullptr, shape->Hkv, shape->S, shape->D, &stk);
         if ((st = make_tmap(&tkp, kc, shape->B, shape->Hkv, shape->S, shape->D, stk, 128)) != AF_OK) return st;
     }
     if (have_q) {
-        void* qc = static_cast<uint8_t*>(workspace) + off_q;
         if ((st = make_tmap(&tqp, qc, shape->B, shape->Hq, shape->S, shape->D, stc, 128)) != AF_OK) return st;
     }
     // Under a causal mask (dense, not over block lists) the first query rows of every head are computed in fp32 by a
@@ -998,11 +1079,17 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     fp.qb = stq.b; fp.qh = stq.h; fp.qs = stq.s; fp.kb = stkv.b; fp.kh = stkv.h; fp.ks = stkv.s;
     fp.dq = dq; fp.dk = dk; fp.dv = dv;
     fp.dq_f32 = dq_dtype == AF_F32; fp.dkv_f32 = dkv_dtype == AF_F32;
+    OnePassArgs op = {};
+    op.q = q; op.stq = stq; op.qcache = qc;
+    op.dq_acc = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + off_acc);
+    op.dq_acc_bytes = bwd_dqacc_bytes(shape);
+    p.dq_acc = nullptr;
     return shape->D == 128
                ? launch_bwd<128>(shape, tq, tk, tv, tdo, have_k ? &tkp : nullptr, have_q ? &tqp : nullptr, k, stkv, kc, o,
-                                 d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream, fp)
+                                 d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream, fp,
+                                 onepass ? &op : nullptr)
                : launch_bwd<64>(shape, tq, tk, tv, tdo, have_k ? &tkp : nullptr, have_q ? &tqp : nullptr, k, stkv, kc, o,
-                                d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream, fp);
+                                d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream, fp, nullptr);
 }
 }  // namespace
 

@@ -38,15 +38,17 @@ template <int D>
 struct FirstRowsSmem {
     static constexpr int PANEL = kFirstHeads * kFirstRows;                   // 64 stacked query rows
     static constexpr int LDK = D + 1;                                        // padded row of K' and V (bank spread)
-    static constexpr int FLOATS = 2 * kFirstRows * LDK + 2 * kFirstRows * D + 3 * PANEL * D + 3 * PANEL * kFirstRows + PANEL;
+    static constexpr int FLOATS = 2 * kFirstRows * LDK + 2 * kFirstRows * D + 3 * PANEL * D + 3 * PANEL * kFirstRows + PANEL +
+                                  kFirstRows * D;   // ... + {cos, sin} of the first positions, [kFirstRows][R/2] float2
     static constexpr int BYTES = FLOATS * 4;
 };
 
-// y = R(pos)^(sign) x for one row held in shared memory (in place): columns d < R/2 pair with d + R/2
+// y = R(pos)^(sign) x for one row held in shared memory (in place): columns d < R/2 pair with d + R/2.
+// table: the {cos, sin} rows of the first positions, staged in shared memory.
 __device__ __forceinline__ void first_rows_rotate(float* row, int R, const float2* table, int pos, float sign, int lane) {
     const int half = R >> 1;
     for (int i = lane; i < half; i += 32) {
-        const float2 cs = __ldg(table + static_cast<size_t>(pos) * half + i);
+        const float2 cs = table[pos * half + i];
         const float a = row[i], b = row[i + half], s = cs.y * sign;
         row[i] = a * cs.x - b * s;
         row[i + half] = b * cs.x + a * s;
@@ -69,6 +71,7 @@ __global__ void __launch_bounds__(256) bwd_first_rows_kernel(const FirstRowsPara
     float* dPs = Ps + PANEL * NR;         // [PANEL][NR] dO . v
     float* dSs = dPs + PANEL * NR;        // [PANEL][NR]
     float* dl = dSs + PANEL * NR;         // [PANEL] delta
+    float2* cs = reinterpret_cast<float2*>(dl + PANEL);   // [NR][R/2] {cos, sin} of positions 0 .. NR - 1
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int b = blockIdx.x / p.Hkv, hk = blockIdx.x % p.Hkv;
@@ -77,35 +80,77 @@ __global__ void __launch_bounds__(256) bwd_first_rows_kernel(const FirstRowsPara
     const __nv_bfloat16* vbase = p.v + b * p.kb + hk * p.kh;
 
     grid_dep_launch();
-    // keys and values of the first rows; gradients start at zero
+    // Every global read below is a 16-byte load issued in a batch before its first use: with one CTA per
+    // (batch, kv head) the kernel is a chain of memory latencies, not of arithmetic.
+    // {cos, sin} of the first positions (the table rows of positions 0 .. rows - 1 are contiguous)
+    if (p.R > 0) {
+        const int n4 = rows * (p.R >> 1) / 2;   // float4 = two {cos, sin} pairs; R / 2 is a multiple of 8
+        for (int idx = tid; idx < n4; idx += 256)
+            reinterpret_cast<float4*>(cs)[idx] = __ldg(reinterpret_cast<const float4*>(p.table) + idx);
+    }
+    // keys and values of the first rows (8 bf16 per load); gradients start at zero
+    static_assert(NR * D / 8 == 256 || NR * D / 8 == 128, "one 16-byte chunk of K and of V per thread");
+    if (tid < NR * D / 8) {
+        const int j = tid / (D / 8), d = (tid % (D / 8)) * 8;
+        uint4 kw = make_uint4(0u, 0u, 0u, 0u), vw = kw;
+        if (j < rows) {
+            kw = __ldg(reinterpret_cast<const uint4*>(kbase + j * p.ks + d));
+            vw = __ldg(reinterpret_cast<const uint4*>(vbase + j * p.ks + d));
+        }
+        const uint32_t ka[4] = {kw.x, kw.y, kw.z, kw.w}, va[4] = {vw.x, vw.y, vw.z, vw.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            Kp[j * LDK + d + 2 * u] = bf16lo_to_f32(ka[u]);
+            Kp[j * LDK + d + 2 * u + 1] = bf16hi_to_f32(ka[u]);
+            Vs[j * LDK + d + 2 * u] = bf16lo_to_f32(va[u]);
+            Vs[j * LDK + d + 2 * u + 1] = bf16hi_to_f32(va[u]);
+        }
+    }
     for (int idx = tid; idx < NR * D; idx += 256) {
-        const int j = idx / D, d = idx - j * D;
-        const bool in = j < rows;
-        Kp[j * LDK + d] = in ? __bfloat162float(kbase[j * p.ks + d]) : 0.f;
-        Vs[j * LDK + d] = in ? __bfloat162float(vbase[j * p.ks + d]) : 0.f;
         dKp[idx] = 0.f;
         dVs[idx] = 0.f;
     }
     __syncthreads();
     if (p.R > 0)
-        for (int j = warp; j < rows; j += 8) first_rows_rotate(Kp + j * LDK, p.R, p.table, j, 1.f, lane);
+        for (int j = warp; j < rows; j += 8) first_rows_rotate(Kp + j * LDK, p.R, cs, j, 1.f, lane);
     __syncthreads();
 
     for (int h0 = 0; h0 < p.group; h0 += kFirstHeads) {
         const int nh = min(kFirstHeads, p.group - h0);
         const int prow = nh * NR;          // panel rows in use: r = hh * NR + i
         // 1. queries (rotated) and upstream gradients of the panel
-        for (int idx = tid; idx < PANEL * D; idx += 256) {
-            const int r = idx / D, d = idx - r * D, hh = r / NR, i = r - hh * NR;
-            const bool in = hh < nh && i < rows;
-            const int h = hk * p.group + h0 + hh;
-            Qp[idx] = in ? __bfloat162float(p.q[b * p.qb + h * p.qh + i * p.qs + d]) : 0.f;
-            dOs[idx] = in ? __bfloat162float(p.d_o[((static_cast<size_t>(b) * p.Hq + h) * p.S + i) * D + d]) : 0.f;
+        {
+            constexpr int CH = PANEL * D / 8 / 256;   // 16-byte chunks per thread and array
+            uint4 qw[CH], gw[CH];
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const int idx = (tid + c * 256) * 8;
+                const int r = idx / D, d = idx - r * D, hh = r / NR, i = r - hh * NR;
+                const int h = hk * p.group + h0 + hh;
+                qw[c] = make_uint4(0u, 0u, 0u, 0u);
+                gw[c] = qw[c];
+                if (hh < nh && i < rows) {
+                    qw[c] = __ldg(reinterpret_cast<const uint4*>(p.q + b * p.qb + h * p.qh + i * p.qs + d));
+                    gw[c] = __ldg(reinterpret_cast<const uint4*>(p.d_o + ((static_cast<size_t>(b) * p.Hq + h) * p.S + i) * D + d));
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const int idx = (tid + c * 256) * 8;
+                const uint32_t qa[4] = {qw[c].x, qw[c].y, qw[c].z, qw[c].w}, ga[4] = {gw[c].x, gw[c].y, gw[c].z, gw[c].w};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    Qp[idx + 2 * u] = bf16lo_to_f32(qa[u]);
+                    Qp[idx + 2 * u + 1] = bf16hi_to_f32(qa[u]);
+                    dOs[idx + 2 * u] = bf16lo_to_f32(ga[u]);
+                    dOs[idx + 2 * u + 1] = bf16hi_to_f32(ga[u]);
+                }
+            }
         }
         __syncthreads();
         if (p.R > 0)
             for (int r = warp; r < prow; r += 8)
-                if (r % NR < rows) first_rows_rotate(Qp + r * D, p.R, p.table, r % NR, 1.f, lane);
+                if (r % NR < rows) first_rows_rotate(Qp + r * D, p.R, cs, r % NR, 1.f, lane);
         __syncthreads();
         // 2. scores s_rj = c <q'_r, k'_j> + slope (j - i) for the kept pairs (j <= i, i - j <= window), and dP_rj = <dO_r, v_j>
         for (int idx = tid; idx < PANEL * NR; idx += 256) {
@@ -177,36 +222,70 @@ __global__ void __launch_bounds__(256) bwd_first_rows_kernel(const FirstRowsPara
         // 7. dQ_r = R(i)^T dQ'_r, written over the zeros the dQ kernel left in these rows
         if (p.R > 0)
             for (int r = warp; r < prow; r += 8)
-                if (r % NR < rows) first_rows_rotate(dQp + r * D, p.R, p.table, r % NR, -1.f, lane);
+                if (r % NR < rows) first_rows_rotate(dQp + r * D, p.R, cs, r % NR, -1.f, lane);
         __syncthreads();
         grid_dep_wait();   // (first use of an output: the MMA kernels before this one in the stream are complete)
-        for (int idx = tid; idx < PANEL * D; idx += 256) {
+        for (int idx = tid * 4; idx < PANEL * D; idx += 256 * 4) {
             const int r = idx / D, d = idx - r * D, hh = r / NR, i = r - hh * NR;
             if (hh < nh && i < rows) {
                 const size_t off = ((static_cast<size_t>(b) * p.Hq + hk * p.group + h0 + hh) * p.S + i) * D + d;
-                if (p.dq_f32) static_cast<float*>(p.dq)[off] = dQp[idx];
-                else static_cast<__nv_bfloat16*>(p.dq)[off] = __float2bfloat16_rn(dQp[idx]);
+                const float4 y = *reinterpret_cast<const float4*>(dQp + idx);
+                if (p.dq_f32) *reinterpret_cast<float4*>(static_cast<float*>(p.dq) + off) = y;
+                else *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.dq) + off) = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
             }
         }
         __syncthreads();
     }
     // dK_j = R(j)^T dK'_j; both gradients are added to what the dK/dV kernel wrote for the later query rows
     if (p.R > 0)
-        for (int j = warp; j < rows; j += 8) first_rows_rotate(dKp + j * D, p.R, p.table, j, -1.f, lane);
+        for (int j = warp; j < rows; j += 8) first_rows_rotate(dKp + j * D, p.R, cs, j, -1.f, lane);
     __syncthreads();
     grid_dep_wait();
-    for (int idx = tid; idx < NR * D; idx += 256) {
-        const int j = idx / D, d = idx - j * D;
-        if (j < rows) {
-            const size_t off = ((static_cast<size_t>(b) * p.Hkv + hk) * p.S + j) * D + d;
-            if (p.dkv_f32) {
-                static_cast<float*>(p.dk)[off] += dKp[idx];
-                static_cast<float*>(p.dv)[off] += dVs[idx];
-            } else {
-                __nv_bfloat16* dk = static_cast<__nv_bfloat16*>(p.dk);
-                __nv_bfloat16* dv = static_cast<__nv_bfloat16*>(p.dv);
-                dk[off] = __float2bfloat16_rn(__bfloat162float(dk[off]) + dKp[idx]);
-                dv[off] = __float2bfloat16_rn(__bfloat162float(dv[off]) + dVs[idx]);
+    // four columns per thread and pass; both passes' loads are issued before the first add
+    constexpr int PASSES = NR * D / 4 / 256;
+    const size_t out_base = (static_cast<size_t>(b) * p.Hkv + hk) * p.S * D;   // rows j of this kv head are contiguous
+    if (p.dkv_f32) {
+        float4 ok[PASSES], ov[PASSES];
+#pragma unroll
+        for (int c = 0; c < PASSES; ++c) {
+            const int idx = (tid + c * 256) * 4;
+            if (idx / D < rows) {
+                ok[c] = *reinterpret_cast<const float4*>(static_cast<float*>(p.dk) + out_base + idx);
+                ov[c] = *reinterpret_cast<const float4*>(static_cast<float*>(p.dv) + out_base + idx);
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < PASSES; ++c) {
+            const int idx = (tid + c * 256) * 4;
+            if (idx / D < rows) {
+                const float4 a = *reinterpret_cast<const float4*>(dKp + idx), g = *reinterpret_cast<const float4*>(dVs + idx);
+                *reinterpret_cast<float4*>(static_cast<float*>(p.dk) + out_base + idx) =
+                    make_float4(ok[c].x + a.x, ok[c].y + a.y, ok[c].z + a.z, ok[c].w + a.w);
+                *reinterpret_cast<float4*>(static_cast<float*>(p.dv) + out_base + idx) =
+                    make_float4(ov[c].x + g.x, ov[c].y + g.y, ov[c].z + g.z, ov[c].w + g.w);
+            }
+        }
+    } else {
+        uint2 ok[PASSES], ov[PASSES];
+#pragma unroll
+        for (int c = 0; c < PASSES; ++c) {
+            const int idx = (tid + c * 256) * 4;
+            if (idx / D < rows) {
+                ok[c] = *reinterpret_cast<const uint2*>(static_cast<__nv_bfloat16*>(p.dk) + out_base + idx);
+                ov[c] = *reinterpret_cast<const uint2*>(static_cast<__nv_bfloat16*>(p.dv) + out_base + idx);
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < PASSES; ++c) {
+            const int idx = (tid + c * 256) * 4;
+            if (idx / D < rows) {
+                const float4 a = *reinterpret_cast<const float4*>(dKp + idx), g = *reinterpret_cast<const float4*>(dVs + idx);
+                *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.dk) + out_base + idx) =
+                    make_uint2(pack_bf16x2(bf16lo_to_f32(ok[c].x) + a.x, bf16hi_to_f32(ok[c].x) + a.y),
+                               pack_bf16x2(bf16lo_to_f32(ok[c].y) + a.z, bf16hi_to_f32(ok[c].y) + a.w));
+                *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(p.dv) + out_base + idx) =
+                    make_uint2(pack_bf16x2(bf16lo_to_f32(ov[c].x) + g.x, bf16hi_to_f32(ov[c].x) + g.y),
+                               pack_bf16x2(bf16lo_to_f32(ov[c].y) + g.z, bf16hi_to_f32(ov[c].y) + g.w));
             }
         }
     }

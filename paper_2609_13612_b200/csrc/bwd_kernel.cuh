@@ -44,6 +44,7 @@ struct BwdParams {
     const int* bs_idx;
     const int* bs_order;   // optional launch order of the stationary blocks (longest lists first), or nullptr
     int skip_rows;         // query rows i < skip_rows are left to bwd_first_rows_kernel (0: none)
+    float* dq_acc;         // one-pass kernel only: fp32 accumulator of dQ' [B, Hq, S, D], zero on entry
 };
 
 // delta[row] = <dO[row], O[row]>; one 16-byte chunk per thread, D/8 threads per row.

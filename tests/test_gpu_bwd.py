@@ -56,13 +56,24 @@ def test_backward_zero_upstream_gradient_and_determinism():
     t = synth.draw_all(w)
     dev = {k: pu.to_dev(v) for k, v in t.items()}
     o, lse = pu.gpu_fwd(w, dev)
-    a = pu.gpu_bwd(w, dev, o, lse)
-    b = pu.gpu_bwd(w, dev, o, lse)
+    # two-kernel sequence: every output is bit-reproducible
+    with af.option(af.OPT_BWD_ONEPASS, 0):
+        a = pu.gpu_bwd(w, dev, o, lse)
+        b = pu.gpu_bwd(w, dev, o, lse)
     for x, y in zip(a, b):
         assert torch.equal(x, y)
+    # one-pass sequence (the default here: D = 128, full workspace): dK and dV are reproducible, the fp32
+    # reductions of dQ in global memory may land in another order
+    c = pu.gpu_bwd(w, dev, o, lse)
+    d = pu.gpu_bwd(w, dev, o, lse)
+    assert torch.equal(c[1], d[1]) and torch.equal(c[2], d[2])
+    assert (c[0].float() - d[0].float()).abs().max().item() <= 2.0 ** -7 * c[0].float().abs().max().item()
     dev["do"] = torch.zeros_like(dev["do"])
     for g in pu.gpu_bwd(w, dev, o, lse):
         assert not g.any()
+    with af.option(af.OPT_BWD_ONEPASS, 0):
+        for g in pu.gpu_bwd(w, dev, o, lse):
+            assert not g.any()
 
 
 def test_backward_strided_inputs():
@@ -75,6 +86,11 @@ def test_backward_strided_inputs():
     for k in ("q", "k", "v"):
         perm[k] = dev[k].permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
     got = pu.gpu_bwd(w, perm, o, lse)
+    assert torch.equal(ref[1], got[1]) and torch.equal(ref[2], got[2])
+    assert (ref[0].float() - got[0].float()).abs().max().item() <= 2.0 ** -7 * ref[0].float().abs().max().item()
+    with af.option(af.OPT_BWD_ONEPASS, 0):
+        ref = pu.gpu_bwd(w, dev, o, lse)
+        got = pu.gpu_bwd(w, perm, o, lse)
     for x, y in zip(ref, got):
         assert torch.equal(x, y)
 
@@ -110,9 +126,9 @@ def test_config5_training_shape_full():
 
 
 def test_backward_workspace_tiers_give_the_same_result():
-    """Three set-ups by workspace size: delta + K' cache + Q' cache (nothing rotated in the dK/dV loop),
-    delta + K' cache (the dQ kernel streams cached K'), delta alone (both kernels rotate on chip).
-    All match the oracle and agree with one another up to a few bf16 roundings of rotated rows."""
+    """Set-ups by workspace size: the one-pass sequence (both caches and the fp32 dQ accumulator), delta + K' cache +
+    Q' cache (nothing rotated in the dK/dV loop), delta + K' cache (the dQ kernel streams cached K'), delta alone
+    (both kernels rotate on chip).  All match the oracle and agree with one another up to a few bf16 roundings."""
     w = W("ws_tiers", 2, 4, 2, 515, 128, theta=5e5, backward=True, seed_id=224)
     t = synth.draw_all(w)
     dev = {k: pu.to_dev(v) for k, v in t.items()}
@@ -121,7 +137,12 @@ def test_backward_workspace_tiers_give_the_same_result():
     table = af.rope_table(rope, w.S)
     n_delta = (w.B * w.Hq * w.S * 4 + 255) // 256 * 256
     n_k = w.B * w.Hkv * w.S * w.D * 2
-    full = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale)
+    n_q = w.B * w.Hq * w.S * w.D * 2
+    assert af.bwd_workspace_bytes(w.B, w.Hq, w.Hkv, w.S, w.D, onepass=False) == n_delta + n_k + n_q
+    assert af.bwd_workspace_bytes(w.B, w.Hq, w.Hkv, w.S, w.D) == n_delta + n_k + 3 * n_q
+    onepass = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale)
+    full_ws = torch.empty(n_delta + n_k + n_q, dtype=torch.uint8, device="cuda")
+    full = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale, workspace=full_ws)
     mid_ws = torch.empty(n_delta + n_k, dtype=torch.uint8, device="cuda")
     mid = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale, workspace=mid_ws)
     small_ws = torch.empty(n_delta, dtype=torch.uint8, device="cuda")
@@ -132,11 +153,11 @@ def test_backward_workspace_tiers_give_the_same_result():
     assert torch.equal(mid[1], small[1]) and torch.equal(mid[2], small[2])
     # elsewhere cos/sin are walked over different runs of rows (or read from the table), so a few bf16
     # roundings of rotated rows may differ by one ulp
-    for a, b in ((full, mid), (mid, small)):
+    for a, b in ((onepass, full), (full, mid), (mid, small)):
         for x, y in zip(a, b):
             assert (x.float() - y.float()).abs().max().item() <= 1e-2
     want = oracle.run_workload(w, t, backward=True)
-    for res in (full, mid, small):
+    for res in (onepass, full, mid, small):
         for name, got, ref in zip(("dQ", "dK", "dV"), res, want):
             pu.assert_close("%s %s" % (w.name, name), pu.to_np(got), ref)
 
@@ -198,3 +219,18 @@ def test_partial_rotary_at_scale_sampled_units():
     torch.cuda.synchronize()
     assert af.device_status()[0] == 0
     _check_units(w, ((1, 1),), t, o, lse, grads, "partial rotary")
+
+
+@pytest.mark.parametrize("mode", [0, 2], ids=["two_kernel", "one_pass"])
+def test_both_backward_sequences_on_long_rows_sampled_units(mode):
+    """S = 4096 with GQA (16.5 kept key tiles per query tile on average: left to itself the library takes the
+    two-kernel sequence here) with either sequence forced, full one-pass workspace in both runs."""
+    w = W("long_rows_%d" % mode, 1, 8, 2, 4096, 128, theta=5e5, backward=True, seed_id=233)
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    o, lse = pu.gpu_fwd(w, dev)
+    with af.option(af.OPT_BWD_ONEPASS, mode):
+        grads = pu.gpu_bwd(w, dev, o, lse)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    _check_units(w, ((0, 1),), t, o, lse, grads, "long rows")

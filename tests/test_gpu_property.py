@@ -6,7 +6,7 @@ ulp of the exact value (parity_util.assert_close_scaled says why).
 
 The kernels branch on many of these parameters - ragged last tiles, head pairs on even groups and row pairs on
 odd ones, the rotary widths with a fast path against the generic one, window edges that fall on tile borders,
-three workspace set-ups of the backward - and the hand-picked cases elsewhere cannot cover their product."""
+workspace set-ups of the backward - and the hand-picked cases elsewhere cannot cover their product."""
 import numpy as np
 import pytest
 import torch
@@ -61,18 +61,20 @@ def test_forward_examples(w, f32_out, hybrid):
 
 
 @settings(max_examples=30, **COMMON)
-@given(w=workloads(backward=True), tier=st.integers(0, 2), dq_f32=st.booleans())
+@given(w=workloads(backward=True), tier=st.integers(0, 3), dq_f32=st.booleans())
 def test_backward_examples(w, tier, dq_f32):
     t = synth.draw_all(w)
     dev = {k: pu.to_dev(v) for k, v in t.items()}
     rope, mask = pu.specs(w)
     table = af.rope_table(rope, w.S) if w.R > 0 else None
     o, lse = af.fwd(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale)
-    # workspace set-ups: delta alone / + rotated-K cache / + rotated-Q cache as well
+    # workspace set-ups: delta alone / + rotated-K cache / + rotated-Q cache as well / + dQ accumulator
     n_delta = (w.B * w.Hq * w.S * 4 + 255) // 256 * 256
     n_k = w.B * w.Hkv * w.S * w.D * 2
     n_q = w.B * w.Hq * w.S * w.D * 2
-    ws = torch.empty(n_delta + (n_k if tier >= 1 else 0) + (n_q if tier >= 2 else 0), dtype=torch.uint8, device="cuda")
+    # (tier 3: room for the fp32 dQ accumulator too - the one-pass sequence where it applies, D = 128)
+    ws = torch.empty(n_delta + (n_k if tier >= 1 else 0) + (n_q if tier >= 2 else 0) + (2 * n_q if tier >= 3 else 0),
+                     dtype=torch.uint8, device="cuda")
     dq, dk, dv = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale,
                         dq_dtype=torch.float32 if dq_f32 else torch.bfloat16, dkv_dtype=torch.float32, workspace=ws)
     torch.cuda.synchronize()
