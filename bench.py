@@ -166,7 +166,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--extras", type=int, default=1, help="also time configs 3-5, the separate-RoPE arm and the sweep")
     ap.add_argument("--cpu-baseline", type=int, default=1)
-    ap.add_argument("--profile", default="", choices=["", "fwd", "hybrid", "bwd", "rope", "decode"],
+    ap.add_argument("--profile", default="", choices=["", "fwd", "hybrid", "bwd", "bwd2", "rope", "decode", "fwd_c3", "fwd_d64", "blocks"],
                     help="run only a few launches of one path (for ncu captures) and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -259,19 +259,31 @@ def main():
         return
     if args.profile:
         # a handful of launches of one path on its configuration, nothing else: the target of ncu captures
-        wl = {"fwd": synth.CONFIGS[1], "hybrid": synth.CONFIGS[1], "bwd": synth.CONFIGS[4],
-              "rope": synth.CONFIGS[3]}[args.profile]
+        wl = {"fwd": synth.CONFIGS[1], "hybrid": synth.CONFIGS[1], "bwd": synth.CONFIGS[4], "bwd2": synth.CONFIGS[4],
+              "rope": synth.CONFIGS[3], "fwd_c3": synth.CONFIGS[2],
+              "fwd_d64": synth.Workload("gpt2_small_geometry_d64", 4, 12, 12, 4096, 64, theta=1.0e4, seed_id=51),
+              "blocks": synth.Workload("bigbird_d64_n4096", 4, 12, 12, 4096, 64, theta=1.0e4, causal=False, seed_id=53)}[args.profile]
         r, m, tb = specs(wl)
         t = {k: to_dev(v) for k, v in synth.draw_all(wl).items()}
+        if args.profile == "blocks":   # the BigBird-like mask of the block-sparse extra (12 % of the 32 x 32 blocks)
+            rng_ = np.random.Generator(np.random.PCG64(np.random.SeedSequence([20260913, 901])))
+            act = np.eye(32, dtype=bool)
+            act[:, 0] = True
+            act[0, :] = True
+            act[np.arange(32), rng_.integers(0, 32, size=32)] = True
+            bmask = af.BlockMask(act, device=dev)
         for _ in range(3):
             if args.profile == "rope":
                 af.rope(t["q"], r, tb)
             elif args.profile == "hybrid":
                 af.fwd_hybrid(t["q"], t["k"], t["v"], r, tb, m, wl.scale)
+            elif args.profile == "blocks":
+                af.fwd_blocks(t["q"], t["k"], t["v"], r, tb, m, wl.scale, bmask)
             else:
                 o_, l_ = af.fwd(t["q"], t["k"], t["v"], r, tb, m, wl.scale)
-                if args.profile == "bwd":
-                    af.bwd(t["q"], t["k"], t["v"], o_, l_, t["do"], r, tb, m, wl.scale)
+                if args.profile in ("bwd", "bwd2"):   # bwd: the sequence the library picks (one-pass here); bwd2: two kernels
+                    with af.option(af.OPT_BWD_ONEPASS, 1 if args.profile == "bwd" else 0):
+                        af.bwd(t["q"], t["k"], t["v"], o_, l_, t["do"], r, tb, m, wl.scale)
         torch.cuda.synchronize()
         print(json.dumps({"profile": args.profile, "workload": wl.name, "device_status": af.device_status()[0]}))
         return
@@ -411,8 +423,7 @@ def main():
         r5, m5, t5 = specs(w5)
         s5 = make_sets(w5, n_sets_for(w5))
         o5, l5 = af.fwd(s5[0]["q"], s5[0]["k"], s5[0]["v"], r5, t5, m5, w5.scale)
-        ws = torch.empty(af.lib().attnfuse_bwd_workspace_bytes(
-            __import__("ctypes").byref(binding._Shape(w5.B, w5.Hq, w5.Hkv, w5.S, w5.D))), dtype=torch.uint8, device=dev)
+        ws = torch.empty(af.bwd_workspace_bytes(w5.B, w5.Hq, w5.Hkv, w5.S, w5.D), dtype=torch.uint8, device=dev)
 
         def fb(i):
             s = s5[i % len(s5)]
@@ -433,12 +444,17 @@ def main():
         t_fb, _, _ = timed(fb, k_ex, w_ex)
         t_fbh, _, _ = timed(fb_hybrid, k_ex, w_ex)
         t_b, _, _ = timed(bonly, k_ex, w_ex)
+        with af.option(af.OPT_BWD_ONEPASS, 0):   # the two-kernel sequence (bit-reproducible dQ) on the same inputs
+            t_b2, _, _ = timed(bonly, k_ex, w_ex)
         ex[w5.name] = {"fwd_bwd_ms": t_fb / k_ex,
                        "fwd_bwd_tflops": (w5.fwd_flops() + w5.bwd_flops()) / (t_fb / k_ex) / 1e9,
                        "hybrid_fwd_bwd_ms": t_fbh / k_ex,
                        "hybrid_fwd_bwd_tflops": (w5.fwd_flops() + w5.bwd_flops()) / (t_fbh / k_ex) / 1e9,
                        "bwd_ms": t_b / k_ex, "bwd_tflops": w5.bwd_flops() / (t_b / k_ex) / 1e9,
-                       "bwd_pct_of_measured_peak": 100 * w5.bwd_flops() / (t_b / k_ex) / 1e9 / peaks["bf16_tflops"]}
+                       "bwd_pct_of_measured_peak": 100 * w5.bwd_flops() / (t_b / k_ex) / 1e9 / peaks["bf16_tflops"],
+                       "bwd_sequence": "one-pass (dK, dV and dQ shares from one kernel per key tile)",
+                       "bwd_two_kernel_sequence_ms": t_b2 / k_ex,
+                       "bwd_two_kernel_sequence_tflops": w5.bwd_flops() / (t_b2 / k_ex) / 1e9}
         del s5
         torch.cuda.empty_cache()
 
@@ -446,8 +462,7 @@ def main():
             r, m, tb = specs(wl)
             ss = make_sets(wl, min(2, n_sets_for(wl)))
             o_, l_ = af.fwd(ss[0]["q"], ss[0]["k"], ss[0]["v"], r, tb, m, wl.scale)
-            wsb = torch.empty(af.lib().attnfuse_bwd_workspace_bytes(
-                __import__("ctypes").byref(binding._Shape(wl.B, wl.Hq, wl.Hkv, wl.S, wl.D))), dtype=torch.uint8, device=dev)
+            wsb = torch.empty(af.bwd_workspace_bytes(wl.B, wl.Hq, wl.Hkv, wl.S, wl.D), dtype=torch.uint8, device=dev)
             t, _, _ = timed(lambda i: af.bwd(ss[i % len(ss)]["q"], ss[i % len(ss)]["k"], ss[i % len(ss)]["v"], o_, l_,
                                              ss[i % len(ss)]["do"], r, tb, m, wl.scale, workspace=wsb), k_ex, w_ex)
             return t / k_ex
@@ -525,8 +540,7 @@ def main():
         t_df, _, _ = timed(lambda i: af.fwd(sb[i % 2]["q"], sb[i % 2]["k"], sb[i % 2]["v"], rb_, tbb, mb_, wb.scale, out=ob,
                                             lse=lb), k_ex, w_ex)
         af.fwd_blocks(sb[0]["q"], sb[0]["k"], sb[0]["v"], rb_, tbb, mb_, wb.scale, bmask, out=ob, lse=lb)
-        wsbb = torch.empty(af.lib().attnfuse_bwd_workspace_bytes(
-            __import__("ctypes").byref(binding._Shape(wb.B, wb.Hq, wb.Hkv, wb.S, wb.D))), dtype=torch.uint8, device=dev)
+        wsbb = torch.empty(af.bwd_workspace_bytes(wb.B, wb.Hq, wb.Hkv, wb.S, wb.D), dtype=torch.uint8, device=dev)
         t_bb, _, _ = timed(lambda i: af.bwd(sb[0]["q"], sb[0]["k"], sb[0]["v"], ob, lb, sb[0]["do"], rb_, tbb, mb_, wb.scale,
                                             workspace=wsbb, blocks=bmask), k_ex, w_ex)
         nnz_b = int(act.sum()) * 128 * 128
@@ -628,8 +642,7 @@ def main():
         rt, mt, tt_ = specs(wt)
         st_ = make_sets(wt, 1)[0]
         ot, lt = af.fwd(st_["q"], st_["k"], st_["v"], rt, tt_, mt, wt.scale)
-        wst = torch.empty(af.lib().attnfuse_bwd_workspace_bytes(
-            __import__("ctypes").byref(binding._Shape(wt.B, wt.Hq, wt.Hkv, wt.S, wt.D))), dtype=torch.uint8, device=dev)
+        wst = torch.empty(af.bwd_workspace_bytes(wt.B, wt.Hq, wt.Hkv, wt.S, wt.D), dtype=torch.uint8, device=dev)
         ex["host_us_per_call"] = {
             "fwd": host_us(lambda i: af.fwd(st_["q"], st_["k"], st_["v"], rt, tt_, mt, wt.scale, out=ot, lse=lt)),
             "bwd": host_us(lambda i: af.bwd(st_["q"], st_["k"], st_["v"], ot, lt, st_["do"], rt, tt_, mt, wt.scale, workspace=wst)),

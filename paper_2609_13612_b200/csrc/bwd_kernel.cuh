@@ -104,7 +104,9 @@ __device__ __forceinline__ bool wg_all(bool v) { return bar_all(v, 3, 256); }
 // Epilogue helper: the 256 threads of the two gradient warpgroups move a [128 x D] fp32 accumulator
 // from TMEM (thread gtid reads lane gtid % 128, column half gtid / 128) through shared memory to
 // global memory, scaling it and, when R > 0, applying the transpose rotation for positions row0..
-// (gradients w.r.t. rotated rows are rotated back).  Global writes are coalesced along D.
+// (gradients w.r.t. rotated rows are rotated back).  Global writes are coalesced along D.  (Writing each
+// thread's TMEM row straight to global memory - no staging, no barriers, cos/sin read per row - measured
+// slower: a warp's store then touches 32 rows, and the store rate is what bounds this epilogue.)
 template <int D>
 __device__ __forceinline__ void store_acc_rotated(uint32_t t_acc, float* stg, int gtid, float mul, int R,
                                                   const float2* table, int row0, int S, void* out, size_t out_row0,
