@@ -203,10 +203,19 @@ af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* 
  * variant is bound by the S x S bias traffic, not by the tensor pipe.
  * relu_attention (the paper names the combinator only; reading): P_ij = max(s_ij, 0) / n_i over the kept
  * pairs, n_i = number of kept pairs of row i (pairs that the mask keeps and whose bias is finite), in place
- * of the softmax; there is no row statistic, so lse must be NULL; not available over block lists.
- * Forward only: attnfuse_bwd covers rope, causal, sliding_window, full, block_sparse, alibi and softmax.
+ * of the softmax; there is no log-sum-exp: with relu_attention `lse` (nullable) receives n_i as a float, the
+ * row statistic that attnfuse_bwd_variant needs; not available over block lists.
  * Errors as for attnfuse_fwd; AF_ERR_SHAPE for bias extents other than 1 / B / Hq, AF_ERR_SPEC for an
- * unknown normaliser, for lse with relu_attention, and for relu_attention with blocks. */
+ * unknown normaliser and for relu_attention with blocks.
+ *
+ * attnfuse_bwd_variant: the backward of the same description.  Arguments as attnfuse_bwd; `lse` is what the
+ * forward of the SAME variant wrote (L, or n_i under relu_attention).  No gradient flows into the bias.  With
+ * relu_attention dS_ij = [s_ij > 0] dP_ij / n_i.  A variant without bias and with the softmax normaliser takes
+ * the sequences of attnfuse_bwd / attnfuse_bwd_blocks.  With a bias or relu_attention: dense only (AF_ERR_SPEC
+ * with blocks), always the two-kernel sequence (deterministic), and with a rotation the workspace must hold
+ * delta and both rotated caches (attnfuse_bwd_workspace_bytes; AF_ERR_WORKSPACE otherwise); the first query
+ * rows get no fp32 treatment there (see attnfuse_bwd), so rows with a handful of keys carry the bf16 roundings
+ * of P and dS at full size. */
 typedef enum { AF_NORM_SOFTMAX = 0, AF_NORM_RELU = 1 } af_normaliser;
 typedef struct {
     af_rope rope;
@@ -217,6 +226,12 @@ typedef struct {
     af_normaliser normaliser;
     const af_blocks* blocks;     /* block_sparse lists or NULL (dense) */
 } af_variant;
+af_status attnfuse_bwd_variant(const af_shape* shape, const void* q, const void* k, const void* v,
+                               const void* o, const float* lse, const void* d_o,
+                               const af_strides* sq, const af_strides* skv, const af_variant* variant,
+                               int gqa_group, float softmax_scale,
+                               void* dq, af_dtype dq_dtype, void* dk, void* dv, af_dtype dkv_dtype,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
 af_status attnfuse_fwd_variant(const af_shape* shape, const void* q, const void* k, const void* v,
                                const af_strides* sq, const af_strides* skv, const af_variant* variant,
                                int gqa_group, float softmax_scale,

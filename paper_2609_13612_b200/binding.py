@@ -119,6 +119,9 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_bwd.restype = i
         L.attnfuse_bwd.argtypes = [P(_Shape), vp, vp, vp, vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp,
                                    P(_Mask), i, f, vp, i, vp, vp, i, vp, sz, vp]
+        L.attnfuse_bwd_variant.restype = i
+        L.attnfuse_bwd_variant.argtypes = [P(_Shape), vp, vp, vp, vp, vp, vp, P(_Strides), P(_Strides), P(_Variant), i, f,
+                                           vp, i, vp, vp, i, vp, sz, vp]
         L.attnfuse_fwd_blocks.restype = i
         L.attnfuse_fwd_blocks.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp, P(_Mask), i, f,
                                           P(_Blocks), vp, i, vp, vp]
@@ -278,8 +281,8 @@ def fwd_variant(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: Ro
                 blocks: Optional["BlockMask"] = None, out: Optional[torch.Tensor] = None,
                 out_dtype: torch.dtype = torch.bfloat16):
     """Forward of a composed variant (Section 3.1): `fwd` plus an optional additive bias (fp32 [1|B, 1|Hq, S, S]
-    on the device), the normaliser ("softmax" or "relu") and optional block lists.  Returns (o, lse); lse is
-    None for the ReLU normaliser."""
+    on the device), the normaliser ("softmax" or "relu") and optional block lists.  Returns (o, lse); for the ReLU
+    normaliser `lse` holds n_i, the number of kept pairs of each row (what `bwd_variant` needs)."""
     _need_cuda(q, k, v, table, out, bias)
     assert q.dtype == k.dtype == v.dtype == torch.bfloat16 and normaliser in ("softmax", "relu")
     B, Hq, S, D = q.shape
@@ -288,7 +291,7 @@ def fwd_variant(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: Ro
     if out is None:
         out = torch.empty((B, Hq, S, D), dtype=out_dtype, device=q.device)
     relu = normaliser == "relu"
-    lse = None if relu else torch.empty((B, Hq, S), dtype=torch.float32, device=q.device)
+    lse = torch.empty((B, Hq, S), dtype=torch.float32, device=q.device)
     if bias is not None:
         assert bias.dtype == torch.float32 and bias.is_contiguous() and bias.dim() == 4 and bias.shape[2:] == (S, S)
     sh = _Shape(B, Hq, Hkv, S, D)
@@ -304,6 +307,41 @@ def fwd_variant(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: Ro
                                       out.data_ptr(), AF_F32 if out.dtype == torch.float32 else AF_BF16,
                                       lse.data_ptr() if lse is not None else None, _stream()))
     return out, lse
+
+
+def bwd_variant(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softmax_scale: float,
+                bias: Optional[torch.Tensor] = None, normaliser: str = "softmax", blocks: Optional["BlockMask"] = None,
+                dq_dtype: torch.dtype = torch.bfloat16, dkv_dtype: torch.dtype = torch.float32, workspace=None):
+    """Backward of a composed variant; `lse` is what `fwd_variant` returned for the same variant.
+    Returns (dq, dk, dv)."""
+    _need_cuda(q, k, v, o, lse, d_o, table, workspace, bias)
+    assert normaliser in ("softmax", "relu")
+    B, Hq, S, D = q.shape
+    Hkv = k.shape[1]
+    assert o.is_contiguous() and d_o.is_contiguous() and lse.is_contiguous()
+    assert o.dtype == d_o.dtype == torch.bfloat16 and lse.dtype == torch.float32
+    if bias is not None:
+        assert bias.dtype == torch.float32 and bias.is_contiguous() and bias.dim() == 4 and bias.shape[2:] == (S, S)
+    sh = _Shape(B, Hq, Hkv, S, D)
+    if workspace is None:
+        plain = bias is None and normaliser == "softmax" and blocks is None
+        workspace = torch.empty(bwd_workspace_bytes(B, Hq, Hkv, S, D, onepass=plain), dtype=torch.uint8, device=q.device)
+    dq = torch.empty((B, Hq, S, D), dtype=dq_dtype, device=q.device)
+    dk = torch.empty((B, Hkv, S, D), dtype=dkv_dtype, device=q.device)
+    dv = torch.empty((B, Hkv, S, D), dtype=dkv_dtype, device=q.device)
+    sq, skv = _strides(q), _strides(k)
+    bl = blocks.struct() if blocks is not None else None
+    var = _Variant(_Rope(rope_spec.theta, rope_spec.rotary_dim, rope_spec.pos_offset),
+                   table.data_ptr() if table is not None else None, _mask_struct(mask),
+                   bias.data_ptr() if bias is not None else None,
+                   bias.shape[0] if bias is not None else 1, bias.shape[1] if bias is not None else 1,
+                   1 if normaliser == "relu" else 0, ctypes.pointer(bl) if bl is not None else None)
+    code = lambda dt: AF_F32 if dt == torch.float32 else AF_BF16
+    _check(lib().attnfuse_bwd_variant(ctypes.byref(sh), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                      lse.data_ptr(), d_o.data_ptr(), ctypes.byref(sq), ctypes.byref(skv), ctypes.byref(var),
+                                      Hq // Hkv, float(softmax_scale), dq.data_ptr(), code(dq_dtype), dk.data_ptr(),
+                                      dv.data_ptr(), code(dkv_dtype), workspace.data_ptr(), workspace.numel(), _stream()))
+    return dq, dk, dv
 
 
 def fwd_hybrid(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor],

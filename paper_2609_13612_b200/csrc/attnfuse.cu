@@ -355,6 +355,17 @@ af_status launch_bwd_variant(const CUtensorMap& tx, const CUtensorMap& ty, const
                     : launch_bwd_variant_bs<D, DKV, ROT_X, ROT_A, false>(tx, ty, ta, tb, ts, p, grid, stream);
 }
 
+// Section 3.1 extras in the backward (additive_bias, relu_attention): the GEN instantiations, dense only.
+template <int D, bool DKV, bool ROT_X>
+af_status launch_bwd_gen(const CUtensorMap& tx, const CUtensorMap& ty, const CUtensorMap& ta, const CUtensorMap& tb,
+                         const CUtensorMap& ts, const BwdParams& p, dim3 grid, cudaStream_t stream) {
+    using L = BwdSmem<D>;
+    auto kern = attn_bwd_kernel<D, DKV, ROT_X, false, false, true>;
+    static std::atomic<unsigned long long> configured{0};
+    if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
+    return launch_kernel(kern, grid, dim3(512, 1, 1), L::BYTES, stream, true, tx, ty, ta, tb, ts, p);
+}
+
 // RoPE pass x [B, H, S, D] (strided) -> x_out (contiguous); R > 0.
 // dependent: launch as a programmatic dependent of the preceding kernel (only inside this library's own sequences).
 af_status launch_rope(const void* x_in, const af_strides& st, void* x_out, int B, int H, int S, int D, int R,
@@ -489,6 +500,21 @@ af_status launch_bwd_mma(const af_shape* sh, const CUtensorMap& tq, const CUtens
     constexpr int only = 0;
 #endif
     dim3 gkv(sh->B * sh->Hkv, tiles, 1), gq(sh->B * sh->Hq, tiles, 1);
+    if (p.bias || p.relu) {
+        // additive_bias / relu_attention: the both-caches set-up with rotation, the plain one without
+        if (p.R > 0) {
+            if (!tkp || !tqp) return AF_ERR_WORKSPACE;
+            if ((st = launch_rope(k, stkv, kcache, sh->B, sh->Hkv, sh->S, D, p.R, p.table, 0, stream, true)) != AF_OK) return st;
+            p.out1 = dq; p.out2 = nullptr; p.out_f32 = dq_f32; p.store_x = 1;
+            if ((st = launch_bwd_gen<D, false, true>(tq, tdo, *tkp, tv, *tqp, p, gq, stream)) != AF_OK) return st;
+            p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32; p.store_x = 0;
+            return launch_bwd_gen<D, true, false>(*tkp, tv, *tqp, tdo, tk, p, gkv, stream);
+        }
+        p.out1 = dq; p.out2 = nullptr; p.out_f32 = dq_f32; p.store_x = 0;
+        if ((st = launch_bwd_gen<D, false, false>(tq, tdo, tk, tv, tk, p, gq, stream)) != AF_OK) return st;
+        p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32; p.store_x = 0;
+        return launch_bwd_gen<D, true, false>(tk, tv, tq, tdo, tk, p, gkv, stream);
+    }
     if (p.R > 0 && tkp && tqp && only == 0) {
         // both caches: K' by the RoPE pass, Q' by the dQ kernel, no on-chip rotation in the dK/dV loop
         if ((st = launch_rope(k, stkv, kcache, sh->B, sh->Hkv, sh->S, D, p.R, p.table, 0, stream, true)) != AF_OK) return st;
@@ -660,7 +686,7 @@ af_status fwd_impl(const af_shape* shape, const void* q, const void* k, const vo
         if ((bias_B != 1 && bias_B != shape->B) || (bias_H != 1 && bias_H != shape->Hq)) return AF_ERR_SHAPE;
         if ((reinterpret_cast<uintptr_t>(bias) & 3u) != 0) return AF_ERR_ALIGN;
     }
-    if (relu && (lse || bs_row_ptr)) return AF_ERR_SPEC;   // no row statistic for the ReLU normaliser; not built over block lists
+    if (relu && bs_row_ptr) return AF_ERR_SPEC;   // the ReLU normaliser is not built over block lists
     af_strides stq, stkv;
     if ((st = resolve_strides(sq, shape->Hq, shape->S, shape->D, &stq)) != AF_OK) return st;
     if ((st = resolve_strides(skv, shape->Hkv, shape->S, shape->D, &stkv)) != AF_OK) return st;
@@ -1004,10 +1030,17 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
                    const float* lse, const void* d_o, const af_strides* sq, const af_strides* skv,
                    const af_rope* rope, const void* rope_table, const af_mask* mask, int gqa_group,
                    float softmax_scale, const af_blocks* blocks, void* dq, af_dtype dq_dtype, void* dk, void* dv,
-                   af_dtype dkv_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+                   af_dtype dkv_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                   const float* bias = nullptr, int bias_B = 1, int bias_H = 1, int relu = 0) {
     af_status st = check_common(shape, rope, rope_table, mask, gqa_group);
     if (st != AF_OK) return st;
     if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv) return AF_ERR_NULL;
+    const bool gen = bias != nullptr || relu != 0;
+    if (bias) {
+        if ((bias_B != 1 && bias_B != shape->B) || (bias_H != 1 && bias_H != shape->Hq)) return AF_ERR_SHAPE;
+        if ((reinterpret_cast<uintptr_t>(bias) & 3u) != 0) return AF_ERR_ALIGN;
+    }
+    if (gen && blocks) return AF_ERR_SPEC;   // the extras are not built over block lists
     if ((dq_dtype != AF_BF16 && dq_dtype != AF_F32) || (dkv_dtype != AF_BF16 && dkv_dtype != AF_F32))
         return AF_ERR_DTYPE;
     if (!workspace || workspace_bytes < bwd_delta_bytes(shape)) return AF_ERR_WORKSPACE;   // the cache is optional
@@ -1037,6 +1070,10 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     p.lse = lse;
     p.delta = nullptr; p.out1 = nullptr; p.out2 = nullptr; p.out_f32 = 0; p.store_x = 0;
     p.bs_ptr = nullptr; p.bs_idx = nullptr; p.bs_order = nullptr; p.skip_rows = 0;
+    p.bias = bias;
+    p.bias_sb = (bias && bias_B > 1) ? static_cast<long long>(bias_H) * shape->S * shape->S : 0;
+    p.bias_sh = (bias && bias_H > 1) ? static_cast<long long>(shape->S) * shape->S : 0;
+    p.relu = relu ? 1 : 0;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     float* delta = static_cast<float*>(workspace);
     // rotated-K and rotated-Q caches: used when there is a rotation and the workspace has room behind delta
@@ -1052,7 +1089,7 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     const double n_tiles = (shape->S + 127) / 128;
     double avg_tiles = p.causal ? 0.5 * (n_tiles + 1) : n_tiles;
     if (p.window >= 0) avg_tiles = std::min(avg_tiles, (p.causal ? 1.0 : 2.0) * p.window / 128.0 + 1.5);
-    const bool onepass = shape->D == 128 && !blocks && workspace_bytes >= off_acc + bwd_dqacc_bytes(shape) &&
+    const bool onepass = shape->D == 128 && !blocks && !gen && workspace_bytes >= off_acc + bwd_dqacc_bytes(shape) &&
                          (mode >= 2 || (mode == 1 && avg_tiles <= 12.0));
     const bool have_k = p.R > 0 && workspace_bytes >= off_q;
     const bool have_q = have_k && workspace_bytes >= off_acc;
@@ -1071,7 +1108,8 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     FirstRowsParams fp = {};
     fp.B = shape->B; fp.Hq = shape->Hq; fp.Hkv = shape->Hkv; fp.S = shape->S; fp.group = gqa_group;
     fp.R = p.R; fp.window = p.window;
-    fp.rows = (p.causal && !blocks) ? (shape->S < kFirstRows ? shape->S : kFirstRows) : 0;
+    // (not with additive_bias / relu_attention either: the fp32 kernel knows neither)
+    fp.rows = (p.causal && !blocks && !gen) ? (shape->S < kFirstRows ? shape->S : kFirstRows) : 0;
     fp.scale = softmax_scale;
     fp.slopes = p.slopes; fp.table = p.table;
     fp.q = static_cast<const __nv_bfloat16*>(q); fp.k = static_cast<const __nv_bfloat16*>(k);
@@ -1102,6 +1140,23 @@ af_status attnfuse_bwd(const af_shape* shape, const void* q, const void* k, cons
                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return bwd_impl(shape, q, k, v, o, lse, d_o, sq, skv, rope, rope_table, mask, gqa_group, softmax_scale, nullptr, dq,
                     dq_dtype, dk, dv, dkv_dtype, workspace, workspace_bytes, cuda_stream);
+}
+
+af_status attnfuse_bwd_variant(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,
+                               const float* lse, const void* d_o, const af_strides* sq, const af_strides* skv,
+                               const af_variant* variant, int gqa_group, float softmax_scale, void* dq, af_dtype dq_dtype,
+                               void* dk, void* dv, af_dtype dkv_dtype, void* workspace, size_t workspace_bytes,
+                               void* cuda_stream) {
+    if (!variant) return AF_ERR_NULL;
+    if (variant->normaliser != AF_NORM_SOFTMAX && variant->normaliser != AF_NORM_RELU) return AF_ERR_SPEC;
+    const af_blocks* bl = variant->blocks;
+    if (bl) {
+        if (!bl->row_ptr || !bl->col_idx || !bl->col_ptr || !bl->row_idx) return AF_ERR_NULL;
+        if (bl->block != 128) return AF_ERR_SPEC;
+    }
+    return bwd_impl(shape, q, k, v, o, lse, d_o, sq, skv, &variant->rope, variant->rope_table, &variant->mask, gqa_group,
+                    softmax_scale, bl, dq, dq_dtype, dk, dv, dkv_dtype, workspace, workspace_bytes, cuda_stream, variant->bias,
+                    variant->bias_B, variant->bias_H, variant->normaliser == AF_NORM_RELU);
 }
 
 af_status attnfuse_bwd_blocks(const af_shape* shape, const void* q, const void* k, const void* v, const void* o,

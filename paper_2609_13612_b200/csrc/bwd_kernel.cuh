@@ -45,6 +45,12 @@ struct BwdParams {
     const int* bs_order;   // optional launch order of the stationary blocks (longest lists first), or nullptr
     int skip_rows;         // query rows i < skip_rows are left to bwd_first_rows_kernel (0: none)
     float* dq_acc;         // one-pass kernel only: fp32 accumulator of dQ' [B, Hq, S, D], zero on entry
+    // Section 3.1 extras (GEN kernels only): additive bias [bias_B, bias_H, S, S] with the element strides of its batch
+    // and head extents (0 where broadcast), and the ReLU normaliser, for which `lse` holds n_i, the number of kept
+    // pairs of the row (what the forward wrote there), and delta is not used.
+    const float* bias;
+    long long bias_sb, bias_sh;
+    int relu;
 };
 
 // delta[row] = <dO[row], O[row]>; one 16-byte chunk per thread, D/8 threads per row.
@@ -238,6 +244,57 @@ __device__ __forceinline__ void grad_pass32(uint32_t t1, uint32_t t2, int col0, 
     }
 }
 
+// The same pass for the variants with an additive bias and / or the ReLU normaliser (Section 3.1: additive_bias,
+// relu_attention), mask, ALiBi and bias decided at run time:
+//   softmax:  p = 2^(c2 s + alibi + log2(e) bias - L2),  ds = p (dP - delta)
+//   RELU:     t = c s + alibi + bias (natural units),  p = max(t, 0) / n,  ds = [t > 0] dP / n   (no delta)
+// A masked pair and a pair whose bias is -inf give p = ds = 0.  For RELU the per-row statistic passed in the place
+// of -L2 is 1 / n.  bias: address of the pair (this lane, column col0), col_stride elements between columns, cols_ok
+// valid columns from col0 on (nullptr: no bias, or this lane's row / key lies outside the sequence).
+template <bool DKV, bool RELU>
+__device__ __forceinline__ void grad_pass32_general(uint32_t t1, uint32_t t2, int col0, uint32_t out_col, float scale_log2,
+                                                    float cbias, float sb, const float* s_nl2, const float* s_ndl, float my_nl2,
+                                                    float my_ndl, int mlo, uint32_t mn, const float* bias, long long col_stride,
+                                                    int cols_ok) {
+    constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+    uint32_t s[32], dp[32], pk[16], dk[16];
+    tmem_ld32(t1 + col0, s);
+    tmem_ld32(t2 + col0, dp);
+    float bv[32];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) bv[c] = (bias && c < cols_ok) ? __ldg(bias + c * col_stride) : 0.f;
+    tmem_wait_ld();
+#pragma unroll
+    for (int c = 0; c < 32; c += 2) {
+        float pe[2], ds[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const float stat = DKV ? s_nl2[col0 + c + u] : my_nl2;
+            const float ndl = DKV ? s_ndl[col0 + c + u] : my_ndl;
+            const bool kept = static_cast<uint32_t>(col0 + c + u - mlo) < mn && bv[c + u] > -INFINITY;
+            // score in the log2 domain without the row statistic
+            const float t2v = fmaf(__uint_as_float(s[c + u]), scale_log2, fmaf(sb, static_cast<float>(c + u), cbias)) + bv[c + u] * kLog2e;
+            const float g = __uint_as_float(dp[c + u]);
+            if (RELU) {
+                const float tn = t2v * kLn2;
+                pe[u] = kept ? fmaxf(tn, 0.f) * stat : 0.f;
+                ds[u] = (kept && tn > 0.f) ? g * stat : 0.f;
+            } else {
+                pe[u] = kept ? ex2(t2v + stat) : 0.f;
+                ds[u] = pe[u] * (g + ndl);
+            }
+        }
+        pk[c >> 1] = pack_bf16x2(pe[0], pe[1]);
+        dk[c >> 1] = pack_bf16x2(ds[0], ds[1]);
+    }
+    if (DKV) {
+        tmem_st16(t1 + out_col, pk);
+        tmem_st16(t2 + out_col, dk);
+    } else {
+        tmem_st16(t1 + out_col, dk);
+    }
+}
+
 // ROT_X / ROT_A: rotate the stationary tile X / every streamed tile A on chip.  With p.store_x the rotated
 // stationary tile is also written to a cache in the caller's workspace through tm_s, so that the other
 // role can stream rotated rows instead of rotating every streamed tile again for every stationary tile.
@@ -257,7 +314,8 @@ __device__ __forceinline__ void grad_pass32(uint32_t t1, uint32_t t2, int col0, 
 #define AF_BSTAMP(role, it, ph) do { } while (0)
 #endif
 
-template <int D, bool DKV, bool ROT_X, bool ROT_A, bool BS = false>
+// GEN: the instantiation for additive_bias / relu_attention (grad_pass32_general), kept apart from the others.
+template <int D, bool DKV, bool ROT_X, bool ROT_A, bool BS = false, bool GEN = false>
 __global__ void __launch_bounds__(512, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_y,
                 const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
@@ -518,8 +576,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
         float my_l2 = 0.f, my_delta = 0.f, my_slope2 = 0.f;
         if (!DKV) {
             const size_t r = (static_cast<size_t>(b) * p.Hq + xh) * p.S + xrow;
-            my_l2 = xrow < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // kept negated
-            my_delta = xrow < p.S ? -p.delta[r] : 0.f;
+            if (GEN && p.relu) {   // lse holds n_i; the pass wants 1 / n_i
+                const float cnt = xrow < p.S ? p.lse[r] : 0.f;
+                my_l2 = cnt > 0.f ? 1.f / cnt : 0.f;
+            } else {
+                my_l2 = xrow < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // kept negated
+                my_delta = xrow < p.S ? -p.delta[r] : 0.f;
+            }
             my_slope2 = alibi ? p.slopes[xh] * kLog2e : 0.f;
         }
         bool ok = true;
@@ -556,8 +619,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 if (tid < 64) {
                     const int qi = a0 + hf * 64 + tid;
                     const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + qi;
-                    sL2[hf * 64 + tid] = qi < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // stored negated
-                    sDl[hf * 64 + tid] = qi < p.S ? -p.delta[r] : 0.f;
+                    if (GEN && p.relu) {
+                        const float cnt = qi < p.S ? p.lse[r] : 0.f;
+                        sL2[hf * 64 + tid] = cnt > 0.f ? 1.f / cnt : 0.f;
+                        sDl[hf * 64 + tid] = 0.f;
+                    } else {
+                        sL2[hf * 64 + tid] = qi < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // stored negated
+                        sDl[hf * 64 + tid] = qi < p.S ? -p.delta[r] : 0.f;
+                    }
                 }
                 my_slope2 = alibi ? p.slopes[ah] * kLog2e : 0.f;
             }
@@ -583,7 +652,22 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 const int col0 = hf * 64 + qt * 32;
                 const uint32_t out_col = hf * 64 + qt * 16;   // bf16 results: start of this warpgroup's own half
                 const float cbias = fmaf(sb, static_cast<float>(col0), bias_base);
-                if (alibi) {
+                if constexpr (GEN) {
+                    // bias of the pair (this lane, first column of the pass): DKV lane = key, columns = queries
+                    const float* bp = nullptr;
+                    long long cs = 1;
+                    int cols_ok = 0;
+                    if (p.bias && xrow < p.S) {
+                        const int hq = DKV ? ah : xh;
+                        const float* bh = p.bias + b * p.bias_sb + hq * p.bias_sh;
+                        if (DKV) { bp = bh + static_cast<long long>(a0 + col0) * p.S + xrow; cs = p.S; }
+                        else { bp = bh + static_cast<long long>(xrow) * p.S + a0 + col0; cs = 1; }
+                        cols_ok = p.S - (a0 + col0);
+                        if (cols_ok <= 0) bp = nullptr;
+                    }
+                    if (p.relu) grad_pass32_general<DKV, true>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, my_l2, my_delta, mlo, mn, bp, cs, cols_ok);
+                    else grad_pass32_general<DKV, false>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, my_l2, my_delta, mlo, mn, bp, cs, cols_ok);
+                } else if (alibi) {
                     if (need_mask) grad_pass32<DKV, true, true>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, my_l2, my_delta, mlo, mn);
                     else grad_pass32<DKV, false, true>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, my_l2, my_delta, mlo, mn);
                 } else {

@@ -739,9 +739,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
             }
-            if (p.lse && !(GEN && p.relu) && i < p.S)
-                p.lse[static_cast<size_t>(bh) * p.S + i] =
-                    l_run > 0.f ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+            if (p.lse && i < p.S) {
+                // softmax: L = m + ln l; relu_attention: n_i, the number of kept pairs of the row (its normaliser)
+                if (GEN && p.relu) p.lse[static_cast<size_t>(bh) * p.S + i] = l_run;
+                else p.lse[static_cast<size_t>(bh) * p.S + i] = l_run > 0.f ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+            }
         }
         if (BS && ok && jhi[q] < jlo[q] && i < p.S) {
             // no active block in this row block: the output row is zero and L = -inf
