@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-from paper_2609_13612_b200 import synth  # noqa: E402
+from paper_2609_13612_b200 import shard, synth  # noqa: E402
 
 METRIC = "fused RoPE+causal attention TFLOP/s (bf16 fwd/bwd) and % of B200 tensor peak"
 UNIT = "TFLOP/s"
@@ -318,7 +318,9 @@ def main():
         raise SystemExit("device-side wait ran out (0x%x): numbers invalid" % detail)
     ms_per_step = total_ms / args.steps
     flops = w.fwd_flops()
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    # whole-job throughput: what all ranks processed (every rank runs the same per-GPU workload) over the slowest
+    # rank's time (total_ms is already the max over ranks)
+    value = shard.aggregate_throughput([flops] * world, ms_per_step * 1e-3) / 1e12
     kern_ms = float(np.mean(per))
     achieved = flops / (kern_ms * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "attn_fwd_kernel<128,2,rope>", "achieved": achieved,
@@ -338,7 +340,7 @@ def main():
 
     e2e_steps = max(3, min(args.steps, 50))
     e2e_ms, _, _ = timed(step_host, e2e_steps, 3)
-    e2e_val = world * flops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    e2e_val = shard.aggregate_throughput([flops] * world, e2e_ms / e2e_steps * 1e-3) / 1e12
     h2d = int(hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2)
     d2h = int(ho.numel() * 2 + hl.numel() * 4)
 

@@ -133,3 +133,41 @@ def test_block_sparse_examples(data):
     pu.assert_close_scaled("bs dQ", pu.to_np(dq), wq)
     pu.assert_close_scaled("bs dK", pu.to_np(dk), wk)
     pu.assert_close_scaled("bs dV", pu.to_np(dv), wv)
+
+
+@settings(max_examples=20, **COMMON)
+@given(w=workloads(backward=True), extent=st.sampled_from(["full", "per_batch", "per_head", "shared"]),
+       minus_inf=st.sampled_from([0.0, 0.0, 0.25]))
+def test_additive_bias_examples(w, extent, minus_inf):
+    """Forward and backward of `additive_bias` composed with whatever else the example draws (Section 3.1)."""
+    sb, sh = {"full": (w.B, w.Hq), "per_batch": (w.B, 1), "per_head": (1, w.Hq), "shared": (1, 1)}[extent]
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([synth.BASE_SEED, w.seed_id, 11])))
+    bias = (0.5 * rng.standard_normal((sb, sh, w.S, w.S))).astype(np.float32)
+    if minus_inf > 0:
+        drop = rng.random(bias.shape) < minus_inf
+        drop[..., np.arange(w.S), np.arange(w.S)] = False      # keep the diagonal: no empty rows
+        bias[drop] = -np.inf
+    t = synth.draw_all(w)
+    dev = {k: pu.to_dev(v) for k, v in t.items()}
+    rope, mask = pu.specs(w)
+    table = af.rope_table(rope, w.S) if w.R > 0 else None
+    bias_dev = torch.from_numpy(bias).cuda()
+    o, lse = af.fwd_variant(dev["q"], dev["k"], dev["v"], rope, table, mask, w.scale, bias=bias_dev)
+    dq, dk, dv = af.bwd_variant(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale, bias=bias_dev,
+                                dq_dtype=torch.float32)
+    torch.cuda.synchronize()
+    assert af.device_status()[0] == 0
+    kw = dict(theta=w.theta, rotary_dim=w.R, pos_offset=w.pos_offset, causal=w.causal, window=w.window,
+              slopes=w.alibi_slopes(), scale=w.scale, bias=bias)
+    want_o, want_l = oracle.fwd(t["q"], t["k"], t["v"], **kw)
+    pu.assert_close_scaled("%r bias O" % (w,), pu.to_np(o), want_o)
+    assert np.abs(pu.to_np(lse) - want_l).max() <= pu.LSE_TOL, w
+    wq, wk, wv = oracle.bwd(t["q"], t["k"], t["v"], t["do"], **kw)
+    # The variant backward has no fp32 pass over the first query rows, and the drawn examples are full of rows whose
+    # probability mass sits on a handful of keys (causal first rows, -inf entries, non-causal ALiBi rows that collapse
+    # onto the last keys): those rows carry the bf16 roundings of P and dS at full size, the case the plain backward
+    # treats separately.  Stated bound for generated examples of this entry point: 4e-2 (measured worst 0.021-0.03).
+    tol = 4e-2
+    pu.assert_close_scaled("%r bias dQ" % (w,), pu.to_np(dq), wq, max_tol=tol)
+    pu.assert_close_scaled("%r bias dK" % (w,), pu.to_np(dk), wk, max_tol=tol)
+    pu.assert_close_scaled("%r bias dV" % (w,), pu.to_np(dv), wv, max_tol=tol)
