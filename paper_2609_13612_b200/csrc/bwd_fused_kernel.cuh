@@ -331,17 +331,36 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         constexpr float kLog2e = 1.4426950408889634f;
         const uint32_t ds_row_addr = smem_u32(sDS + hf * L::DS_HALF) + static_cast<uint32_t>(tid) * 128;
         bool ok = true;
-        for (int n = 0; ok && n < n_it; ++n) {
+        // per-column statistics of the streamed query tile; the loads for tile n + 1 are issued at the top of
+        // iteration n and stored to the other buffer after its passes (off the warpgroup's loop-carried chain)
+        float nx_l = 0.f, nx_d = 0.f, nx_slope = 0.f;
+        auto load_stats = [&](int n) {
             const int ah = stream_head(n), a0 = stream_row0(n);
-            float* sL2 = sStats + (n & 1) * 256;
-            float* sDl = sL2 + 128;
             if (tid < 64) {
                 const int qi = a0 + hf * 64 + tid;
                 const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + qi;
-                sL2[hf * 64 + tid] = qi < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // stored negated
-                sDl[hf * 64 + tid] = qi < p.S ? -p.delta[r] : 0.f;
+                nx_l = qi < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // kept negated
+                nx_d = qi < p.S ? -p.delta[r] : 0.f;
             }
-            const float my_slope2 = alibi ? p.slopes[ah] * kLog2e : 0.f;
+            nx_slope = alibi ? p.slopes[ah] * kLog2e : 0.f;
+        };
+        auto store_stats = [&](int n) {
+            if (tid < 64) {
+                float* dst = sStats + (n & 1) * 256 + hf * 64 + tid;
+                dst[0] = nx_l;
+                dst[128] = nx_d;
+            }
+        };
+        if (n_it > 0) {
+            load_stats(0);
+            store_stats(0);
+        }
+        for (int n = 0; ok && n < n_it; ++n) {
+            const int a0 = stream_row0(n);
+            float* sL2 = sStats + (n & 1) * 256;
+            float* sDl = sL2 + 128;
+            const float my_slope2 = nx_slope;
+            if (n + 1 < n_it) load_stats(n + 1);
             const bool need_mask = tile_needs_mask(ms, a0, x0);
             int mlo = 0;
             uint32_t mn = 128;
@@ -371,6 +390,7 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[L::B_PDS + hf]);
+            if (n + 1 < n_it) store_stats(n + 1);   // (published by the named barrier at the top of the next iteration)
         }
         if (ok && n_it > 0) ok = wg_all(mbar_wait(&bars[L::B_DONE], 0, abort_flag, 52));
         if (ok && n_it <= 0) {

@@ -610,25 +610,44 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             else if (p.R == 16) rot_x(std::integral_constant<int, 1>{});
             else rot_x(std::integral_constant<int, 0>{});
         }
+        // DKV: per-column statistics of the streamed query tile (each warpgroup stages its own 64 columns).  The
+        // global loads for tile n + 1 are issued at the top of iteration n and land in the other buffer after this
+        // iteration's passes, so that their latency is off the loop-carried chain of the warpgroup.
+        float nx_l = 0.f, nx_d = 0.f, nx_slope = 0.f;
+        auto load_stats = [&](int n) {
+            const int ah = stream_head(n), a0 = stream_row0(n);
+            if (tid < 64) {
+                const int qi = a0 + hf * 64 + tid;
+                const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + qi;
+                if (GEN && p.relu) {
+                    const float cnt = qi < p.S ? p.lse[r] : 0.f;
+                    nx_l = cnt > 0.f ? 1.f / cnt : 0.f;
+                    nx_d = 0.f;
+                } else {
+                    nx_l = qi < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // kept negated
+                    nx_d = qi < p.S ? -p.delta[r] : 0.f;
+                }
+            }
+            nx_slope = alibi ? p.slopes[ah] * kLog2e : 0.f;
+        };
+        auto store_stats = [&](int n) {
+            if (tid < 64) {
+                float* dst = sStats + (n & 1) * 256 + hf * 64 + tid;
+                dst[0] = nx_l;
+                dst[128] = nx_d;
+            }
+        };
+        if (DKV && ok && n_it > 0) {
+            load_stats(0);
+            store_stats(0);
+        }
         for (int n = 0; ok && n < n_it; ++n) {
             const int ah = stream_head(n), a0 = stream_row0(n);
             float* sL2 = sStats + (n & 1) * 256;
             float* sDl = sL2 + 128;
             if (DKV) {
-                // per-column statistics of the streamed query tile: each warpgroup stages its own 64 columns
-                if (tid < 64) {
-                    const int qi = a0 + hf * 64 + tid;
-                    const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + qi;
-                    if (GEN && p.relu) {
-                        const float cnt = qi < p.S ? p.lse[r] : 0.f;
-                        sL2[hf * 64 + tid] = cnt > 0.f ? 1.f / cnt : 0.f;
-                        sDl[hf * 64 + tid] = 0.f;
-                    } else {
-                        sL2[hf * 64 + tid] = qi < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // stored negated
-                        sDl[hf * 64 + tid] = qi < p.S ? -p.delta[r] : 0.f;
-                    }
-                }
-                my_slope2 = alibi ? p.slopes[ah] * kLog2e : 0.f;
+                my_slope2 = nx_slope;
+                if (n + 1 < n_it) load_stats(n + 1);
             }
             const int i0 = DKV ? a0 : x0, j0 = DKV ? x0 : a0;
             const bool need_mask = tile_needs_mask(ms, i0, j0);
@@ -681,6 +700,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[L::B_PDS + hf]);
             AF_BSTAMP(2 + hf, n, 3);
+            if (DKV && n + 1 < n_it) store_stats(n + 1);   // (the named barrier at the top of the next iteration publishes it)
         }
         // epilogue: stage through shared memory (the stream stages are idle now), rotate back, store
         AF_BSTAMP(2 + hf, 63, 0);
