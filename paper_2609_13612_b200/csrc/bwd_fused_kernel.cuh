@@ -392,7 +392,9 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
             if (lane == 0) mbar_arrive(&bars[L::B_PDS + hf]);
             if (n + 1 < n_it) store_stats(n + 1);   // (published by the named barrier at the top of the next iteration)
         }
-        if (ok && n_it > 0) ok = wg_all(mbar_wait(&bars[L::B_DONE], 0, abort_flag, 52));
+        // (every thread of both warpgroups takes this barrier, also after a wait that gave up in one of them:
+        // a warpgroup that left its loop early must not leave the other alone at it)
+        ok = wg_all(ok && (n_it <= 0 || mbar_wait(&bars[L::B_DONE], 0, abort_flag, 52)));
         if (ok && n_it <= 0) {
             // no query tile sees this key tile: its gradient rows are zero
             const size_t row0 = (static_cast<size_t>(b) * p.Hkv + xh) * p.S + x0;

@@ -704,7 +704,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
         }
         // epilogue: stage through shared memory (the stream stages are idle now), rotate back, store
         AF_BSTAMP(2 + hf, 63, 0);
-        if (ok && n_it > 0) ok = wg_all(mbar_wait(&bars[L::B_DONE], 0, abort_flag, 30));
+        // (every thread of both warpgroups takes this barrier, also after a wait that gave up in one of them:
+        // a warpgroup that left its loop early must not leave the other alone at it)
+        ok = wg_all(ok && (n_it <= 0 || mbar_wait(&bars[L::B_DONE], 0, abort_flag, 30)));
         AF_BSTAMP(2 + hf, 63, 1);   // accumulators complete
         if (BS && ok && n_it <= 0) {
             // no active block for this stationary block: its gradient rows are zero
