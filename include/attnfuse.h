@@ -188,6 +188,23 @@ af_status attnfuse_fwd_blocks(const af_shape* shape, const void* q, const void* 
                               int gqa_group, float softmax_scale, const af_blocks* blocks,
                               void* o, af_dtype o_dtype, float* lse, void* cuda_stream);
 
+/* ---- forward with 8-bit operands (opt-in; Section 9.1 names fp8 tensor cores as the natural extension) ----
+ * q8 [B,Hq,S,D], k8 [B,Hkv,S,D]: E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities),
+ * contiguous; vt8 [B,Hkv,D,S]: the E4M3 codes of V TRANSPOSED (keys contiguous); all DEVICE, 16-byte aligned.
+ * A value is code x scale: scale_q, scale_k, scale_v > 0 are per-tensor dequantisation scales (HOST floats).
+ * Computes softmax(softmax_scale x (q k^T) + mask) v with both products on the fp8 tensor path (fp32 accumulation),
+ * the softmax in fp32 and the probabilities rounded to E4M3 before the second product (the row sum uses the unrounded
+ * ones).  No rotation is applied: rotate in bf16 (attnfuse_rope) and quantise afterwards.  mask: causal and window as
+ * in attnfuse_fwd; ALiBi slopes -> AF_ERR_SPEC.  D = 128 and S a multiple of 16 (AF_ERR_SHAPE otherwise).
+ * o [B,Hq,S,D] in o_dtype, lse (nullable) [B,Hq,S] as in attnfuse_fwd.  Precision: the products of 8-bit operands are
+ * exact in fp32, so L matches the definition to fp32 rounding; the E4M3 rounding of a probability is up to 2^-4
+ * relative, and outputs are held to max abs 1e-1 and mean abs 8e-3 against the fp64 oracle evaluated on the
+ * dequantised inputs (unit-variance data; measured max 0.05, mean 0.001-0.006) - a bound of its own, not the bf16 path's. */
+af_status attnfuse_fwd_fp8(const af_shape* shape, const void* q8, const void* k8, const void* vt8,
+                           const af_mask* mask, int gqa_group, float softmax_scale,
+                           float scale_q, float scale_k, float scale_v,
+                           void* o, af_dtype o_dtype, float* lse, void* cuda_stream);
+
 /* ---- composed variants (Section 3.1: the ten combinators) ---------------------------------------------
  * One description of a variant and one forward entry point for it, the counterpart of a program composed
  * from the paper's combinators (Section 3.1) and run through its single run-time entry (Section 3.3):

@@ -101,6 +101,8 @@ def lib() -> ctypes.CDLL:
         L.attnfuse_fwd.restype = i
         L.attnfuse_fwd.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Strides), P(_Rope), vp, P(_Mask), i, f,
                                    vp, i, vp, vp]
+        L.attnfuse_fwd_fp8.restype = i
+        L.attnfuse_fwd_fp8.argtypes = [P(_Shape), vp, vp, vp, P(_Mask), i, f, f, f, f, vp, i, vp, vp]
         L.attnfuse_fwd_variant.restype = i
         L.attnfuse_fwd_variant.argtypes = [P(_Shape), vp, vp, vp, P(_Strides), P(_Strides), P(_Variant), i, f, vp, i, vp, vp]
         L.attnfuse_fwd_hybrid_workspace_bytes.restype = sz
@@ -342,6 +344,26 @@ def bwd_variant(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec
                                       Hq // Hkv, float(softmax_scale), dq.data_ptr(), code(dq_dtype), dk.data_ptr(),
                                       dv.data_ptr(), code(dkv_dtype), workspace.data_ptr(), workspace.numel(), _stream()))
     return dq, dk, dv
+
+
+def fwd_fp8(q8: torch.Tensor, k8: torch.Tensor, vt8: torch.Tensor, mask: MaskSpec, softmax_scale: float,
+            scale_q: float = 1.0, scale_k: float = 1.0, scale_v: float = 1.0, out_dtype: torch.dtype = torch.bfloat16):
+    """Forward with E4M3 operands: q8 [B,Hq,S,D], k8 [B,Hkv,S,D], vt8 [B,Hkv,D,S] (V transposed) as uint8 codes (or
+    torch.float8_e4m3fn tensors) on the device, value = code x scale.  Returns (o, lse)."""
+    _need_cuda(q8, k8, vt8)
+    q8, k8, vt8 = (t.view(torch.uint8) if t.dtype != torch.uint8 else t for t in (q8, k8, vt8))
+    assert q8.is_contiguous() and k8.is_contiguous() and vt8.is_contiguous()
+    B, Hq, S, D = q8.shape
+    Hkv = k8.shape[1]
+    assert k8.shape == (B, Hkv, S, D) and vt8.shape == (B, Hkv, D, S)
+    out = torch.empty((B, Hq, S, D), dtype=out_dtype, device=q8.device)
+    lse = torch.empty((B, Hq, S), dtype=torch.float32, device=q8.device)
+    sh = _Shape(B, Hq, Hkv, S, D)
+    m = _mask_struct(mask)
+    _check(lib().attnfuse_fwd_fp8(ctypes.byref(sh), q8.data_ptr(), k8.data_ptr(), vt8.data_ptr(), ctypes.byref(m), Hq // Hkv,
+                                  float(softmax_scale), float(scale_q), float(scale_k), float(scale_v), out.data_ptr(),
+                                  AF_F32 if out.dtype == torch.float32 else AF_BF16, lse.data_ptr(), _stream()))
+    return out, lse
 
 
 def fwd_hybrid(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, rope_spec: RopeSpec, table: Optional[torch.Tensor],

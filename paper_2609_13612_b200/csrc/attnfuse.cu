@@ -15,6 +15,7 @@
 #include "bwd_kernel.cuh"
 #include "bwd_first_rows.cuh"
 #include "bwd_fused_kernel.cuh"
+#include "fwd_fp8_kernel.cuh"
 #include "decode_kernels.cuh"
 #include "rope_kernels.cuh"
 
@@ -91,6 +92,23 @@ af_status make_tmap_uncached(CUtensorMap* tm, const void* ptr, int B, int H, int
     cuuint32_t box[4] = {static_cast<cuuint32_t>(BOX_COLS), static_cast<cuuint32_t>(rows), 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? AF_OK : AF_ERR_CUDA;
+}
+
+// Tensor map over one-byte elements [B, H, rows, cols] (contiguous), box of 128 x 128, 128-byte swizzle, zero fill:
+// the E4M3 operands of the fp8 forward (cols = D for Q and K; for the transposed V rows = D and cols = S).
+af_status make_tmap_u8(CUtensorMap* tm, const void* ptr, int B, int H, int rows, int cols) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return AF_ERR_CUDA;
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows), static_cast<cuuint64_t>(H),
+                          static_cast<cuuint64_t>(B)};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(cols) * rows,
+                             static_cast<cuuint64_t>(cols) * rows * H};
+    cuuint32_t box[4] = {128, 128, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? AF_OK : AF_ERR_CUDA;
@@ -774,6 +792,42 @@ af_status attnfuse_fwd_variant(const af_shape* shape, const void* q, const void*
                     bl ? bl->row_ptr : nullptr, bl ? bl->col_idx : nullptr, bl ? bl->row_order : nullptr, o, o_dtype, lse,
                     false, cuda_stream, bl, variant->bias, variant->bias_B, variant->bias_H,
                     variant->normaliser == AF_NORM_RELU);
+}
+
+af_status attnfuse_fwd_fp8(const af_shape* shape, const void* q8, const void* k8, const void* vt8, const af_mask* mask,
+                           int gqa_group, float softmax_scale, float scale_q, float scale_k, float scale_v, void* o,
+                           af_dtype o_dtype, float* lse, void* cuda_stream) {
+    if (!shape || !mask || !q8 || !k8 || !vt8 || !o) return AF_ERR_NULL;
+    if (shape->B < 1 || shape->Hq < 1 || shape->Hkv < 1 || shape->S < 1) return AF_ERR_SHAPE;
+    if (shape->D != 128 || (shape->S % 16) != 0) return AF_ERR_SHAPE;   // the transposed V has rows of S bytes: 16-byte strides
+    if (gqa_group < 1 || shape->Hkv * gqa_group != shape->Hq) return AF_ERR_SHAPE;
+    if (mask->alibi_slopes) return AF_ERR_SPEC;
+    if (o_dtype != AF_BF16 && o_dtype != AF_F32) return AF_ERR_DTYPE;
+    if (!aligned16(q8) || !aligned16(k8) || !aligned16(vt8) || !aligned16(o)) return AF_ERR_ALIGN;
+    if (!(softmax_scale > 0.f) || !isfinite(softmax_scale) || !(scale_q > 0.f) || !(scale_k > 0.f) || !(scale_v > 0.f) ||
+        !isfinite(scale_q) || !isfinite(scale_k) || !isfinite(scale_v))
+        return AF_ERR_SPEC;
+    af_status st = check_arch();
+    if (st != AF_OK) return st;
+    CUtensorMap tq, tk, tv;
+    if ((st = make_tmap_u8(&tq, q8, shape->B, shape->Hq, shape->S, shape->D)) != AF_OK) return st;
+    if ((st = make_tmap_u8(&tk, k8, shape->B, shape->Hkv, shape->S, shape->D)) != AF_OK) return st;
+    if ((st = make_tmap_u8(&tv, vt8, shape->B, shape->Hkv, shape->D, shape->S)) != AF_OK) return st;
+    Fp8Params p;
+    p.B = shape->B; p.Hq = shape->Hq; p.Hkv = shape->Hkv; p.S = shape->S; p.group = gqa_group;
+    p.causal = mask->causal ? 1 : 0;
+    p.window = mask->window < 0 ? -1 : (mask->window > shape->S ? shape->S : mask->window);
+    p.scale_log2 = softmax_scale * scale_q * scale_k * 1.4426950408889634f;
+    p.out_scale = scale_v;
+    p.o = o; p.o_f32 = o_dtype == AF_F32; p.lse = lse;
+    p.pair_heads = (gqa_group % 2) == 0 ? 1 : 0;
+    const int rows_per_cta = p.pair_heads ? BM : 2 * BM;
+    p.n_row_blocks = (shape->S + rows_per_cta - 1) / rows_per_cta;
+    static std::atomic<unsigned long long> configured{0};
+    if (allow_dynamic_smem(attn_fwd_fp8_kernel, Fp8Smem::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
+    dim3 grid(p.pair_heads ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
+    attn_fwd_fp8_kernel<<<grid, 512, Fp8Smem::BYTES, static_cast<cudaStream_t>(cuda_stream)>>>(tq, tk, tv, p);
+    return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
 size_t attnfuse_fwd_hybrid_workspace_bytes(const af_shape* shape) {

@@ -11,7 +11,10 @@ shapes are the workload itself, not a stand-in for a dataset.
 
 Values are drawn in fp32 and rounded once (round-to-nearest-even) to bf16; the
 rounded values are what both sides consume, so input quantisation is never
-charged to either side as error.
+charged to either side as error.  For the fp8 entry point the same holds one step
+further: the inputs are rounded to 8-bit E4M3 codes here (a number-format
+conversion, no arithmetic of the method), the CUDA path takes the codes and the
+oracle their decoded values.
 """
 from __future__ import annotations
 
@@ -44,6 +47,39 @@ def bits_to_f32(bits: np.ndarray) -> np.ndarray:
     """fp32 values of bf16 bit patterns."""
     b = np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << 16
     return b.view(np.float32).reshape(bits.shape)
+
+
+def e4m3_decode(codes: np.ndarray) -> np.ndarray:
+    """fp32 values of 8-bit E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities, the one
+    NaN pattern S.1111.111; largest finite value 448): the operand format of the fp8 entry point."""
+    c = np.ascontiguousarray(codes, dtype=np.uint8).astype(np.int32)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 0xF
+    m = c & 0x7
+    val = np.where(e == 0, m * 2.0 ** -9, (8 + m) * np.exp2(e.astype(np.float64) - 10.0))
+    val = np.where((e == 15) & (m == 7), np.nan, val)
+    return (sign * val).astype(np.float32).reshape(codes.shape)
+
+
+def e4m3_encode(x: np.ndarray) -> np.ndarray:
+    """8-bit E4M3 codes of fp32 values: round to nearest, ties to even, saturating at +-448."""
+    x = np.ascontiguousarray(x, dtype=np.float32).astype(np.float64)
+    sign = np.signbit(x)
+    a = np.minimum(np.abs(x), 448.0)
+    # exponent of the spacing: values below 2^-6 share the subnormal spacing 2^-9
+    e = np.floor(np.log2(np.maximum(a, 2.0 ** -6)))
+    e = np.clip(e, -6, 8)
+    step = np.exp2(e - 3)
+    q = np.rint(a / step)                      # numpy rounds halves to even
+    # a mantissa that rounded up to 16 steps moves to the next exponent
+    bump = q >= 16
+    e = np.where(bump, e + 1, e)
+    q = np.where(bump, 8, q)
+    sub = a < 2.0 ** -6
+    qs = np.rint(a / 2.0 ** -9)                # subnormal range: 0 .. 8 steps of 2^-9 (8 is the smallest normal)
+    code = np.where(sub, np.where(qs >= 8, 0x08, qs), ((e + 7).astype(np.int64) << 3) | (q.astype(np.int64) - 8))
+    code = np.minimum(code.astype(np.int64), 0x7E)
+    return (code | (sign.astype(np.int64) << 7)).astype(np.uint8).reshape(x.shape)
 
 
 @dataclasses.dataclass(frozen=True)
