@@ -166,7 +166,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--extras", type=int, default=1, help="also time configs 3-5, the separate-RoPE arm and the sweep")
     ap.add_argument("--cpu-baseline", type=int, default=1)
-    ap.add_argument("--profile", default="", choices=["", "fwd", "hybrid", "bwd", "bwd2", "rope", "decode", "fwd_c3", "fwd_d64", "blocks"],
+    ap.add_argument("--profile", default="", choices=["", "fwd", "hybrid", "bwd", "bwd2", "rope", "decode", "fwd_c3", "fwd_d64", "blocks", "fp8"],
                     help="run only a few launches of one path (for ncu captures) and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -256,6 +256,21 @@ def main():
             af.decode(qd, kc[i % 3], vc[i % 3], af.MaskSpec(True, -1, None), 128 ** -0.5)
         torch.cuda.synchronize()
         print(json.dumps({"profile": "decode", "workload": "llama3_70b_decode_32768", "device_status": af.device_status()[0]}))
+        return
+    if args.profile == "fp8":
+        # the opt-in forward with E4M3 operands on the Llama-3-8B shape (causal, no rotation inside)
+        wl = synth.CONFIGS[1]
+        g8 = torch.Generator(device=dev).manual_seed(11)
+        x8 = {}
+        for name, H_ in (("q", wl.Hq), ("k", wl.Hkv), ("v", wl.Hkv)):
+            x = torch.randn((wl.B, H_, wl.S, wl.D), device=dev, generator=g8)
+            sc = float(x.abs().max()) / 448.0
+            y = (x / sc).to(torch.float8_e4m3fn)
+            x8[name] = (y.transpose(2, 3).contiguous() if name == "v" else y, sc)
+        for _ in range(3):
+            af.fwd_fp8(x8["q"][0], x8["k"][0], x8["v"][0], af.MaskSpec(causal=True), wl.scale, x8["q"][1], x8["k"][1], x8["v"][1])
+        torch.cuda.synchronize()
+        print(json.dumps({"profile": "fp8", "workload": wl.name + " (E4M3 operands, no RoPE)", "device_status": af.device_status()[0]}))
         return
     if args.profile:
         # a handful of launches of one path on its configuration, nothing else: the target of ncu captures
