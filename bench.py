@@ -445,6 +445,24 @@ def main():
                     "dequantised inputs; compare with the bf16 kernel without RoPE on the same shape (rotation_calculus_sweep, S = 4096)"}
         del sets8
         torch.cuda.empty_cache()
+        # Composed variants of Section 3.1 on the same shape: a shared additive bias [1, 1, S, S] (fp32, 64 MB, read once per
+        # head: the variant is bound by that traffic) and the ReLU normaliser, forward and backward.
+        sv_ = make_sets(synth.Workload("variants_on_c2_shape", wl.B, wl.Hq, wl.Hkv, wl.S, wl.D, theta=wl.theta, backward=True,
+                                       seed_id=55), 1)[0]
+        rv, mv, tv_ = specs(wl)
+        bias_v = torch.randn((1, 1, wl.S, wl.S), device=dev, generator=torch.Generator(device=dev).manual_seed(5)) * 0.5
+        wsv = torch.empty(af.bwd_workspace_bytes(wl.B, wl.Hq, wl.Hkv, wl.S, wl.D, onepass=False), dtype=torch.uint8, device=dev)
+        var = {}
+        for tag, kw in (("additive_bias", dict(bias=bias_v)), ("relu_attention", dict(normaliser="relu"))):
+            tf_, _, _ = timed(lambda i: af.fwd_variant(sv_["q"], sv_["k"], sv_["v"], rv, tv_, mv, wl.scale, **kw), k_ex, w_ex)
+            ov, lv = af.fwd_variant(sv_["q"], sv_["k"], sv_["v"], rv, tv_, mv, wl.scale, **kw)
+            tb_, _, _ = timed(lambda i: af.bwd_variant(sv_["q"], sv_["k"], sv_["v"], ov, lv, sv_["do"], rv, tv_, mv, wl.scale,
+                                                       workspace=wsv, **kw), k_ex, w_ex)
+            var[tag] = {"fwd_ms": tf_ / k_ex, "fwd_tflops": wl.fwd_flops() / (tf_ / k_ex) / 1e9,
+                        "bwd_ms": tb_ / k_ex, "bwd_tflops": 2.5 * wl.fwd_flops() / (tb_ / k_ex) / 1e9}
+        ex["composed_variants_on_c2_shape"] = var
+        del sv_, bias_v, wsv
+        torch.cuda.empty_cache()
         for wl in synth.CONFIGS[1:4]:
             ms_f, ss = fwd_ms(wl, True)
             ms_s, _ = fwd_ms(wl, False, ss)
