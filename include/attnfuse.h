@@ -59,7 +59,7 @@ typedef struct { float theta; int rotary_dim; int pos_offset; } af_rope;
  * the scaled score. */
 typedef struct { int causal; int window; const float* alibi_slopes; } af_mask;
 
-int         attnfuse_version(void);
+int         attnfuse_version(void);   /* 100 x major + minor: 110 adds the variant, one-pass backward and fp8 entries */
 const char* attnfuse_strerror(af_status st);
 
 /* ---- tuning options ---------------------------------------------------------------------------------

@@ -574,7 +574,7 @@ size_t bwd_dqacc_bytes(const af_shape* sh) {
 
 extern "C" {
 
-int attnfuse_version(void) { return 100; }
+int attnfuse_version(void) { return 110; }
 
 const char* attnfuse_strerror(af_status st) {
     switch (st) {
