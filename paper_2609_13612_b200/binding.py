@@ -494,9 +494,9 @@ def fwd_host_staging_bytes(B: int, Hq: int, Hkv: int, S: int, D: int) -> int:
 
 def bwd_workspace_bytes(B: int, Hq: int, Hkv: int, S: int, D: int, onepass: bool = True) -> int:
     """Workspace size of the backward: with `onepass` the size that admits the one-pass sequence (delta, both
-    rotated caches and the fp32 dQ accumulator; D = 128), otherwise delta and the two caches."""
+    rotated caches and the fp32 dQ accumulator), otherwise delta and the two caches."""
     sh = _Shape(B, Hq, Hkv, S, D)
-    if onepass and D == 128:
+    if onepass:
         return lib().attnfuse_bwd_onepass_workspace_bytes(ctypes.byref(sh))
     return lib().attnfuse_bwd_workspace_bytes(ctypes.byref(sh))
 

@@ -421,6 +421,7 @@ af_status launch_bwd_mma(const af_shape* sh, const CUtensorMap& tq, const CUtens
                          cudaStream_t stream);
 
 struct OnePassArgs;
+template <int D>
 af_status launch_bwd_onepass(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                              const CUtensorMap& tdo, const CUtensorMap& tkp, const CUtensorMap& tqp, const void* k,
                              const af_strides& stkv, void* kcache, const void* o, const void* d_o, BwdParams p, void* dq,
@@ -435,15 +436,10 @@ af_status launch_bwd(const af_shape* sh, const CUtensorMap& tq, const CUtensorMa
                      cudaStream_t stream, const FirstRowsParams& fp, const OnePassArgs* onepass) {
     p.skip_rows = fp.rows;
     af_status st;
-    if constexpr (D == 128) {
-        st = onepass ? launch_bwd_onepass(sh, tq, tk, tv, tdo, tkp ? *tkp : tk, tqp ? *tqp : tq, k, stkv, kcache, o, d_o, p, dq, dq_f32, dk, dv,
-                                          dkv_f32, delta, *onepass, stream)
-                     : launch_bwd_mma<D>(sh, tq, tk, tv, tdo, tkp, tqp, k, stkv, kcache, o, d_o, p, dq, dq_f32, dk, dv,
-                                         dkv_f32, delta, blocks, stream);
-    } else {
-        st = launch_bwd_mma<D>(sh, tq, tk, tv, tdo, tkp, tqp, k, stkv, kcache, o, d_o, p, dq, dq_f32, dk, dv, dkv_f32,
-                               delta, blocks, stream);
-    }
+    st = onepass ? launch_bwd_onepass<D>(sh, tq, tk, tv, tdo, tkp ? *tkp : tk, tqp ? *tqp : tq, k, stkv, kcache, o, d_o, p, dq, dq_f32,
+                                         dk, dv, dkv_f32, delta, *onepass, stream)
+                 : launch_bwd_mma<D>(sh, tq, tk, tv, tdo, tkp, tqp, k, stkv, kcache, o, d_o, p, dq, dq_f32, dk, dv,
+                                     dkv_f32, delta, blocks, stream);
     if (st != AF_OK || fp.rows == 0) return st;
     return launch_first_rows<D>(fp, stream);
 }
@@ -457,12 +453,12 @@ struct OnePassArgs {
     float* dq_acc;
     size_t dq_acc_bytes;
 };
+template <int D>
 af_status launch_bwd_onepass(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                              const CUtensorMap& tdo, const CUtensorMap& tkp, const CUtensorMap& tqp, const void* k,
                              const af_strides& stkv, void* kcache, const void* o, const void* d_o, BwdParams p, void* dq,
                              int dq_f32, void* dk, void* dv, int dkv_f32, float* delta, const OnePassArgs& a,
                              cudaStream_t stream) {
-    constexpr int D = 128;
     using L = BwdFusedSmem<D>;
     if (cudaMemsetAsync(a.dq_acc, 0, a.dq_acc_bytes, stream) != cudaSuccess) return AF_ERR_CUDA;
     const long long rows = static_cast<long long>(sh->B) * sh->Hq * sh->S;
@@ -1134,7 +1130,7 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     CUtensorMap tkp, tqp;
     const size_t off_k = bwd_delta_bytes(shape), off_q = off_k + bwd_kcache_bytes(shape);
     const size_t off_acc = off_q + bwd_qcache_bytes(shape);
-    // One-pass sequence: D = 128, dense, room for both caches and the fp32 dQ' accumulator, and not switched off.
+    // One-pass sequence: dense, room for both caches and the fp32 dQ' accumulator, and not switched off.
     // Left to itself (option value 1) the choice goes by the average number of kept key tiles per query tile: the
     // one-pass kernel costs more per tile pair than the two roles of the two-kernel sequence together, but the dQ
     // role pays a fixed set-up and epilogue per query tile, which dominates while rows are short (measured: ahead at
@@ -1143,8 +1139,10 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     const double n_tiles = (shape->S + 127) / 128;
     double avg_tiles = p.causal ? 0.5 * (n_tiles + 1) : n_tiles;
     if (p.window >= 0) avg_tiles = std::min(avg_tiles, (p.causal ? 1.0 : 2.0) * p.window / 128.0 + 1.5);
-    const bool onepass = shape->D == 128 && !blocks && !gen && workspace_bytes >= off_acc + bwd_dqacc_bytes(shape) &&
-                         (mode >= 2 || (mode == 1 && avg_tiles <= 12.0));
+    // At D = 64 the one-pass sequence measured 1.21-1.25 times faster on every shape tried (short and long rows,
+    // grouped queries, window, no causal mask): shared-memory traffic per tile pair is half that of D = 128.
+    const bool onepass = !blocks && !gen && workspace_bytes >= off_acc + bwd_dqacc_bytes(shape) &&
+                         (mode >= 2 || (mode == 1 && (shape->D == 64 || avg_tiles <= 12.0)));
     const bool have_k = p.R > 0 && workspace_bytes >= off_q;
     const bool have_q = have_k && workspace_bytes >= off_acc;
     void* kc = static_cast<uint8_t*>(workspace) + off_k;
@@ -1181,7 +1179,8 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
                                  d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream, fp,
                                  onepass ? &op : nullptr)
                : launch_bwd<64>(shape, tq, tk, tv, tdo, have_k ? &tkp : nullptr, have_q ? &tqp : nullptr, k, stkv, kc, o,
-                                d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream, fp, nullptr);
+                                d_o, p, dq, dq_dtype == AF_F32, dk, dv, dkv_dtype == AF_F32, delta, blocks, stream, fp,
+                                onepass ? &op : nullptr);
 }
 }  // namespace
 

@@ -91,14 +91,14 @@ def test_backward_examples(w, tier, dq_f32):
     # reach) measured up to 0.049 there and nothing above 2e-2 outside these classes.  The paper composes ALiBi with
     # causal only; no benchmark configuration is of this kind.  Stated bound for that class: the common bound plus twice
     # that estimate, 2e-2 + 2 x 2^-9 sqrt(g S) (measured: 0.091 at g S = 2128, where the estimate itself is 0.090).
-    tol = pu.MAX_ABS_TOL
-    if w.causal and 0 <= w.window < 16:
-        tol = 4e-2
+    tol, mean_tol = pu.MAX_ABS_TOL, pu.MEAN_ABS_TOL
+    if 0 <= w.window < 16:      # with or without the causal rule (two-sided: at most 2 W + 1 keys per row)
+        tol, mean_tol = 4e-2, 2 * pu.MEAN_ABS_TOL      # nothing averages on any row: the mean error doubles as well
     if not w.causal and w.alibi:
         tol = 2e-2 + 2.0 * 2.0 ** -9 * float(np.sqrt(w.group * w.S))
-    pu.assert_close_scaled("%r dQ" % (w,), pu.to_np(dq), wq, max_tol=tol)
-    pu.assert_close_scaled("%r dK" % (w,), pu.to_np(dk), wk, max_tol=tol)
-    pu.assert_close_scaled("%r dV" % (w,), pu.to_np(dv), wv, max_tol=tol)
+    pu.assert_close_scaled("%r dQ" % (w,), pu.to_np(dq), wq, max_tol=tol, mean_tol=mean_tol)
+    pu.assert_close_scaled("%r dK" % (w,), pu.to_np(dk), wk, max_tol=tol, mean_tol=mean_tol)
+    pu.assert_close_scaled("%r dV" % (w,), pu.to_np(dv), wv, max_tol=tol, mean_tol=mean_tol)
 
 
 @st.composite
