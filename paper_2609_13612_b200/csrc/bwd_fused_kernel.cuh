@@ -25,9 +25,10 @@
 // role's CTAs are short (few key tiles per query tile), behind on long rows.  (A variant with ONE dP^T buffer
 // handed back as soon as it is in registers and ONE dQ'^T buffer of its own measured slower still, 8.0 k.)
 // D = 64: the same kernel; dQ'^T then has M = 64 rows, which tcgen05 keeps in the first 16 lanes of each 32-lane quarter of
-// TMEM (row d in lane 32 (d / 16) + d % 16), so half of the reducing lanes carry a row.  Shared-memory traffic per tile
-// pair is half that of D = 128 and the sequence measured 1.21-1.25 times faster than the two-kernel one on every shape
-// tried (0.691 -> 0.561 ms at B = 4, 12 heads, N = 4096).
+// TMEM (row d in lane 32 (d / 16) + d % 16), so half of the reducing lanes carry a row; and the accumulators leave 128
+// TMEM columns free, so the partials get two 64-column buffers of their own and T2 never waits for a read-out.
+// Shared-memory traffic per tile pair is half that of D = 128; the sequence measured 1.23-1.31 times faster than the
+// two-kernel one on every shape tried (0.691 -> 0.546 ms at B = 4, 12 heads, N = 4096).
 // Warp roles (512 threads): warp 0 TMA producer; warps 1, 2, 3 MMA issuers (T1 and dV; T2 and dK'; dQ'^T), one
 // per SM sub-partition; warps 4-7 read the dQ'^T partials out of TMEM and add them to global memory; warps 8-11
 // and 12-15 are the two gradient warpgroups.
@@ -117,6 +118,11 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
     constexpr int NBOX = D / BOX_COLS;
     constexpr uint32_t TMEM_COLS = 512;
     constexpr uint32_t T1 = 0, T2 = 128, ACC1 = 256, ACC2 = 256 + D;
+    // Where the dQ'^T partial of a half lands.  D = 128: TMEM is full, it takes the half of T2 whose dP^T has just been
+    // consumed, and the next dP^T of that half waits for its read-out.  D = 64: the accumulators leave 128 columns free,
+    // the partials get two 64-column buffers of their own there and T2 never waits for them.
+    constexpr bool kOwnDq = D == 64;
+    constexpr uint32_t TDQ = kOwnDq ? 384 : T2;
     constexpr uint32_t IDESC_TH = idesc_bf16_f32(128, 64, 0, 0);     // S^T / dP^T half: 64 streamed rows
     constexpr uint32_t IDESC_ACC = idesc_bf16_f32(128, D, 0, 1);     // dV, dK': B MN-major
     constexpr uint32_t IDESC_DQ = idesc_bf16_f32(D, 64, 1, 1);       // dQ'^T half: A = K'^T and B = dS^T both MN-major
@@ -255,7 +261,7 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                     if (next) {
                         if (hf == 0) ok = wait_stream(n + 1);
                         // T2's half is free once the dQ'^T partial of the same rows has been read out of it
-                        if (ok && who == 1) ok = mbar_wait(&bars[L::B_T2FREE + hf], n & 1, abort_flag, 46);
+                        if (ok && who == 1 && !kOwnDq) ok = mbar_wait(&bars[L::B_T2FREE + hf], n & 1, abort_flag, 46);
                         if (!ok) break;
                         tc_fence_after_sync();
                         issue_T(n + 1, hf);
@@ -275,10 +281,12 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
                     ok = mbar_wait(&bars[L::B_PDS + hf], n & 1, abort_flag, 48);
+                    // (own buffers: the previous tile's partial of this half must have been read out)
+                    if (ok && kOwnDq && n > 0) ok = mbar_wait(&bars[L::B_T2FREE + hf], (n - 1) & 1, abort_flag, 54);
                     if (!ok) break;
                     tc_fence_after_sync();
                     const uint32_t b_lo = desc_lo(smem_u32(sDS + hf * L::DS_HALF), 16);
-                    const uint32_t dst = tmem_base + T2 + hf * 64;
+                    const uint32_t dst = tmem_base + TDQ + hf * 64;
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         if (kk == 0) mma_ss_lo<false>(dst, a_lo + kk * 128, b_lo + kk * 128, dhi, IDESC_DQ);
@@ -296,7 +304,7 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         // of each 32-lane quarter (row d in lane 32 (d / 16) + d % 16); the other 16 lanes of a warp hold nothing.
         const int d = D == 128 ? (warp & 3) * 32 + lane : (warp & 3) * 16 + (lane & 15);
         const bool has_row = D == 128 || lane < 16;
-        const uint32_t tsrc = tmem_base + T2 + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const uint32_t tsrc = tmem_base + TDQ + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         bool ok = true;
         for (int n = 0; ok && n < n_it; ++n) {
             const int ah = stream_head(n), a0 = stream_row0(n);
