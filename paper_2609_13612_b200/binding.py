@@ -513,8 +513,7 @@ def bwd(q, k, v, o, lse, d_o, rope_spec: RopeSpec, table, mask: MaskSpec, softma
     assert o.dtype == d_o.dtype == torch.bfloat16 and lse.dtype == torch.float32
     sh = _Shape(B, Hq, Hkv, S, D)
     if workspace is None:
-        workspace = torch.empty(bwd_workspace_bytes(B, Hq, Hkv, S, D, onepass=blocks is None), dtype=torch.uint8,
-                                device=q.device)
+        workspace = torch.empty(bwd_workspace_bytes(B, Hq, Hkv, S, D), dtype=torch.uint8, device=q.device)
     dq = torch.empty((B, Hq, S, D), dtype=dq_dtype, device=q.device)
     dk = torch.empty((B, Hkv, S, D), dtype=dkv_dtype, device=q.device)
     dv = torch.empty((B, Hkv, S, D), dtype=dkv_dtype, device=q.device)

@@ -452,6 +452,7 @@ struct OnePassArgs {
     void* qcache;
     float* dq_acc;
     size_t dq_acc_bytes;
+    const af_blocks* blocks;   // block-sparse lists or nullptr
 };
 template <int D>
 af_status launch_bwd_onepass(const af_shape* sh, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
@@ -474,9 +475,13 @@ af_status launch_bwd_onepass(const af_shape* sh, const CUtensorMap& tq, const CU
     p.delta = delta;
     p.out1 = dv; p.out2 = dk; p.out_f32 = dkv_f32; p.store_x = 0;
     p.dq_acc = a.dq_acc;
-    auto kern = attn_bwd_fused_kernel<D>;
-    static std::atomic<unsigned long long> configured{0};
-    if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
+    // block lists by key block (the stationary block of this kernel)
+    p.bs_ptr = a.blocks ? a.blocks->col_ptr : nullptr;
+    p.bs_idx = a.blocks ? a.blocks->row_idx : nullptr;
+    p.bs_order = a.blocks ? a.blocks->col_order : nullptr;
+    auto kern = a.blocks ? attn_bwd_fused_kernel<D, true> : attn_bwd_fused_kernel<D, false>;
+    static std::atomic<unsigned long long> configured[2];
+    if (allow_dynamic_smem(kern, L::BYTES, configured[a.blocks ? 1 : 0]) != AF_OK) return AF_ERR_CUDA;
     const unsigned tiles = static_cast<unsigned>((sh->S + 127) / 128);
     dim3 grid(sh->B * sh->Hkv, tiles, 1);
     st = p.R > 0 ? launch_kernel(kern, grid, dim3(512, 1, 1), L::BYTES, stream, true, tkp, tv, tqp, tdo, p)
@@ -1139,10 +1144,11 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     const double n_tiles = (shape->S + 127) / 128;
     double avg_tiles = p.causal ? 0.5 * (n_tiles + 1) : n_tiles;
     if (p.window >= 0) avg_tiles = std::min(avg_tiles, (p.causal ? 1.0 : 2.0) * p.window / 128.0 + 1.5);
-    // At D = 64 the one-pass sequence measured 1.21-1.25 times faster on every shape tried (short and long rows,
+    // At D = 64 the one-pass sequence measured 1.2-1.3 times faster on every shape tried (short and long rows,
     // grouped queries, window, no causal mask): shared-memory traffic per tile pair is half that of D = 128.
-    const bool onepass = !blocks && !gen && workspace_bytes >= off_acc + bwd_dqacc_bytes(shape) &&
-                         (mode >= 2 || (mode == 1 && (shape->D == 64 || avg_tiles <= 12.0)));
+    // Over block lists (short lists are the rule there) it is taken at D = 64 and, at D = 128, only on request.
+    const bool onepass = !gen && workspace_bytes >= off_acc + bwd_dqacc_bytes(shape) &&
+                         (mode >= 2 || (mode == 1 && (shape->D == 64 || (!blocks && avg_tiles <= 12.0))));
     const bool have_k = p.R > 0 && workspace_bytes >= off_q;
     const bool have_q = have_k && workspace_bytes >= off_acc;
     void* kc = static_cast<uint8_t*>(workspace) + off_k;
@@ -1173,6 +1179,7 @@ af_status bwd_impl(const af_shape* shape, const void* q, const void* k, const vo
     op.q = q; op.stq = stq; op.qcache = qc;
     op.dq_acc = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + off_acc);
     op.dq_acc_bytes = bwd_dqacc_bytes(shape);
+    op.blocks = blocks;
     p.dq_acc = nullptr;
     return shape->D == 128
                ? launch_bwd<128>(shape, tq, tk, tv, tdo, have_k ? &tkp : nullptr, have_q ? &tqp : nullptr, k, stkv, kc, o,

@@ -108,7 +108,9 @@ __device__ __forceinline__ void grad_pass32_fused(uint32_t t1, uint32_t t2, int 
     }
 }
 
-template <int D>
+// BS: block-sparse attention (Section 4.3) - the streamed query tiles of a key block come from its list of active
+// blocks (p.bs_ptr / p.bs_idx by key block, p.bs_order the launch order) instead of a contiguous range.
+template <int D, bool BS = false>
 __global__ void __launch_bounds__(512, 1)
 attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_y,
                       const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const BwdParams p) {
@@ -143,13 +145,23 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const MaskSpec ms{p.S, p.causal, p.window, p.skip_rows};
     const int b = blockIdx.x / p.Hkv, xh = blockIdx.x - b * p.Hkv;
-    const int x0 = static_cast<int>(blockIdx.y) * 128;   // heaviest key tiles first under a causal mask
+    // heaviest key tiles first under a causal mask; with block lists the caller's order
+    const int x0 = ((BS && p.bs_order) ? __ldg(p.bs_order + blockIdx.y) : static_cast<int>(blockIdx.y)) * 128;
     int lo, hi;
     qtile_range(ms, x0, lo, hi);
+    int bs_base = 0;
+    if constexpr (BS) {   // positions in the key block's list instead of a tile range
+        bs_base = __ldg(p.bs_ptr + x0 / 128);
+        lo = 0;
+        hi = __ldg(p.bs_ptr + x0 / 128 + 1) - bs_base - 1;
+    }
     const int per_head = hi - lo + 1;
     const int n_it = per_head > 0 ? per_head * p.group : 0;
     auto stream_head = [&](int n) { return xh * p.group + n / per_head; };
-    auto stream_row0 = [&](int n) { return (lo + n % per_head) * 128; };
+    auto stream_row0 = [&](int n) {
+        const int pos = lo + n % per_head;
+        return (BS ? __ldg(p.bs_idx + bs_base + pos) : pos) * 128;
+    };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::N_BARS; ++i) {

@@ -113,11 +113,14 @@ def run_bwd(w, active, workspace_tier=2, dq_dtype=torch.bfloat16):
     rope, mask = pu.specs(w)
     table = af.rope_table(rope, w.S) if w.R > 0 else None
     n_delta = (w.B * w.Hq * w.S * 4 + 255) // 256 * 256
+    # tier 3: room for the fp32 dQ accumulator as well, and the one-pass sequence forced (over block lists it is the
+    # default only at D = 64)
     n_ws = n_delta + (w.B * w.Hkv * w.S * w.D * 2 if workspace_tier >= 1 else 0) + \
-        (w.B * w.Hq * w.S * w.D * 2 if workspace_tier >= 2 else 0)
+        (w.B * w.Hq * w.S * w.D * 2 if workspace_tier >= 2 else 0) + (w.B * w.Hq * w.S * w.D * 4 if workspace_tier >= 3 else 0)
     ws = torch.empty(n_ws, dtype=torch.uint8, device="cuda")
-    dq, dk, dv = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale, workspace=ws,
-                        blocks=bm, dq_dtype=dq_dtype)
+    with af.option(af.OPT_BWD_ONEPASS, 2 if workspace_tier >= 3 else 0):
+        dq, dk, dv = af.bwd(dev["q"], dev["k"], dev["v"], o, lse, dev["do"], rope, table, mask, w.scale, workspace=ws,
+                            blocks=bm, dq_dtype=dq_dtype)
     torch.cuda.synchronize()
     assert af.device_status()[0] == 0
     want = oracle.bwd(t["q"], t["k"], t["v"], t["do"], theta=w.theta, rotary_dim=w.R, pos_offset=w.pos_offset,
@@ -135,6 +138,9 @@ BWD_CASES = [
     (W("bsb_bigbird_no_cache", 1, 4, 2, 900, 128, theta=1e4, causal=False, backward=True, seed_id=425), lambda nb: bigbird_blocks(nb, seed=14), 0),
     (W("bsb_d64_norope", 1, 4, 4, 700, 64, rotary_dim=0, causal=False, backward=True, seed_id=426), lambda nb: bigbird_blocks(nb, seed=15), 2),
     (W("bsb_window_alibi", 1, 4, 2, 900, 128, theta=1e4, window=300, alibi=True, backward=True, seed_id=427), lambda nb: np.tril(np.ones((nb, nb), bool)), 2),
+    (W("bsb_onepass_bigbird_d64", 2, 6, 2, 1100, 64, theta=1e4, causal=False, backward=True, seed_id=428), lambda nb: bigbird_blocks(nb, seed=16), 3),
+    (W("bsb_onepass_bigbird_causal_d128", 1, 8, 2, 1100, 128, theta=5e5, backward=True, seed_id=429), lambda nb: bigbird_blocks(nb, seed=17, causal=True), 3),
+    (W("bsb_onepass_window_alibi", 1, 4, 2, 900, 128, theta=1e4, window=300, alibi=True, backward=True, seed_id=431), lambda nb: np.tril(np.ones((nb, nb), bool)), 3),
 ]
 
 
@@ -148,6 +154,7 @@ def test_block_sparse_backward_empty_lists_give_zero_gradient_rows():
     a = np.zeros((4, 4), dtype=bool)
     a[0, 1] = a[2, 0] = a[2, 3] = True      # query blocks 1, 3 and key block 2 are never touched
     run_bwd(w, a)
+    run_bwd(w, a, workspace_tier=3)
 
 
 def test_bigbird_n4096_forward_and_backward():
