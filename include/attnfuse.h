@@ -78,10 +78,10 @@ typedef enum {
                                   about 1.4 times the rounding error on rotated keys; forward only) */
     AF_OPT_BS_ROWPAIR = 3,     /* AF_BS_ROWPAIR, default 1: block-sparse forward with an odd GQA group gives a CTA two
                                   row blocks of one head when the caller supplied pair lists */
-    AF_OPT_BWD_ONEPASS = 4,    /* AF_BWD_ONEPASS, default 1: where the one-pass sequence of attnfuse_bwd applies (dense, workspace
+    AF_OPT_BWD_ONEPASS = 4,    /* AF_BWD_ONEPASS, default 1: where the one-pass sequence of attnfuse_bwd applies (workspace
                                   of attnfuse_bwd_onepass_workspace_bytes) it is taken where it measured faster: always at
                                   D = 64, at D = 128 when rows are short (at most 12 kept key tiles per query tile on
-                                  average); 2: whenever it applies; 0: never - always the two-kernel sequence, whose dQ is
+                                  average, and not over block lists); 2: whenever it applies; 0: never - always the two-kernel sequence, whose dQ is
                                   bit-reproducible */
     AF_OPT_COUNT_ = 5
 } af_option;
@@ -313,7 +313,7 @@ af_status attnfuse_decode(const af_shape* shape, const void* q, const void* k, c
  * kernels rotate everything they touch on chip.  Results of the three set-ups agree up to the bf16
  * rounding of a few rotated elements.  These three are deterministic: no atomics, every accumulator has one
  * owner and a fixed order of additions.
- * One-pass sequence (dense masks): with a workspace of attnfuse_bwd_onepass_workspace_bytes(shape) -
+ * One-pass sequence (dense masks and block lists): with a workspace of attnfuse_bwd_onepass_workspace_bytes(shape) -
  * the three pieces above followed by an fp32 accumulator of dQ (B*Hq*S*D*4 bytes) - and where option
  * AF_OPT_BWD_ONEPASS selects it, RoPE passes write both caches and ONE kernel per key tile forms dK, dV and its
  * share of dQ (five tile products per kept tile pair instead of seven; S and dP are not recomputed a second
