@@ -166,7 +166,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--extras", type=int, default=1, help="also time configs 3-5, the separate-RoPE arm and the sweep")
     ap.add_argument("--cpu-baseline", type=int, default=1)
-    ap.add_argument("--profile", default="", choices=["", "fwd", "hybrid", "bwd", "bwd2", "rope", "decode", "fwd_c3", "fwd_d64", "blocks", "fp8"],
+    ap.add_argument("--profile", default="", choices=["", "fwd", "hybrid", "bwd", "bwd2", "rope", "decode", "fwd_c3", "fwd_d64", "bwd_d64", "blocks", "fp8"],
                     help="run only a few launches of one path (for ncu captures) and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -277,6 +277,7 @@ def main():
         wl = {"fwd": synth.CONFIGS[1], "hybrid": synth.CONFIGS[1], "bwd": synth.CONFIGS[4], "bwd2": synth.CONFIGS[4],
               "rope": synth.CONFIGS[3], "fwd_c3": synth.CONFIGS[2],
               "fwd_d64": synth.Workload("gpt2_small_geometry_d64", 4, 12, 12, 4096, 64, theta=1.0e4, seed_id=51),
+              "bwd_d64": synth.Workload("gpt2_small_geometry_d64", 4, 12, 12, 4096, 64, theta=1.0e4, backward=True, seed_id=51),
               "blocks": synth.Workload("bigbird_d64_n4096", 4, 12, 12, 4096, 64, theta=1.0e4, causal=False, seed_id=53)}[args.profile]
         r, m, tb = specs(wl)
         t = {k: to_dev(v) for k, v in synth.draw_all(wl).items()}
@@ -296,8 +297,8 @@ def main():
                 af.fwd_blocks(t["q"], t["k"], t["v"], r, tb, m, wl.scale, bmask)
             else:
                 o_, l_ = af.fwd(t["q"], t["k"], t["v"], r, tb, m, wl.scale)
-                if args.profile in ("bwd", "bwd2"):   # bwd: the sequence the library picks (one-pass here); bwd2: two kernels
-                    with af.option(af.OPT_BWD_ONEPASS, 1 if args.profile == "bwd" else 0):
+                if args.profile in ("bwd", "bwd2", "bwd_d64"):   # the sequence the library picks (one-pass here); bwd2: two kernels
+                    with af.option(af.OPT_BWD_ONEPASS, 0 if args.profile == "bwd2" else 1):
                         af.bwd(t["q"], t["k"], t["v"], o_, l_, t["do"], r, tb, m, wl.scale)
         torch.cuda.synchronize()
         print(json.dumps({"profile": args.profile, "workload": wl.name, "device_status": af.device_status()[0]}))
