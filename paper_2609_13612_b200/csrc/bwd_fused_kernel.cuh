@@ -31,7 +31,16 @@
 // two-kernel one on every shape tried (0.691 -> 0.546 ms at B = 4, 12 heads, N = 4096).
 // Warp roles (512 threads): warp 0 TMA producer; warps 1, 2, 3 MMA issuers (T1 and dV; T2 and dK'; dQ'^T), one
 // per SM sub-partition; warps 4-7 read the dQ'^T partials out of TMEM and add them to global memory; warps 8-11
-// and 12-15 are the two gradient warpgroups.
+// and 12-15 are the two gradient warpgroups, one per column half.  A gradient warpgroup works in two phases per
+// tile (P^T from S^T, then dS^T from dP^T) and announces each on a barrier of its own, so that S^T of the next
+// tile is issued while dS^T is still being formed and dP^T of the next tile while the next P^T is.  A timeline of
+// the D = 64 kernel (4.4 k cycles per tile pair): phase P 1.5-2.3 k cycles for 64 columns (the exponentials of
+// both warpgroups share one special-function unit per sub-partition: 1 k cycles per tile pair is its floor, and
+// a microbenchmark of the phase alone gives 0.76 k for one warp per sub-partition, 1.1 k for two), phase dS
+// 0.9-1.1 k, the rest waits on the products.  Measured and not kept: both warpgroups on the same half with the
+// phases interleaved by half (each phase pays the TMEM load and store latencies again: 5.2 k cycles per pair);
+// working out the next tile's mask and addresses between the two phases (the warpgroups fall into step and the
+// shared exponential unit stretches phase P: 4.9 k).
 #pragma once
 #include "bwd_kernel.cuh"
 
@@ -49,8 +58,9 @@ struct BwdFusedSmem {
     static constexpr int OFF_STATS = OFF_DS + 2 * DS_HALF;
     static constexpr int OFF_BAR = OFF_STATS + 2 * 2 * 128 * 4;
     static constexpr int B_XFULL = 0, B_YFULL = 1, B_AFULL = 2, B_BFULL = B_AFULL + NST, B_EMPTY = B_BFULL + NST,
-                         B_TFULL = B_EMPTY + NST, B_PDS = B_TFULL + 2, B_DQFULL = B_PDS + 2, B_DSFREE = B_DQFULL + 2,
-                         B_T2FREE = B_DSFREE + 2, B_DONE = B_T2FREE + 2, N_BARS = B_DONE + 1;
+                         B_SFULL = B_EMPTY + NST, B_DPFULL = B_SFULL + 2, B_PRDY = B_DPFULL + 2, B_PDS = B_PRDY + 2,
+                         B_DQFULL = B_PDS + 2, B_DSFREE = B_DQFULL + 2, B_T2FREE = B_DSFREE + 2, B_DONE = B_T2FREE + 2,
+                         N_BARS = B_DONE + 1;
     static constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;
     static constexpr int NEEDED = OFF_MISC + 16;
     // The layout needs 1024-byte alignment (swizzle atoms).  The request leaves what room there is for rounding
@@ -61,25 +71,35 @@ struct BwdFusedSmem {
     static_assert(128 * STG_STRIDE * 4 <= 2 * NST * TILE, "staging buffer must fit in the stream stages");
 };
 
+// timeline stamps for tuning (compiled out unless AF_TRACE): as AF_BSTAMP, with the buffer's address read once per
+// thread (`trc`) so that a stamp costs a clock read and a store
+#ifdef AF_TRACE
+#define AF_FSTAMP(role, it, ph)                                                                  \
+    do {                                                                                         \
+        if (trc && (threadIdx.x & 31) == 0 && (it) < 64) trc[((role) * 64 + (it)) * 8 + (ph)] = clock64(); \
+    } while (0)
+#else
+#define AF_FSTAMP(role, it, ph) do { } while (0)
+#endif
+
+constexpr int kFusedLightRegs = 64, kFusedReduceRegs = 96, kFusedGradRegs = 176;
 constexpr uint32_t kFusedSmemCode = 0x40;   // status code: dynamic shared memory too misaligned for the layout
 
-// One 32-column pass of a gradient warpgroup in the one-pass kernel: as grad_pass32 of the dK/dV role, but dS^T
-// goes to shared memory (row = this thread's key, 16-byte chunks `chunk0`.. of its 128-byte row, swizzled).
+// The gradient warpgroups work on a half tile (64 streamed rows) in two phases, so that each of the two products
+// that feed them is re-issued for the next tile as soon as its own result has been consumed:
+//   phase P:  S^T half -> P^T (bf16 into TMEM for dV; fp32 kept in registers), after which T1's half is free;
+//   phase dS: dP^T half -> dS^T = P^T (dP^T - delta) to shared memory (row = this thread's key, 16-byte chunks
+//             `chunk0`.. of its 128-byte row, swizzled), after which T2's half is free.
 template <bool MASKED, bool ALIBI>
-__device__ __forceinline__ void grad_pass32_fused(uint32_t t1, uint32_t t2, int col0, uint32_t out_col, float scale_log2,
-                                                  float cbias, float sb, const float* s_nl2, const float* s_ndl, int mlo,
-                                                  uint32_t mn, uint32_t ds_row_addr, int row7, int chunk0) {
-    uint32_t s[32], dp[32], pk[16], dk[16];
-    tmem_ld32(t1 + col0, s);
-    tmem_ld32(t2 + col0, dp);
-    tmem_wait_ld();
+__device__ __forceinline__ void grad_phase_p32(uint32_t t1, int col0, uint32_t out_col, float scale_log2, float cbias, float sb,
+                                               const float* s_nl2, int mlo, uint32_t mn, uint32_t* s) {
+    // s: 32 columns of S^T already in registers; overwritten in place with the bits of the fp32 probabilities
+    uint32_t pk[16];
     const float2 sc2 = make_float2(scale_log2, scale_log2), cb2 = make_float2(cbias, cbias);
 #pragma unroll
     for (int e = 0; e < 32; e += 4) {
         const float4 a4 = *reinterpret_cast<const float4*>(s_nl2 + col0 + e);
-        const float4 b4 = *reinterpret_cast<const float4*>(s_ndl + col0 + e);
         const float2 nl[2] = {make_float2(a4.x, a4.y), make_float2(a4.z, a4.w)};
-        const float2 nd[2] = {make_float2(b4.x, b4.y), make_float2(b4.z, b4.w)};
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             const int c = e + 2 * u;
@@ -93,12 +113,29 @@ __device__ __forceinline__ void grad_pass32_fused(uint32_t t1, uint32_t t2, int 
                 pe.x = (static_cast<uint32_t>(col0 + c - mlo) < mn) ? pe.x : 0.f;
                 pe.y = (static_cast<uint32_t>(col0 + c + 1 - mlo) < mn) ? pe.y : 0.f;
             }
-            const float2 ds = __fmul2_rn(pe, __fadd2_rn(make_float2(__uint_as_float(dp[c]), __uint_as_float(dp[c + 1])), nd[u]));
+            s[c] = __float_as_uint(pe.x);
+            s[c + 1] = __float_as_uint(pe.y);
             pk[c >> 1] = pack_bf16x2(pe.x, pe.y);
-            dk[c >> 1] = pack_bf16x2(ds.x, ds.y);
         }
     }
     tmem_st16(t1 + out_col, pk);
+}
+
+__device__ __forceinline__ void grad_phase_ds32(const uint32_t* dp, int col0, const float* s_ndl, const uint32_t* pe_keep,
+                                                uint32_t ds_row_addr, int row7, int chunk0) {
+    uint32_t dk[16];
+#pragma unroll
+    for (int e = 0; e < 32; e += 4) {
+        const float4 b4 = *reinterpret_cast<const float4*>(s_ndl + col0 + e);
+        const float2 nd[2] = {make_float2(b4.x, b4.y), make_float2(b4.z, b4.w)};
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int c = e + 2 * u;
+            const float2 ds = __fmul2_rn(make_float2(__uint_as_float(pe_keep[c]), __uint_as_float(pe_keep[c + 1])),
+                                         __fadd2_rn(make_float2(__uint_as_float(dp[c]), __uint_as_float(dp[c + 1])), nd[u]));
+            dk[c >> 1] = pack_bf16x2(ds.x, ds.y);
+        }
+    }
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         const uint32_t a = ds_row_addr + (static_cast<uint32_t>((chunk0 + c) ^ row7) << 4);
@@ -157,17 +194,26 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
     }
     const int per_head = hi - lo + 1;
     const int n_it = per_head > 0 ? per_head * p.group : 0;
-    auto stream_head = [&](int n) { return xh * p.group + n / per_head; };
-    auto stream_row0 = [&](int n) {
-        const int pos = lo + n % per_head;
-        return (BS ? __ldg(p.bs_idx + bs_base + pos) : pos) * 128;
+    // Streamed tile n = (query head xh * group + n / per_head, position lo + n % per_head): every role walks the
+    // sequence with a cursor of its own (a division per tile sat on the gradient warpgroups' loop-carried chain).
+    struct Cursor {
+        int pos, head;
     };
+    const Cursor first{0, xh * p.group};
+    auto advance = [&](Cursor& c) {
+        if (++c.pos == per_head) {
+            c.pos = 0;
+            ++c.head;
+        }
+    };
+    auto row0_of = [&](const Cursor& c) { return (BS ? __ldg(p.bs_idx + bs_base + lo + c.pos) : lo + c.pos) * 128; };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::N_BARS; ++i) {
             uint32_t cnt = 1;
-            if (i == L::B_PDS || i == L::B_PDS + 1 || i == L::B_T2FREE || i == L::B_T2FREE + 1) cnt = 4;   // per-warp arrives
-            if (i == L::B_TFULL || i == L::B_TFULL + 1 || i == L::B_DSFREE || i == L::B_DSFREE + 1 || i == L::B_DONE ||
+            if (i == L::B_PDS || i == L::B_PDS + 1 || i == L::B_PRDY || i == L::B_PRDY + 1 || i == L::B_T2FREE || i == L::B_T2FREE + 1)
+                cnt = 4;   // per-warp arrives
+            if (i == L::B_DSFREE || i == L::B_DSFREE + 1 || i == L::B_DONE ||
                 (i >= L::B_EMPTY && i < L::B_EMPTY + NST))
                 cnt = 2;   // one arrival from each of two MMA issuers
             mbar_init(&bars[i], cnt);
@@ -183,9 +229,16 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+#ifdef AF_TRACE
+    long long* const trc = (blockIdx.x == 0 && blockIdx.y == 0) ? g_trace : nullptr;
+#endif
     grid_dep_wait();     // delta, the RoPE passes and the zeroed accumulator precede this grid in the stream
     grid_dep_launch();
+    if (warp == 0) AF_FSTAMP(5, 0, 0);
 
+    // register budgets per role (they sum to the 512 a scheduler's four warps share): the gradient warpgroups
+    // keep a half tile of probabilities next to a half tile of dP^T
+    if (warp < 4) setmaxnreg_dec<kFusedLightRegs>();
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -197,8 +250,10 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                 tma_load_4d(sX + bx * BOX_BYTES, &tm_x, &bars[L::B_XFULL], bx * BOX_COLS, x0, xh, b);
                 tma_load_4d(sY + bx * BOX_BYTES, &tm_y, &bars[L::B_YFULL], bx * BOX_COLS, x0, xh, b);
             }
+            Cursor cur = first;
             for (int n = 0; n < n_it; ++n) {
-                const int st = n % NST, ah = stream_head(n), a0 = stream_row0(n);
+                const int st = n % NST, ah = cur.head, a0 = row0_of(cur);
+                advance(cur);
                 if (!mbar_wait(&bars[L::B_EMPTY + st], ((n / NST) & 1) ^ 1, abort_flag, 41)) break;
                 mbar_arrive_expect_tx(&bars[L::B_AFULL + st], TILE);
                 mbar_arrive_expect_tx(&bars[L::B_BFULL + st], TILE);
@@ -229,7 +284,7 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                     if (kk == 0) mma_ss_lo<false>(t_dst + hf * 64, s_lo + off, r_lo + off, dhi, IDESC_TH);
                     else mma_ss_lo<true>(t_dst + hf * 64, s_lo + off, r_lo + off, dhi, IDESC_TH);
                 }
-                mma_commit(&bars[L::B_TFULL + hf]);
+                mma_commit(&bars[(who == 0 ? L::B_SFULL : L::B_DPFULL) + hf]);
             };
             auto wait_stream = [&](int n) {
                 const int st = n % NST;
@@ -250,8 +305,11 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                 const bool next = n + 1 < n_it;
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
-                    ok = mbar_wait(&bars[L::B_PDS + hf], n & 1, abort_flag, 45);
+                    AF_FSTAMP(who, n, hf * 4);
+                    // issuer 0 goes on when P^T of the half is in TMEM, issuer 1 when dS^T is in shared memory
+                    ok = mbar_wait(&bars[(who == 0 ? L::B_PRDY : L::B_PDS) + hf], n & 1, abort_flag, 45);
                     if (!ok) break;
+                    AF_FSTAMP(who, n, hf * 4 + 1);
                     tc_fence_after_sync();
                     if (who == 0) {
 #pragma unroll
@@ -276,8 +334,10 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                         if (ok && who == 1 && !kOwnDq) ok = mbar_wait(&bars[L::B_T2FREE + hf], n & 1, abort_flag, 46);
                         if (!ok) break;
                         tc_fence_after_sync();
+                        AF_FSTAMP(who, n, hf * 4 + 2);
                         issue_T(n + 1, hf);
                     }
+                    AF_FSTAMP(who, n, hf * 4 + 3);
                 }
                 if (!ok) break;
                 if (!next) mma_commit(&bars[L::B_DONE]);
@@ -292,10 +352,13 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
             for (int n = 0; ok && n < n_it; ++n) {
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
+                    AF_FSTAMP(6, n, hf * 4);
                     ok = mbar_wait(&bars[L::B_PDS + hf], n & 1, abort_flag, 48);
+                    AF_FSTAMP(6, n, hf * 4 + 1);
                     // (own buffers: the previous tile's partial of this half must have been read out)
                     if (ok && kOwnDq && n > 0) ok = mbar_wait(&bars[L::B_T2FREE + hf], (n - 1) & 1, abort_flag, 54);
                     if (!ok) break;
+                    AF_FSTAMP(6, n, hf * 4 + 2);
                     tc_fence_after_sync();
                     const uint32_t b_lo = desc_lo(smem_u32(sDS + hf * L::DS_HALF), 16);
                     const uint32_t dst = tmem_base + TDQ + hf * 64;
@@ -306,6 +369,7 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                     }
                     mma_commit(&bars[L::B_DQFULL + hf]);
                     mma_commit(&bars[L::B_DSFREE + hf]);
+                    AF_FSTAMP(6, n, hf * 4 + 3);
                 }
             }
         }
@@ -316,14 +380,19 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         // of each 32-lane quarter (row d in lane 32 (d / 16) + d % 16); the other 16 lanes of a warp hold nothing.
         const int d = D == 128 ? (warp & 3) * 32 + lane : (warp & 3) * 16 + (lane & 15);
         const bool has_row = D == 128 || lane < 16;
+        setmaxnreg_dec<kFusedReduceRegs>();
         const uint32_t tsrc = tmem_base + TDQ + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         bool ok = true;
+        Cursor cur = first;
         for (int n = 0; ok && n < n_it; ++n) {
-            const int ah = stream_head(n), a0 = stream_row0(n);
+            const int ah = cur.head, a0 = row0_of(cur);
+            advance(cur);
 #pragma unroll 1
             for (int hf = 0; hf < 2; ++hf) {
+                if (warp == 4) AF_FSTAMP(4, n, hf * 4);
                 ok = mbar_wait_warp(&bars[L::B_DQFULL + hf], n & 1, abort_flag, 49);
                 if (!ok) break;
+                if (warp == 4) AF_FSTAMP(4, n, hf * 4 + 1);
                 tc_fence_after_sync();
                 uint32_t v[64];
                 tmem_ld32(tsrc + hf * 64, v);
@@ -332,6 +401,7 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars[L::B_T2FREE + hf]);
+                if (warp == 4) AF_FSTAMP(4, n, hf * 4 + 2);
                 const int q0 = a0 + hf * 64;
                 float* dst = p.dq_acc + ((static_cast<size_t>(b) * p.Hq + ah) * p.S + q0) * D + d;
                 const int nq = min(64, p.S - q0);
@@ -344,10 +414,12 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                     for (int q = 0; q < 64; ++q)
                         if (has_row && q < nq) asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst + q * D), "f"(__uint_as_float(v[q])) : "memory");
                 }
+                if (warp == 4) AF_FSTAMP(4, n, hf * 4 + 3);
             }
         }
     } else if (warp >= 8) {
         // ------------------------------------------------------------ gradient warpgroups (one TMEM lane = key row per thread)
+        setmaxnreg_inc<kFusedGradRegs>();
         const int gtid = threadIdx.x - 256;
         const int hf = gtid >> 7;                    // column half (64 streamed rows) owned by this warpgroup
         const int tid = gtid & 127;
@@ -359,35 +431,43 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         const uint32_t ds_row_addr = smem_u32(sDS + hf * L::DS_HALF) + static_cast<uint32_t>(tid) * 128;
         bool ok = true;
         // per-column statistics of the streamed query tile; the loads for tile n + 1 are issued at the top of
-        // iteration n and stored to the other buffer after its passes (off the warpgroup's loop-carried chain)
+        // iteration n and stored to the other buffer after its passes (off the warpgroup's loop-carried chain).
+        // Nothing touches the loaded registers before store_stats: any arithmetic at the load would make the warp
+        // sit out the load's latency in front of the wait for S^T (measured: 1.1 k cycles per tile).
         float nx_l = 0.f, nx_d = 0.f, nx_slope = 0.f;
-        auto load_stats = [&](int n) {
-            const int ah = stream_head(n), a0 = stream_row0(n);
+        bool nx_in = false;
+        int nx_a0 = 0;
+        Cursor cur = first;
+        auto load_stats = [&]() {   // of the tile under the cursor, which then moves on
+            const int ah = cur.head, a0 = row0_of(cur);
+            advance(cur);
+            nx_a0 = a0;
             if (tid < 64) {
                 const int qi = a0 + hf * 64 + tid;
-                const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + qi;
-                nx_l = qi < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // kept negated
-                nx_d = qi < p.S ? -p.delta[r] : 0.f;
+                const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + min(qi, p.S - 1);
+                nx_in = qi < p.S;
+                nx_l = p.lse[r];
+                nx_d = p.delta[r];
             }
-            nx_slope = alibi ? p.slopes[ah] * kLog2e : 0.f;
+            if (alibi) nx_slope = p.slopes[ah];
         };
         auto store_stats = [&](int n) {
             if (tid < 64) {
                 float* dst = sStats + (n & 1) * 256 + hf * 64 + tid;
-                dst[0] = nx_l;
-                dst[128] = nx_d;
+                dst[0] = nx_in ? -nx_l * kLog2e : -INFINITY;   // kept negated
+                dst[128] = nx_in ? -nx_d : 0.f;
             }
         };
         if (n_it > 0) {
-            load_stats(0);
+            load_stats();
             store_stats(0);
         }
         for (int n = 0; ok && n < n_it; ++n) {
-            const int a0 = stream_row0(n);
+            const int a0 = nx_a0;
             float* sL2 = sStats + (n & 1) * 256;
             float* sDl = sL2 + 128;
-            const float my_slope2 = nx_slope;
-            if (n + 1 < n_it) load_stats(n + 1);
+            const float my_slope2 = nx_slope * kLog2e;
+            if (n + 1 < n_it) load_stats();
             const bool need_mask = tile_needs_mask(ms, a0, x0);
             int mlo = 0;
             uint32_t mn = 128;
@@ -395,28 +475,54 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
             const float sb = -my_slope2;
             const float bias_base = sb * static_cast<float>(a0 - xrow);
             // the previous tile's dS^T half must have been consumed by both MMAs that read it
-            ok = mbar_wait(&bars[L::B_DSFREE + hf], (n & 1) ^ 1, abort_flag, 50);
-            ok = bar_all(ok && mbar_wait(&bars[L::B_TFULL + hf], n & 1, abort_flag, 51), 1 + hf, 128);
+            if ((warp & 3) == 0) AF_FSTAMP(2 + hf, n, 0);
+            ok = bar_all(ok && mbar_wait(&bars[L::B_SFULL + hf], n & 1, abort_flag, 51), 1 + hf, 128);
             if (!ok) break;
+            if ((warp & 3) == 0) AF_FSTAMP(2 + hf, n, 1);
             tc_fence_after_sync();
+            // both 32-column chunks are requested up front; the second one lands while the first is worked on
+            uint32_t pe_keep[64];
+            tmem_ld32(tb + T1 + hf * 64, pe_keep);
+            tmem_wait_ld();
+            tmem_ld32(tb + T1 + hf * 64 + 32, pe_keep + 32);
 #pragma unroll
             for (int qt = 0; qt < 2; ++qt) {
                 const int col0 = hf * 64 + qt * 32;
                 const uint32_t out_col = hf * 64 + qt * 16;
                 const float cbias = fmaf(sb, static_cast<float>(col0), bias_base);
+                if (qt == 1) tmem_wait_ld();
                 if (alibi) {
-                    if (need_mask) grad_pass32_fused<true, true>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, mlo, mn, ds_row_addr, tid & 7, qt * 4);
-                    else grad_pass32_fused<false, true>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, mlo, mn, ds_row_addr, tid & 7, qt * 4);
+                    if (need_mask) grad_phase_p32<true, true>(tb + T1, col0, out_col, p.scale_log2, cbias, sb, sL2, mlo, mn, pe_keep + qt * 32);
+                    else grad_phase_p32<false, true>(tb + T1, col0, out_col, p.scale_log2, cbias, sb, sL2, mlo, mn, pe_keep + qt * 32);
                 } else {
-                    if (need_mask) grad_pass32_fused<true, false>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, mlo, mn, ds_row_addr, tid & 7, qt * 4);
-                    else grad_pass32_fused<false, false>(tb + T1, tb + T2, col0, out_col, p.scale_log2, cbias, sb, sL2, sDl, mlo, mn, ds_row_addr, tid & 7, qt * 4);
+                    if (need_mask) grad_phase_p32<true, false>(tb + T1, col0, out_col, p.scale_log2, cbias, sb, sL2, mlo, mn, pe_keep + qt * 32);
+                    else grad_phase_p32<false, false>(tb + T1, col0, out_col, p.scale_log2, cbias, sb, sL2, mlo, mn, pe_keep + qt * 32);
                 }
             }
             tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars[L::B_PRDY + hf]);
+            if ((warp & 3) == 0) AF_FSTAMP(2 + hf, n, 2);
+            // the previous tile's dS^T half must have been consumed by both MMAs that read it
+            ok = mbar_wait(&bars[L::B_DSFREE + hf], (n & 1) ^ 1, abort_flag, 50);
+            // (the vote keeps the warpgroup together: a warp that gave up must not leave the others at the barrier above)
+            ok = bar_all(ok && mbar_wait(&bars[L::B_DPFULL + hf], n & 1, abort_flag, 53), 1 + hf, 128);
+            if (!ok) break;
+            if ((warp & 3) == 0) AF_FSTAMP(2 + hf, n, 3);
+            tc_fence_after_sync();
+            uint32_t dp[64];
+            tmem_ld32(tb + T2 + hf * 64, dp);
+            tmem_wait_ld();
+            tmem_ld32(tb + T2 + hf * 64 + 32, dp + 32);
+            grad_phase_ds32(dp, hf * 64, sDl, pe_keep, ds_row_addr, tid & 7, 0);
+            tmem_wait_ld();
+            grad_phase_ds32(dp + 32, hf * 64 + 32, sDl, pe_keep + 32, ds_row_addr, tid & 7, 4);
             fence_proxy_async_smem();   // dS^T in shared memory is read by the tensor core's asynchronous proxy
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars[L::B_PDS + hf]);
+            if ((warp & 3) == 0) AF_FSTAMP(2 + hf, n, 4);
             if (n + 1 < n_it) store_stats(n + 1);   // (published by the named barrier at the top of the next iteration)
         }
         // (every thread of both warpgroups takes this barrier, also after a wait that gave up in one of them:
