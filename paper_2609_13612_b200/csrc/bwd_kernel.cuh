@@ -361,6 +361,19 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
         const int pos = lo + (DKV ? n % per_head : n);
         return (BS ? __ldg(p.bs_idx + bs_base + pos) : pos) * 128;
     };
+    // The producer and the gradient warpgroups walk the same sequence with a cursor instead: a division and a modulo
+    // per tile are some 350 cycles of dependent integer arithmetic each, on the warpgroups' loop-carried chain.
+    struct Cursor {
+        int pos, head;
+    };
+    const Cursor first{0, DKV ? xh * p.group : xh / p.group};
+    auto advance = [&](Cursor& c) {
+        if (++c.pos == per_head) {
+            c.pos = 0;
+            ++c.head;
+        }
+    };
+    auto row0_of = [&](const Cursor& c) { return (BS ? __ldg(p.bs_idx + bs_base + lo + c.pos) : lo + c.pos) * 128; };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::N_BARS; ++i) {
@@ -400,8 +413,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
                 tma_load_4d(sX + bx * BOX_BYTES, &tm_x, &bars[L::B_XFULL], bx * BOX_COLS, x0, xh, b);
                 tma_load_4d(sY + bx * BOX_BYTES, &tm_y, &bars[L::B_YFULL], bx * BOX_COLS, x0, xh, b);
             }
+            Cursor cur = first;
             for (int n = 0; n < n_it; ++n) {
-                const int st = n % NST, ah = stream_head(n), a0 = stream_row0(n);
+                const int st = n % NST, ah = cur.head, a0 = row0_of(cur);
+                advance(cur);
                 if (!mbar_wait(&bars[L::B_EMPTY + st], ((n / NST) & 1) ^ 1, abort_flag, 21)) break;
                 mbar_arrive_expect_tx(&bars[L::B_AFULL + st], TILE);
                 mbar_arrive_expect_tx(&bars[L::B_BFULL + st], TILE);
@@ -613,41 +628,48 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
         // DKV: per-column statistics of the streamed query tile (each warpgroup stages its own 64 columns).  The
         // global loads for tile n + 1 are issued at the top of iteration n and land in the other buffer after this
         // iteration's passes, so that their latency is off the loop-carried chain of the warpgroup.
+        // (Nothing touches the loaded registers before store_stats: arithmetic at the load would make the warp sit out
+        // the load's latency in front of its wait for the scores.)
         float nx_l = 0.f, nx_d = 0.f, nx_slope = 0.f;
-        auto load_stats = [&](int n) {
-            const int ah = stream_head(n), a0 = stream_row0(n);
+        bool nx_in = false;
+        Cursor cur_stats = first;
+        auto load_stats = [&]() {   // of the tile under the cursor, which then moves on
+            const int ah = cur_stats.head, a0 = row0_of(cur_stats);
+            advance(cur_stats);
             if (tid < 64) {
                 const int qi = a0 + hf * 64 + tid;
-                const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + qi;
-                if (GEN && p.relu) {
-                    const float cnt = qi < p.S ? p.lse[r] : 0.f;
-                    nx_l = cnt > 0.f ? 1.f / cnt : 0.f;
-                    nx_d = 0.f;
-                } else {
-                    nx_l = qi < p.S ? -p.lse[r] * kLog2e : -INFINITY;   // kept negated
-                    nx_d = qi < p.S ? -p.delta[r] : 0.f;
-                }
+                const size_t r = (static_cast<size_t>(b) * p.Hq + ah) * p.S + min(qi, p.S - 1);
+                nx_in = qi < p.S;
+                nx_l = p.lse[r];
+                if (!(GEN && p.relu)) nx_d = p.delta[r];
             }
-            nx_slope = alibi ? p.slopes[ah] * kLog2e : 0.f;
+            if (alibi) nx_slope = p.slopes[ah];
         };
         auto store_stats = [&](int n) {
             if (tid < 64) {
                 float* dst = sStats + (n & 1) * 256 + hf * 64 + tid;
-                dst[0] = nx_l;
-                dst[128] = nx_d;
+                if (GEN && p.relu) {
+                    dst[0] = (nx_in && nx_l > 0.f) ? 1.f / nx_l : 0.f;   // 1 / n_i
+                    dst[128] = 0.f;
+                } else {
+                    dst[0] = nx_in ? -nx_l * kLog2e : -INFINITY;   // kept negated
+                    dst[128] = nx_in ? -nx_d : 0.f;
+                }
             }
         };
         if (DKV && ok && n_it > 0) {
-            load_stats(0);
+            load_stats();
             store_stats(0);
         }
+        Cursor cur = first;
         for (int n = 0; ok && n < n_it; ++n) {
-            const int ah = stream_head(n), a0 = stream_row0(n);
+            const int ah = cur.head, a0 = row0_of(cur);
+            advance(cur);
             float* sL2 = sStats + (n & 1) * 256;
             float* sDl = sL2 + 128;
             if (DKV) {
-                my_slope2 = nx_slope;
-                if (n + 1 < n_it) load_stats(n + 1);
+                my_slope2 = nx_slope * kLog2e;
+                if (n + 1 < n_it) load_stats();
             }
             const int i0 = DKV ? a0 : x0, j0 = DKV ? x0 : a0;
             const bool need_mask = tile_needs_mask(ms, i0, j0);
