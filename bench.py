@@ -139,16 +139,18 @@ def run_reference(args, w):
         return
     cores = len(os.sched_getaffinity(0))
     per_step = max(1.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
-    vals, sample = [], ""
+    vals, secs, sample = [], [], ""
     for i in range(args.warmup + args.steps):
-        v, sample, _ = oracle_rate(w, per_step)
+        v, sample, dt = oracle_rate(w, per_step)
         if i >= args.warmup:
             vals.append(v)
+            secs.append(dt)
     value = float(np.mean(vals))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": None, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "ms_per_step": float(np.mean(secs)) * 1e3,   # one step = one bounded sample of the workload (see cpu_baseline.sample)
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "config": {"workload": w.name, "B": w.B, "Hq": w.Hq, "Hkv": w.Hkv, "S": w.S, "D": w.D,
                                         "variant": "rope(theta=%g)+causal" % w.theta},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
