@@ -83,7 +83,12 @@ typedef enum {
                                   D = 64, at D = 128 when rows are short (at most 12 kept key tiles per query tile on
                                   average, and not over block lists); 2: whenever it applies; 0: never - always the two-kernel sequence, whose dQ is
                                   bit-reproducible */
-    AF_OPT_COUNT_ = 5
+    AF_OPT_FWD_ALIBI_MMA = 5,  /* AF_FWD_ALIBI_MMA, default 1: the forward kernel adds the ALiBi term slope (j - i) with one
+                                  more K step of the score product (the slope split into two bf16 values, the key column
+                                  exact in bf16) instead of one fused multiply-add per score in the softmax warps - in the kernels that rotate
+                                  on chip, where it measured faster; 2: in every forward kernel; 0: never.  Not used by the additive_bias / relu_attention variants nor together with
+                                  AF_OPT_FWD_KEYS_BF16 (no shared memory left for the two small operand tiles) */
+    AF_OPT_COUNT_ = 6
 } af_option;
 af_status attnfuse_set_option(af_option option, int value);
 int       attnfuse_get_option(af_option option);

@@ -155,7 +155,7 @@ def version() -> int:
 
 
 # af_option values (include/attnfuse.h)
-OPT_FWD_QTILES, OPT_FWD_PAIR_HEADS, OPT_FWD_KEYS_BF16, OPT_BS_ROWPAIR, OPT_BWD_ONEPASS = range(5)
+OPT_FWD_QTILES, OPT_FWD_PAIR_HEADS, OPT_FWD_KEYS_BF16, OPT_BS_ROWPAIR, OPT_BWD_ONEPASS, OPT_FWD_ALIBI_MMA = range(6)
 
 
 def set_option(option: int, value: int) -> None:

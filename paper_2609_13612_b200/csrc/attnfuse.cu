@@ -145,6 +145,7 @@ constexpr OptionDef kOptionDefs[AF_OPT_COUNT_] = {
     {"AF_FWD_KEYS_BF16", 0},    // AF_OPT_FWD_KEYS_BF16
     {"AF_BS_ROWPAIR", 1},       // AF_OPT_BS_ROWPAIR
     {"AF_BWD_ONEPASS", 1},      // AF_OPT_BWD_ONEPASS
+    {"AF_FWD_ALIBI_MMA", 1},    // AF_OPT_FWD_ALIBI_MMA
 };
 std::atomic<int> g_options[AF_OPT_COUNT_];
 std::once_flag g_options_once;
@@ -292,6 +293,8 @@ af_status launch_fwd_variant(const CUtensorMap& tq, const CUtensorMap& tk, const
     if (allow_dynamic_smem(kern, L::BYTES, configured) != AF_OK) return AF_ERR_CUDA;
     // an even GQA group lets the two query tiles of a CTA be two heads of one kv head (same key range)
     p.pair_heads = (NQ == 2 && (p.group % 2) == 0 && opt(AF_OPT_FWD_PAIR_HEADS)) ? 1 : 0;
+    // (measured: +5 % at config 3 with the rotation warps at work, -1 % without them; option value 2 takes it there too)
+    p.alibi_mma = (L::HAS_AX && !GEN && p.slopes && (opt(AF_OPT_FWD_ALIBI_MMA) >= 2 || (ROPE && opt(AF_OPT_FWD_ALIBI_MMA) == 1))) ? 1 : 0;
     const int rows_per_cta = p.pair_heads ? BM : BM * NQ;
     p.n_row_blocks = (p.S + rows_per_cta - 1) / rows_per_cta;
     dim3 grid(p.pair_heads ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);
@@ -316,6 +319,8 @@ af_status launch_fwd_blocks_variant(const CUtensorMap& tq, const CUtensorMap& tk
     // NQ = 2: two heads of one kv head on the same row block (even GQA group), or - with pair lists - the row
     // blocks 2 rb and 2 rb + 1 of one head
     p.pair_heads = (NQ == 2 && !p.bs_rowpair) ? 1 : 0;
+    // (measured: +5 % at config 3 with the rotation warps at work, -1 % without them; option value 2 takes it there too)
+    p.alibi_mma = (L::HAS_AX && !GEN && p.slopes && (opt(AF_OPT_FWD_ALIBI_MMA) >= 2 || (ROPE && opt(AF_OPT_FWD_ALIBI_MMA) == 1))) ? 1 : 0;
     p.n_row_blocks = (p.S + BM - 1) / BM;
     if (p.bs_rowpair) p.n_row_blocks = (p.n_row_blocks + 1) / 2;
     dim3 grid(p.pair_heads ? p.B * p.Hq / 2 : p.B * p.Hq, p.n_row_blocks, 1);

@@ -41,6 +41,11 @@ struct FwdParams {
     const float* bias;
     long long bias_sb, bias_sh;
     int relu;              // Section 3.1, relu_attention: P = max(s, 0) / (kept pairs of the row) in place of the softmax
+    // ALiBi by the tensor core (set by the host when the layout has room for the operand tiles, see FwdSmem::HAS_AX):
+    // the term slope (j - i) is linear in the key column, so one more K step of the S product adds it - S += A B^T
+    // with A = [kb_hi, kb_lo, 0 ...] in every query row and B = [e, e, 0 ...] in key row e (kb = slope / c split
+    // into two bf16 values, e exact in bf16) - and the softmax warps run their plain straight-line code.
+    int alibi_mma;
 #ifdef AF_TRACE
     long long* trace;
 #endif
@@ -62,7 +67,13 @@ struct FwdSmem {
                          B_SFULL = B_VEMPTY + VS, B_PREADY = B_SFULL + 2 * NQ, B_ODONE = B_PREADY + 4 * NQ,   // SFULL: per column half; PREADY: per P part (up to 4)
                          B_TFULL = B_ODONE + NQ, B_TEMPTY = B_TFULL + 1, N_BARS = B_TEMPTY + 1;
     static constexpr int OFF_MISC = OFF_BAR + N_BARS * 8;
-    static constexpr int BYTES = OFF_MISC + 16 + 1024;  // + alignment slack
+    // operand tiles of the ALiBi K step: [128 rows x 16 columns] bf16, K-major, no swizzle (core matrices of 8 rows x
+    // 16 bytes; 128 bytes between the two core matrices of a row group, 256 bytes between row groups): one for the
+    // key side, one per query tile.  Left out where they do not fit (the TAB variant's table stage takes the room).
+    static constexpr int AX_TILE = 128 * 16 * 2;
+    static constexpr int OFF_AX = (OFF_MISC + 16 + 127) / 128 * 128;
+    static constexpr bool HAS_AX = OFF_AX + (NQ + 1) * AX_TILE + 1024 <= 232448;
+    static constexpr int BYTES = (HAS_AX ? OFF_AX + (NQ + 1) * AX_TILE : OFF_MISC + 16) + 1024;  // + alignment slack
 };
 
 // Optional timeline instrumentation for tuning (compiled out unless AF_TRACE is defined): one CTA
@@ -455,6 +466,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
+        const bool alibi_mma = L::HAS_AX && !GEN && p.alibi_mma && p.slopes != nullptr;
+        if (alibi_mma) {
+            // the operand tiles of the ALiBi K step, written by this warp (its lane 0 issues every MMA that reads them)
+            uint8_t* ax = smem + L::OFF_AX;
+            for (int c = lane; c < (NQ + 1) * (L::AX_TILE / 16); c += 32) {
+                const int tile = c / (L::AX_TILE / 16), cc = c % (L::AX_TILE / 16);
+                const int r = (cc >> 4) * 8 + (cc & 7);      // 16-byte chunk cc: row group cc / 16, K half (cc / 8) % 2, row cc % 8
+                uint32_t w0 = 0u;
+                if (((cc >> 3) & 1) == 0) {
+                    if (tile == 0) {
+                        w0 = pack_bf16x2(static_cast<float>(r), static_cast<float>(r));
+                    } else {
+                        const float kb = p.slopes[tile == 1 ? hq[0] : hq[NQ - 1]] * 1.4426950408889634f / p.scale_log2;
+                        const float hi = __bfloat162float(__float2bfloat16_rn(kb));
+                        w0 = pack_bf16x2(hi, kb - hi);
+                    }
+                }
+                *reinterpret_cast<uint4*>(ax + static_cast<size_t>(c) * 16) = make_uint4(w0, 0u, 0u, 0u);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+        }
         if (lane == 0) {
             const int B_KREADY = (ROPE && p.rot_k) ? L::B_KROT : L::B_KFULL;
             constexpr int B_QREADY = ROPE ? L::B_QROT : L::B_QFULL;
@@ -473,6 +506,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
                     if (kk == 0) mma_ss_lo<false>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
                     else mma_ss_lo<true>(d, q_lo + off, k_lo + off, dhi, IDESC_S);
+                }
+                if (alibi_mma) {
+                    const uint32_t ax = smem_u32(smem + L::OFF_AX);
+                    mma_ss_lo<true>(d, desc_lo(ax + (1 + q) * L::AX_TILE, 128), desc_lo(ax, 128), desc_hi_noswizzle(256), IDESC_S);
                 }
                 mma_commit(&bars[L::B_SFULL + 2 * q]);
             };
@@ -616,7 +653,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int i = i0[q] + row;
         const int bh = b * p.Hq + hq[q];
         const float slope2 = p.slopes ? p.slopes[hq[q]] * 1.4426950408889634f : 0.f;
-        const bool alibi = p.slopes != nullptr;
+        // (with the ALiBi K step the scores arrive with the term already in them)
+        const bool alibi = p.slopes != nullptr && !(L::HAS_AX && !GEN && p.alibi_mma);
         const float kb = slope2 / p.scale_log2;
         float m_run = -INFINITY, l_run = 0.f;
         bool ok = true;

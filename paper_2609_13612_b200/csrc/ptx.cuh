@@ -240,6 +240,10 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) 
 __device__ __forceinline__ uint32_t desc_hi(uint32_t sbo_bytes) {
     return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
 }
+// the same for an operand without swizzle (layout type 0: core matrices of 8 rows x 16 bytes, stored contiguously)
+__device__ __forceinline__ uint32_t desc_hi_noswizzle(uint32_t sbo_bytes) {
+    return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14);
+}
 
 // Arrive on `bar` once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {

@@ -68,6 +68,29 @@ def test_forward_keys_rotated_in_packed_bf16(w):
         run_case(w, lse_tol=2e-2)
 
 
+ALIBI_CASES = [w for w in SMALL if w.alibi] + [
+    W("alibi_gqa_d64", 2, 6, 2, 450, 64, theta=1e4, alibi=True, seed_id=171),
+    W("alibi_no_rope_window", 1, 4, 4, 390, 128, rotary_dim=0, window=130, alibi=True, seed_id=172),
+    W("alibi_odd_group", 1, 3, 1, 300, 128, theta=1e4, alibi=True, seed_id=173),
+]
+
+
+@pytest.mark.parametrize("w", ALIBI_CASES, ids=lambda w: w.name)
+def test_forward_alibi_in_the_softmax_warps(w):
+    """ALiBi has two implementations in the forward kernel: by default one more K step of the score product adds
+    slope (j - i) (run by every other ALiBi case of this suite); with the option off the softmax warps add it,
+    one fused multiply-add per score.  Both are held to the oracle."""
+    with af.option(af.OPT_FWD_ALIBI_MMA, 0):
+        run_case(w)
+
+
+@pytest.mark.parametrize("w", ALIBI_CASES, ids=lambda w: w.name)
+def test_forward_alibi_by_the_tensor_core(w):
+    assert af.get_option(af.OPT_FWD_ALIBI_MMA) == 1   # the default: in the kernels that rotate on chip
+    with af.option(af.OPT_FWD_ALIBI_MMA, 2):          # here: also without RoPE
+        run_case(w)
+
+
 @pytest.mark.parametrize("w", SMALL[3:8], ids=lambda w: w.name)
 def test_forward_small_one_query_tile_per_cta(w):
     with af.option(af.OPT_FWD_QTILES, 1):
