@@ -103,7 +103,8 @@ __device__ __forceinline__ void grad_phase_p32(uint32_t t1, int col0, uint32_t o
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
             const int c = e + 2 * u;
-            float2 t = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, __fadd2_rn(cb2, nl[u]));
+            // (without ALiBi the row's bias is zero: one packed add per column pair less)
+            float2 t = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, ALIBI ? __fadd2_rn(cb2, nl[u]) : nl[u]);
             if (ALIBI) {
                 t.x = fmaf(sb, static_cast<float>(c), t.x);
                 t.y = fmaf(sb, static_cast<float>(c + 1), t.y);
