@@ -304,7 +304,7 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                 // MN-major B operand of the accumulator MMAs: 16 streamed rows (2 KB) per K step
                 const uint32_t m_lo = desc_lo(smem_u32((who == 0 ? sB : sA) + st * TILE), BOX_BYTES);
                 const bool next = n + 1 < n_it;
-#pragma unroll
+#pragma unroll 1   // (rolled: half the issuer's loop code; the instruction path is the tightest resource of this kernel)
                 for (int hf = 0; hf < 2; ++hf) {
                     AF_FSTAMP(who, n, hf * 4);
                     // issuer 0 goes on when P^T of the half is in TMEM, issuer 1 when dS^T is in shared memory
@@ -351,7 +351,7 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
             const uint32_t dhi = desc_hi(1024);
             const uint32_t a_lo = desc_lo(smem_u32(sX), BOX_BYTES);   // MN-major: 16 key rows (2 KB) per K step
             for (int n = 0; ok && n < n_it; ++n) {
-#pragma unroll
+#pragma unroll 1   // (rolled: half the issuer's loop code; the instruction path is the tightest resource of this kernel)
                 for (int hf = 0; hf < 2; ++hf) {
                     AF_FSTAMP(6, n, hf * 4);
                     ok = mbar_wait(&bars[L::B_PDS + hf], n & 1, abort_flag, 48);
