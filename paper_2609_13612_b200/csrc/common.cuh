@@ -250,7 +250,7 @@ __device__ __forceinline__ void rotate_tile_tab(uint8_t* tile, const uint8_t* ta
     constexpr int ROW_BYTES = CP * 32;       // 2 R
     constexpr int NB = CP < 2 ? CP : 2;      // rows in flight per thread
     const int rg = tid / CP, cp = tid % CP;
-#pragma unroll
+#pragma unroll 1   // (rolled, like rotate_tile_fast)
     for (int k0 = 0; k0 < CP; k0 += NB) {
         uint4 lo[NB], hi[NB], c[NB], s[NB];
 #pragma unroll
