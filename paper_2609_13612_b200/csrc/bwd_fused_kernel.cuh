@@ -279,11 +279,10 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
             auto issue_T = [&](int n, int hf) {
                 const int st = n % NST;
                 const uint32_t r_lo = desc_lo(smem_u32((who == 0 ? sA : sB) + st * TILE) + hf * 64 * 128, 16);
-#pragma unroll
+#pragma unroll 2   // (partly rolled: loop code against issue slots per MMA)
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = ((kk >> 2) * BOX_BYTES + (kk & 3) * 32) >> 4;
-                    if (kk == 0) mma_ss_lo<false>(t_dst + hf * 64, s_lo + off, r_lo + off, dhi, IDESC_TH);
-                    else mma_ss_lo<true>(t_dst + hf * 64, s_lo + off, r_lo + off, dhi, IDESC_TH);
+                    mma_ss_lo_rt(t_dst + hf * 64, s_lo + off, r_lo + off, dhi, IDESC_TH, kk > 0 ? 1u : 0u);
                 }
                 mma_commit(&bars[(who == 0 ? L::B_SFULL : L::B_DPFULL) + hf]);
             };
@@ -363,11 +362,9 @@ attn_bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                     tc_fence_after_sync();
                     const uint32_t b_lo = desc_lo(smem_u32(sDS + hf * L::DS_HALF), 16);
                     const uint32_t dst = tmem_base + TDQ + hf * 64;
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        if (kk == 0) mma_ss_lo<false>(dst, a_lo + kk * 128, b_lo + kk * 128, dhi, IDESC_DQ);
-                        else mma_ss_lo<true>(dst, a_lo + kk * 128, b_lo + kk * 128, dhi, IDESC_DQ);
-                    }
+#pragma unroll 2
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_ss_lo_rt(dst, a_lo + kk * 128, b_lo + kk * 128, dhi, IDESC_DQ, kk > 0 ? 1u : 0u);
                     mma_commit(&bars[L::B_DQFULL + hf]);
                     mma_commit(&bars[L::B_DSFREE + hf]);
                     AF_FSTAMP(6, n, hf * 4 + 3);
