@@ -70,3 +70,23 @@ def test_no_cpu_fallback():
     q = torch.zeros(1, 1, 128, 128, dtype=torch.bfloat16)
     with pytest.raises(af.AttnFuseError):
         af.fwd(q, q, q, af.RopeSpec(), None, af.MaskSpec(), 0.1)
+
+
+def test_option_table_matches_the_header(libpath):
+    """Every af_option of the header exists in the library with the default the header states, the binding names the
+    same numbers, and a value set is the value read back (host-side table: no GPU needed)."""
+    import paper_2609_13612_b200 as af
+    src = open(os.path.join(ROOT, "include", "attnfuse.h")).read()
+    decl = re.findall(r"(AF_OPT_[A-Z0-9_]+)\s*=\s*(\d+),\s*/\*\s*(AF_[A-Z0-9_]+), default (\d+)", src)
+    count = int(re.search(r"AF_OPT_COUNT_\s*=\s*(\d+)", src).group(1))
+    assert len(decl) == count == 6
+    for name, number, _env, default in decl:
+        number, default = int(number), int(default)
+        assert getattr(af, name[3:]) == number, name           # AF_OPT_X in the header is OPT_X in the binding
+        if os.environ.get(_env) is None:
+            assert af.get_option(number) == default, name
+        with af.option(number, default + 1):
+            assert af.get_option(number) == default + 1
+        assert af.get_option(number) == (default if os.environ.get(_env) is None else af.get_option(number))
+    with pytest.raises(af.AttnFuseError):
+        af.set_option(count, 0)
